@@ -1,0 +1,266 @@
+// CPU oracle for the weight-quantised linear layer (int4/int8 asymmetric, group-quantised along K).
+//
+// THIS FILE IS TEST INFRASTRUCTURE.  It defines what the CUDA library must compute and is timed as
+// the CPU baseline; the product never calls it.  It shares no code, header, table or helper with
+// the CUDA path: every conversion (fp16 rounding included) is written out here a second time.
+//
+// Style: plain scalar loops in the order of the definitions, fp64 accumulation, no blocking, no
+// fusion.  The only parallelism is an optional OpenMP "for" over independent output rows.
+//
+// Pins (tests that hold each function to something other than itself):
+//   orc_quantize_w4 / w8   Eq. 1 end points and monotonicity, a hand-worked group, lossless
+//                          round-trip of exactly representable weights.
+//   orc_dequant            the same lossless round-trip (w_hat == w exactly).
+//   orc_linear_wa16        long-double triple loop over dequantised weights; subset-sum and
+//                          constant-q closed forms.
+//   orc_act_quant          hand-worked rows; a_q exact for integer-valued rows with amax = 127.
+//   orc_group_partials     Python-integer brute force.
+//   orc_linear_w4a8        the per-group identity  sum_k a*s*(q-z) = s*(sum a*q - z*sum a)  in
+//                          exact rational arithmetic; equality with orc_linear_wa16 when the
+//                          activations are exactly representable in int8.
+//   fp16 conversions       exhaustive round trip over all 65536 bit patterns and comparison with
+//                          numpy's float16 on random and boundary values.
+//
+// Readings of the paper taken here (the paper states Eq. 1 with symbols only):
+//   * clip_min = 0, clip_max = 15 (int4) or 255 (int8); codes are unsigned.
+//   * groups are `group` consecutive k of one weight row; per-channel means group == K.
+//   * scale s = fp16((w_max - w_min) / (clip_max - clip_min)); the code q is computed against the
+//     rounded s; the zero point is the real number z = fp16(-w_min / s), so w_hat = s * (q - z).
+//   * round() is round-half-to-even in fp32.
+//   * a group with w_max == w_min (or whose scale rounds to 0 in fp16) gets s = 1, q = 0,
+//     z = fp16(-w_min).  A scale or zero that overflows fp16 saturates at +-65504.
+//   * activations: per token, symmetric, a_q in [-127, 127], a_scale = amax / 127 in fp32.
+
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+extern "C" {
+
+// ---------------------------------------------------------------------------------------------
+// IEEE binary16 <-> binary32, written from the format definition (1 sign, 5 exponent, 10 fraction
+// bits, bias 15, subnormals below 2^-14).  Round to nearest, ties to even.
+// ---------------------------------------------------------------------------------------------
+float orc_f16_to_f32(uint16_t h) {
+    const int sign = (h >> 15) & 1;
+    const int e = (h >> 10) & 0x1F;
+    const int f = h & 0x3FF;
+    double v;
+    if (e == 0) {
+        v = std::ldexp((double)f, -24);  // subnormal: f * 2^-10 * 2^-14
+    } else if (e == 31) {
+        v = f ? (double)NAN : (double)INFINITY;
+    } else {
+        v = std::ldexp(1.0 + (double)f / 1024.0, e - 15);
+    }
+    return (float)(sign ? -v : v);
+}
+
+uint16_t orc_f32_to_f16(float x) {
+    uint32_t u;
+    std::memcpy(&u, &x, 4);
+    const uint16_t sign = (uint16_t)((u >> 16) & 0x8000u);
+    if (std::isnan(x)) return (uint16_t)(sign | 0x7E00u);
+    double a = std::fabs((double)x);
+    if (std::isinf(x)) return (uint16_t)(sign | 0x7C00u);
+    if (a == 0.0) return sign;
+    int ex;  // a = m * 2^ex with m in [0.5, 1)
+    (void)std::frexp(a, &ex);
+    int e = ex - 1;          // floor(log2 a)
+    if (e < -14) e = -14;    // subnormal range shares the exponent of the smallest normal
+    // spacing of representable numbers in this binade is 2^(e-10); nearbyint is half-to-even
+    double n = std::nearbyint(std::ldexp(a, 10 - e));
+    if (n >= 2048.0) {  // rounded up into the next binade
+        n = 1024.0;
+        e += 1;
+    }
+    if (e > 15) return (uint16_t)(sign | 0x7C00u);  // overflow -> infinity
+    if (n < 1024.0) return (uint16_t)(sign | (uint16_t)n);  // subnormal (e == -14) or zero
+    return (uint16_t)(sign | ((uint16_t)(e + 15) << 10) | ((uint16_t)n - 1024u));
+}
+
+static inline uint16_t f16_saturating(float v) {
+    uint16_t h = orc_f32_to_f16(v);
+    if ((h & 0x7FFFu) == 0x7C00u) h = (uint16_t)((h & 0x8000u) | 0x7BFFu);  // +-65504
+    return h;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Eq. 1 (asymmetric quantisation), applied per (row n, group g of `group` consecutive k).
+// q: [N, K] codes in [0, clip_max]; scale_bits / zero_bits: [N, K/group] fp16 bit patterns.
+// ---------------------------------------------------------------------------------------------
+static void quantize_rows(const float* W, int N, int K, int group, int clip_max, uint8_t* q,
+                          uint16_t* scale_bits, uint16_t* zero_bits) {
+    const int G = K / group;
+#pragma omp parallel for schedule(static)
+    for (int n = 0; n < N; ++n) {
+        for (int g = 0; g < G; ++g) {
+            const float* w = W + (size_t)n * K + (size_t)g * group;
+            float mn = w[0], mx = w[0];
+            for (int k = 1; k < group; ++k) {
+                if (w[k] < mn) mn = w[k];
+                if (w[k] > mx) mx = w[k];
+            }
+            const float s32 = (mx - mn) / (float)clip_max;
+            uint16_t sb = f16_saturating(s32);
+            float s = orc_f16_to_f32(sb);
+            uint8_t* qo = q + (size_t)n * K + (size_t)g * group;
+            if (!(s > 0.0f)) {  // constant group, or a range too small for fp16
+                sb = 0x3C00u;   // 1.0
+                s = 1.0f;
+                for (int k = 0; k < group; ++k) qo[k] = 0;
+            } else {
+                for (int k = 0; k < group; ++k) {
+                    const float t = (w[k] - mn) / s;
+                    int c = (int)std::rintf(t);
+                    if (c < 0) c = 0;
+                    if (c > clip_max) c = clip_max;
+                    qo[k] = (uint8_t)c;
+                }
+            }
+            scale_bits[(size_t)n * G + g] = sb;
+            zero_bits[(size_t)n * G + g] = f16_saturating(-mn / s);
+        }
+    }
+}
+
+void orc_quantize_w4(const float* W, int N, int K, int group, uint8_t* q, uint16_t* scale_bits,
+                     uint16_t* zero_bits) {
+    quantize_rows(W, N, K, group, 15, q, scale_bits, zero_bits);
+}
+
+// int8 per-channel variant (the LM head): one group per row, codes in [0, 255].
+void orc_quantize_w8(const float* W, int N, int K, uint8_t* q, uint16_t* scale_bits,
+                     uint16_t* zero_bits) {
+    quantize_rows(W, N, K, K, 255, q, scale_bits, zero_bits);
+}
+
+// w_hat[n, k] = s[n, g] * (q[n, k] - z[n, g]) in fp64.
+void orc_dequant(const uint8_t* q, const uint16_t* scale_bits, const uint16_t* zero_bits, int N,
+                 int K, int group, double* w_hat) {
+    const int G = K / group;
+#pragma omp parallel for schedule(static)
+    for (int n = 0; n < N; ++n)
+        for (int k = 0; k < K; ++k) {
+            const double s = (double)orc_f16_to_f32(scale_bits[(size_t)n * G + k / group]);
+            const double z = (double)orc_f16_to_f32(zero_bits[(size_t)n * G + k / group]);
+            w_hat[(size_t)n * K + k] = s * ((double)q[(size_t)n * K + k] - z);
+        }
+}
+
+// Weight-only path (W4A16 / W8A16): y[m, n] = sum_k x[m, k] * w_hat[n, k], fp64, natural k order.
+// x holds the activation values already widened (exactly) to fp32.
+void orc_linear_wa16(const float* x, const uint8_t* q, const uint16_t* scale_bits,
+                     const uint16_t* zero_bits, int M, int N, int K, int group, double* y) {
+    const int G = K / group;
+#pragma omp parallel for schedule(static)
+    for (int n = 0; n < N; ++n) {
+        for (int m = 0; m < M; ++m) {
+            double acc = 0.0;
+            for (int k = 0; k < K; ++k) {
+                const double s = (double)orc_f16_to_f32(scale_bits[(size_t)n * G + k / group]);
+                const double z = (double)orc_f16_to_f32(zero_bits[(size_t)n * G + k / group]);
+                const double w_hat = s * ((double)q[(size_t)n * K + k] - z);
+                acc += (double)x[(size_t)m * K + k] * w_hat;
+            }
+            y[(size_t)m * N + n] = acc;
+        }
+    }
+}
+
+// Dynamic per-token symmetric int8 activation quantisation.
+//   amax = max_k |x[m, k]|;  a_q = clamp(rint(x * (127 / amax)), -127, 127);  a_scale = amax / 127
+//   A_g[m, g] = sum_{k in g} a_q[m, k]   (the factor of the zero-point correction)
+void orc_act_quant(const float* x, int M, int K, int group, int8_t* a_q, float* a_scale,
+                   int32_t* A_g) {
+    const int G = K / group;
+#pragma omp parallel for schedule(static)
+    for (int m = 0; m < M; ++m) {
+        const float* xr = x + (size_t)m * K;
+        float amax = 0.0f;
+        for (int k = 0; k < K; ++k) {
+            const float a = std::fabs(xr[k]);
+            if (a > amax) amax = a;
+        }
+        if (amax == 0.0f) {
+            for (int k = 0; k < K; ++k) a_q[(size_t)m * K + k] = 0;
+            for (int g = 0; g < G; ++g) A_g[(size_t)m * G + g] = 0;
+            a_scale[m] = 0.0f;
+            continue;
+        }
+        const float inv = 127.0f / amax;
+        for (int k = 0; k < K; ++k) {
+            int c = (int)std::rintf(xr[k] * inv);
+            if (c < -127) c = -127;
+            if (c > 127) c = 127;
+            a_q[(size_t)m * K + k] = (int8_t)c;
+        }
+        for (int g = 0; g < G; ++g) {
+            int32_t s = 0;
+            for (int k = 0; k < group; ++k) s += a_q[(size_t)m * K + (size_t)g * group + k];
+            A_g[(size_t)m * G + g] = s;
+        }
+        a_scale[m] = amax / 127.0f;
+    }
+}
+
+// Integer group partials: P[m, n, g] = sum_{k in g} a_q[m, k] * q[n, k]   (exact, int32).
+void orc_group_partials(const int8_t* a_q, const uint8_t* q, int M, int N, int K, int group,
+                        int32_t* P) {
+    const int G = K / group;
+#pragma omp parallel for schedule(static)
+    for (int n = 0; n < N; ++n)
+        for (int m = 0; m < M; ++m)
+            for (int g = 0; g < G; ++g) {
+                int32_t acc = 0;
+                for (int k = g * group; k < (g + 1) * group; ++k)
+                    acc += (int32_t)a_q[(size_t)m * K + k] * (int32_t)q[(size_t)n * K + k];
+                P[((size_t)m * N + n) * G + g] = acc;
+            }
+}
+
+// W4A8: y[m, n] = a_scale[m] * sum_g s[n, g] * (P[m, n, g] - z[n, g] * A_g[m, g]), fp64.
+void orc_linear_w4a8(const float* x, const uint8_t* q, const uint16_t* scale_bits,
+                     const uint16_t* zero_bits, int M, int N, int K, int group, double* y) {
+    const int G = K / group;
+    int8_t* a_q = new int8_t[(size_t)M * K];
+    float* a_scale = new float[M];
+    int32_t* A_g = new int32_t[(size_t)M * G];
+    orc_act_quant(x, M, K, group, a_q, a_scale, A_g);
+#pragma omp parallel for schedule(static)
+    for (int n = 0; n < N; ++n)
+        for (int m = 0; m < M; ++m) {
+            double acc = 0.0;
+            for (int g = 0; g < G; ++g) {
+                int32_t P = 0;
+                for (int k = g * group; k < (g + 1) * group; ++k)
+                    P += (int32_t)a_q[(size_t)m * K + k] * (int32_t)q[(size_t)n * K + k];
+                const double s = (double)orc_f16_to_f32(scale_bits[(size_t)n * G + g]);
+                const double z = (double)orc_f16_to_f32(zero_bits[(size_t)n * G + g]);
+                acc += s * ((double)P - z * (double)A_g[(size_t)m * G + g]);
+            }
+            y[(size_t)m * N + n] = (double)a_scale[m] * acc;
+        }
+    delete[] a_q;
+    delete[] a_scale;
+    delete[] A_g;
+}
+
+int orc_num_threads(void) {
+#ifdef _OPENMP
+    int n = 1;
+#pragma omp parallel
+    {
+#pragma omp single
+        n = omp_get_num_threads();
+    }
+    return n;
+#else
+    return 1;
+#endif
+}
+
+}  // extern "C"
