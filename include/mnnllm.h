@@ -1,0 +1,166 @@
+/*
+ * mnnllm.h - C ABI of the B200 (sm_100a) weight-quantised linear layer.
+ *
+ * The operation is the Linear operator of Section 5.1: activations x [M, K] ("[e, l]") times
+ * weights W [N, K] ("[h, l]") give y [M, N] ("[e, h]"), with W stored as asymmetric int4 (or int8)
+ * codes produced by Eq. 1 of Section 4.2 and dequantised inside the kernel.  On a GPU the
+ * activations stay floating point (W4A16 / W8A16); the W4A8 path first quantises them to int8 per
+ * token so that integer matrix instructions can be used (Section 4.2).
+ *
+ * Conventions shared by every entry point
+ *   - Pointers marked "host" are ordinary CPU memory, pointers marked "device" are CUDA global
+ *     memory of the current device.  The caller owns every buffer; the library never allocates or
+ *     frees device memory and keeps no reference after a call returns.
+ *   - Matrices are dense row-major.  W is [N, K]; groups are `group` consecutive k of one row,
+ *     G = K / group groups per row.
+ *   - GPU entry points only enqueue work on `stream` (a cudaStream_t passed as void*) and return at
+ *     once; errors reported are argument and launch errors.  Results are ready when the stream
+ *     reaches that point.
+ *   - Device pointers must be 16-byte aligned; the packed weight buffer must be 128-byte aligned.
+ *   - There is no CPU fallback: on a device that is not compute capability 10.x the GPU entry
+ *     points return MNNLLM_ERR_UNSUPPORTED.
+ *   - Every function returns MNNLLM_OK (0) on success; nothing is written on an argument error.
+ */
+#ifndef MNNLLM_H_
+#define MNNLLM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    MNNLLM_OK = 0,
+    MNNLLM_ERR_INVALID_ARG = 1, /* null pointer, non-positive size, bad header */
+    MNNLLM_ERR_UNSUPPORTED = 2, /* group size, dtype, shape or device not supported */
+    MNNLLM_ERR_ALIGNMENT = 3,   /* a pointer breaks the alignment rules above */
+    MNNLLM_ERR_CUDA = 4,        /* a CUDA runtime call failed (launch, attribute, ...) */
+    MNNLLM_ERR_TIMEOUT = 5,     /* a bounded device-side wait gave up (see mnnllm_read_status) */
+    MNNLLM_ERR_WORKSPACE = 6    /* workspace pointer null or too small */
+} mnnllm_status;
+
+typedef enum { MNNLLM_F16 = 0, MNNLLM_BF16 = 1, MNNLLM_F32 = 2 } mnnllm_dtype;
+
+const char* mnnllm_status_string(int status);
+
+/* ------------------------------------------------------------------------------------------------
+ * Weight packing (host only, done once when the model is loaded).
+ *
+ * Eq. 1 (Section 4.2) with clip_min = 0 and clip_max = 15, applied to every group of one row:
+ *     scale = fp16((w_max - w_min) / 15),   q = clamp(round((w - w_min) / scale), 0, 15),
+ *     zero  = fp16(-w_min / scale),         so that  w ~ scale * (q - zero).
+ * round() is fp32 round-half-to-even and the division uses the fp16-rounded scale.  A group whose
+ * range is zero (or rounds to a zero scale) gets scale = 1, q = 0, zero = fp16(-w_min); scale and
+ * zero saturate at +-65504.
+ *
+ * The packed buffer is position independent (it may be copied anywhere, to the device as is).
+ * Layout: a 128-byte header (magic, version, bits, N, K, group, counts, strides), then one record
+ * per block of 16 rows, each record a run of chunks of 512 k (the last chunk of a row may be
+ * shorter).  A chunk holds its codes as 512-byte slabs of 16 rows x 64 k - 16 bytes for each of the
+ * 32 threads of a warp: thread 4r+c owns k = 16c..16c+15 of rows r and r+8, nibbles interleaved so
+ * that `word & 0x0F0F0F0F` and `(word >> 4) & 0x0F0F0F0F` are four consecutive k each - followed by
+ * the chunk's (scale, zero) fp16 pairs ordered [row][group].  Every chunk is a contiguous,
+ * 16-byte-aligned run, i.e. one bulk copy.  Rows beyond N in the last block are stored as q = 0,
+ * scale = 0, zero = 0.
+ * ---------------------------------------------------------------------------------------------- */
+
+/* Bytes needed for the packed form of an [N, K] matrix; 0 if the arguments are not supported
+ * (N, K >= 1, group in {64, 128}, K a multiple of group). */
+size_t mnnllm_packed_size_w4(int N, int K, int group);
+
+/* W: host, fp32 [N, K].  packed_out: host, mnnllm_packed_size_w4(N, K, group) bytes, written in full. */
+int mnnllm_pack_w4(const float* W, int N, int K, int group, void* packed_out);
+
+/* Inverse of the reorder, for parity checks: reads a packed buffer (host) and writes the codes
+ * q [N, K] (one per byte, 0..15) and the fp16 bit patterns of scale and zero, each [N, G].
+ * N, K and group are taken from the header. */
+int mnnllm_unpack_w4(const void* packed, uint8_t* q, uint16_t* scale_bits, uint16_t* zero_bits);
+
+/* Reads N, K and group of a packed buffer (host); any output pointer may be null. */
+int mnnllm_packed_info(const void* packed, int* N, int* K, int* group, int* bits);
+
+/* int8 per-channel variant (Section 4.2: the LM head is kept in int8): Eq. 1 with clip_max = 255,
+ * one group per row (group = K), codes stored as unsigned bytes, scale and zero fp16 per row. */
+size_t mnnllm_packed_size_w8(int N, int K);
+int mnnllm_pack_w8(const float* W, int N, int K, void* packed_out);
+int mnnllm_unpack_w8(const void* packed, uint8_t* q, uint16_t* scale_bits, uint16_t* zero_bits);
+
+/* ------------------------------------------------------------------------------------------------
+ * W4A16: y[m, n] = sum_g scale[n, g] * sum_{k in g} (q[n, k] - zero[n, g]) * x[m, k]
+ * (Section 4.2, "W4A16 ... on GPUs"; Section 5.1 for the operand shapes).  Accumulation is fp32.
+ *
+ *   x       device, fp16 [M, K]
+ *   packed  device, a buffer written by mnnllm_pack_w4 for the same N, K, group
+ *   y       device, fp16 [M, N] (or the dtype given to the _ex form), overwritten
+ *   M >= 1  any M is accepted; the kernel is built for decode (M <= 8 per pass over the weights)
+ *
+ * The header of `packed` lives in device memory and is not read by the host: N, K and group are
+ * the caller's statement of what was packed.
+ * ---------------------------------------------------------------------------------------------- */
+int mnnllm_linear_w4a16(const void* x, const void* packed, void* y, int M, int N, int K, int group,
+                        void* stream);
+
+/* Same with explicit dtypes: x_dtype MNNLLM_F16; y_dtype MNNLLM_F16, MNNLLM_BF16 or MNNLLM_F32
+ * (fp32 logits for the LM head). */
+int mnnllm_linear_w4a16_ex(const void* x, const void* packed, void* y, int M, int N, int K, int group,
+                           int x_dtype, int y_dtype, void* stream);
+
+/* Several independent W4A16 problems that share M (for example q, k, v of one layer, or gate and
+ * up) in ONE launch.  `problems` is a host array of `count` (1..MNNLLM_MAX_BATCH) descriptors; it
+ * is copied into the launch and may be reused when the call returns. */
+#define MNNLLM_MAX_BATCH 8
+typedef struct {
+    const void* x;      /* device fp16 [M, K] */
+    const void* packed; /* device */
+    void* y;            /* device [M, N] of y_dtype */
+    int N, K, group;
+    int y_dtype;
+} mnnllm_w4a16_problem;
+int mnnllm_linear_w4a16_batch(const mnnllm_w4a16_problem* problems, int count, int M, void* stream);
+
+/* W8A16 with per-channel int8 weights packed by mnnllm_pack_w8. */
+int mnnllm_linear_w8a16(const void* x, const void* packed, void* y, int M, int N, int K, int y_dtype,
+                        void* stream);
+
+/* ------------------------------------------------------------------------------------------------
+ * W4A8 (Section 4.2: "activation values are quantized to int8 ... W4A8"):
+ *   per token m:   amax = max_k |x[m, k]|,  a_scale[m] = amax / 127,
+ *                  a_q[m, k] = clamp(round(x[m, k] * (127 / amax)), -127, 127)   (0 if amax == 0)
+ *   per group g:   P[m, n, g] = sum_{k in g} a_q[m, k] * q[n, k]      (int32, exact)
+ *                  A[m, g]    = sum_{k in g} a_q[m, k]
+ *   y[m, n] = a_scale[m] * sum_g scale[n, g] * (P[m, n, g] - zero[n, g] * A[m, g])    (fp32)
+ *
+ *   x          device [M, K] of x_dtype (MNNLLM_F16 or MNNLLM_BF16)
+ *   y          device [M, N] of y_dtype, overwritten
+ *   workspace  device scratch of at least mnnllm_workspace_size_w4a8(M, N, K, group) bytes,
+ *              256-byte aligned; holds a_q, a_scale, A between the two kernels.  Contents are
+ *              undefined afterwards; two calls that may overlap on the GPU need separate workspaces.
+ * ---------------------------------------------------------------------------------------------- */
+size_t mnnllm_workspace_size_w4a8(int M, int N, int K, int group);
+int mnnllm_linear_w4a8(const void* x, const void* packed, void* y, int M, int N, int K, int group,
+                       int x_dtype, int y_dtype, void* workspace, size_t workspace_bytes, void* stream);
+
+/* The activation quantiser alone (first kernel of the W4A8 path), writing caller-owned outputs:
+ * a_q int8 [M, K], a_scale fp32 [M], A int32 [M, G]. */
+int mnnllm_quantize_activations(const void* x, int x_dtype, int M, int K, int group, int8_t* a_q,
+                                float* a_scale, int32_t* A, void* stream);
+
+/* Parity/debug form of the W4A8 path: runs the same tensor-core main loop and stores every int32
+ * group partial, P device int32 [M, N, G], together with a_q, a_scale and A as above. */
+int mnnllm_debug_w4a8_partials(const void* x, int x_dtype, const void* packed, int32_t* P, int8_t* a_q,
+                               float* a_scale, int32_t* A, int M, int N, int K, int group, void* stream);
+
+/* Device-side waits in the kernels are bounded; one that gives up records a code in a status word
+ * instead of spinning.  This call synchronises `stream`, reads the word, clears it and returns
+ * MNNLLM_OK or MNNLLM_ERR_TIMEOUT (detail, if not null, receives the raw word). */
+int mnnllm_read_status(void* stream, uint32_t* detail);
+
+/* 1 if the current CUDA device can run the kernels (compute capability 10.x), else 0. */
+int mnnllm_device_supported(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MNNLLM_H_ */

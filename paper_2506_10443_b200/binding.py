@@ -1,0 +1,228 @@
+"""ctypes binding of ``libmnnllm_b200.so``: the same names as ``include/mnnllm.h`` without the
+``mnnllm_`` prefix, argument marshalling only.  Device buffers are passed as ``torch.Tensor`` (their
+``data_ptr()`` is used) or as raw integer addresses; streams as ``torch.cuda.Stream``, a raw
+``cudaStream_t`` integer, or ``None`` for torch's current stream.
+
+There is no fallback: if the library has not been built, importing this module raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence, Tuple
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libmnnllm_b200.so")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        "libmnnllm_b200.so is missing: build it with `python -m paper_2506_10443_b200.build` "
+        "(there is no CPU or PyTorch fallback)")
+
+lib = ctypes.CDLL(LIB_PATH)
+
+F16, BF16, F32 = 0, 1, 2
+OK = 0
+MAX_BATCH = 8
+_c = ctypes
+_P = _c.c_void_p
+
+
+class MnnllmError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        lib.mnnllm_status_string.restype = _c.c_char_p
+        super().__init__("%s: %s (status %d)" % (where, lib.mnnllm_status_string(status).decode(), status))
+
+
+class _Problem(_c.Structure):
+    _fields_ = [("x", _P), ("packed", _P), ("y", _P), ("N", _c.c_int), ("K", _c.c_int), ("group", _c.c_int),
+                ("y_dtype", _c.c_int)]
+
+
+def _sig(name, restype, argtypes):
+    f = getattr(lib, name)
+    f.restype = restype
+    f.argtypes = argtypes
+    return f
+
+
+_sig("mnnllm_status_string", _c.c_char_p, [_c.c_int])
+_sig("mnnllm_packed_size_w4", _c.c_size_t, [_c.c_int, _c.c_int, _c.c_int])
+_sig("mnnllm_pack_w4", _c.c_int, [_P, _c.c_int, _c.c_int, _c.c_int, _P])
+_sig("mnnllm_unpack_w4", _c.c_int, [_P, _P, _P, _P])
+_sig("mnnllm_packed_info", _c.c_int, [_P, _P, _P, _P, _P])
+_sig("mnnllm_packed_size_w8", _c.c_size_t, [_c.c_int, _c.c_int])
+_sig("mnnllm_pack_w8", _c.c_int, [_P, _c.c_int, _c.c_int, _P])
+_sig("mnnllm_unpack_w8", _c.c_int, [_P, _P, _P, _P])
+_sig("mnnllm_linear_w4a16", _c.c_int, [_P, _P, _P, _c.c_int, _c.c_int, _c.c_int, _c.c_int, _P])
+_sig("mnnllm_linear_w4a16_ex", _c.c_int,
+     [_P, _P, _P, _c.c_int, _c.c_int, _c.c_int, _c.c_int, _c.c_int, _c.c_int, _P])
+_sig("mnnllm_linear_w4a16_batch", _c.c_int, [_c.POINTER(_Problem), _c.c_int, _c.c_int, _P])
+_sig("mnnllm_linear_w8a16", _c.c_int, [_P, _P, _P, _c.c_int, _c.c_int, _c.c_int, _c.c_int, _P])
+_sig("mnnllm_workspace_size_w4a8", _c.c_size_t, [_c.c_int, _c.c_int, _c.c_int, _c.c_int])
+_sig("mnnllm_linear_w4a8", _c.c_int,
+     [_P, _P, _P, _c.c_int, _c.c_int, _c.c_int, _c.c_int, _c.c_int, _c.c_int, _P, _c.c_size_t, _P])
+_sig("mnnllm_quantize_activations", _c.c_int, [_P, _c.c_int, _c.c_int, _c.c_int, _c.c_int, _P, _P, _P, _P])
+_sig("mnnllm_debug_w4a8_partials", _c.c_int,
+     [_P, _c.c_int, _P, _P, _P, _P, _P, _c.c_int, _c.c_int, _c.c_int, _c.c_int, _P])
+_sig("mnnllm_read_status", _c.c_int, [_P, _c.POINTER(_c.c_uint32)])
+_sig("mnnllm_device_supported", _c.c_int, [])
+
+EXPORTS = [
+    "mnnllm_status_string", "mnnllm_packed_size_w4", "mnnllm_pack_w4", "mnnllm_unpack_w4", "mnnllm_packed_info",
+    "mnnllm_packed_size_w8", "mnnllm_pack_w8", "mnnllm_unpack_w8", "mnnllm_linear_w4a16", "mnnllm_linear_w4a16_ex",
+    "mnnllm_linear_w4a16_batch", "mnnllm_linear_w8a16", "mnnllm_workspace_size_w4a8", "mnnllm_linear_w4a8",
+    "mnnllm_quantize_activations", "mnnllm_debug_w4a8_partials", "mnnllm_read_status", "mnnllm_device_supported",
+]
+
+
+def _ptr(t) -> int:
+    if t is None:
+        return 0
+    if isinstance(t, int):
+        return t
+    if isinstance(t, np.ndarray):
+        return t.ctypes.data
+    return int(t.data_ptr())  # torch.Tensor
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        import torch
+        return int(torch.cuda.current_stream().cuda_stream)
+    if isinstance(stream, int):
+        return stream
+    return int(stream.cuda_stream)
+
+
+def _check(status: int, where: str) -> None:
+    if status != OK:
+        raise MnnllmError(status, where)
+
+
+# ---- host side ---------------------------------------------------------------------------------
+def packed_size_w4(N: int, K: int, group: int) -> int:
+    return int(lib.mnnllm_packed_size_w4(N, K, group))
+
+
+def pack_w4(W: np.ndarray, group: int) -> np.ndarray:
+    """fp32 [N, K] host weights -> packed uint8 host buffer (128-byte aligned)."""
+    W = np.ascontiguousarray(W, dtype=np.float32)
+    N, K = W.shape
+    size = packed_size_w4(N, K, group)
+    if size == 0:
+        raise MnnllmError(2, "packed_size_w4(%d, %d, %d)" % (N, K, group))
+    out = aligned_empty(size)
+    _check(lib.mnnllm_pack_w4(_ptr(W), N, K, group, _ptr(out)), "pack_w4")
+    return out
+
+
+def unpack_w4(packed: np.ndarray) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
+    N, K, group, bits = packed_info(packed)
+    q = np.empty((N, K), np.uint8)
+    s = np.empty((N, K // group), np.uint16)
+    z = np.empty((N, K // group), np.uint16)
+    _check(lib.mnnllm_unpack_w4(_ptr(packed), _ptr(q), _ptr(s), _ptr(z)), "unpack_w4")
+    return q, s, z
+
+
+def packed_info(packed: np.ndarray) -> Tuple[int, int, int, int]:
+    v = [_c.c_int(0) for _ in range(4)]
+    _check(lib.mnnllm_packed_info(_ptr(packed), *[_c.addressof(x) for x in v]), "packed_info")
+    return tuple(int(x.value) for x in v)
+
+
+def packed_size_w8(N: int, K: int) -> int:
+    return int(lib.mnnllm_packed_size_w8(N, K))
+
+
+def pack_w8(W: np.ndarray) -> np.ndarray:
+    W = np.ascontiguousarray(W, dtype=np.float32)
+    N, K = W.shape
+    size = packed_size_w8(N, K)
+    if size == 0:
+        raise MnnllmError(2, "packed_size_w8(%d, %d)" % (N, K))
+    out = aligned_empty(size)
+    _check(lib.mnnllm_pack_w8(_ptr(W), N, K, _ptr(out)), "pack_w8")
+    return out
+
+
+def unpack_w8(packed: np.ndarray) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
+    N, K, group, bits = packed_info(packed)
+    q = np.empty((N, K), np.uint8)
+    s = np.empty((N, 1), np.uint16)
+    z = np.empty((N, 1), np.uint16)
+    _check(lib.mnnllm_unpack_w8(_ptr(packed), _ptr(q), _ptr(s), _ptr(z)), "unpack_w8")
+    return q, s, z
+
+
+def aligned_empty(nbytes: int, align: int = 128) -> np.ndarray:
+    """Uninitialised uint8 host array whose address is a multiple of ``align``."""
+    raw = np.empty(nbytes + align, np.uint8)
+    off = (-raw.ctypes.data) % align
+    return raw[off:off + nbytes]
+
+
+# ---- device side -------------------------------------------------------------------------------
+def device_supported() -> bool:
+    return bool(lib.mnnllm_device_supported())
+
+
+def linear_w4a16(x, packed, y, M: int, N: int, K: int, group: int, stream=None) -> None:
+    _check(lib.mnnllm_linear_w4a16(_ptr(x), _ptr(packed), _ptr(y), M, N, K, group, _stream(stream)), "linear_w4a16")
+
+
+def linear_w4a16_ex(x, packed, y, M, N, K, group, x_dtype=F16, y_dtype=F16, stream=None) -> None:
+    _check(lib.mnnllm_linear_w4a16_ex(_ptr(x), _ptr(packed), _ptr(y), M, N, K, group, x_dtype, y_dtype,
+                                      _stream(stream)), "linear_w4a16_ex")
+
+
+def make_batch(problems: Sequence[dict]):
+    """Marshals a list of dicts (x, packed, y, N, K, group, y_dtype) into the C array once, so that a
+    benchmark loop can re-issue the same launch without Python-side allocation."""
+    arr = (_Problem * len(problems))()
+    for a, p in zip(arr, problems):
+        a.x, a.packed, a.y = _ptr(p["x"]), _ptr(p["packed"]), _ptr(p["y"])
+        a.N, a.K, a.group, a.y_dtype = p["N"], p["K"], p["group"], p.get("y_dtype", F16)
+    return arr
+
+
+def linear_w4a16_batch(problems, M: int, stream=None) -> None:
+    arr = problems if isinstance(problems, _c.Array) else make_batch(problems)
+    _check(lib.mnnllm_linear_w4a16_batch(arr, len(arr), M, _stream(stream)), "linear_w4a16_batch")
+
+
+def linear_w8a16(x, packed, y, M, N, K, y_dtype=F16, stream=None) -> None:
+    _check(lib.mnnllm_linear_w8a16(_ptr(x), _ptr(packed), _ptr(y), M, N, K, y_dtype, _stream(stream)), "linear_w8a16")
+
+
+def workspace_size_w4a8(M: int, N: int, K: int, group: int) -> int:
+    return int(lib.mnnllm_workspace_size_w4a8(M, N, K, group))
+
+
+def linear_w4a8(x, packed, y, M, N, K, group, workspace, workspace_bytes, x_dtype=F16, y_dtype=F16,
+                stream=None) -> None:
+    _check(lib.mnnllm_linear_w4a8(_ptr(x), _ptr(packed), _ptr(y), M, N, K, group, x_dtype, y_dtype, _ptr(workspace),
+                                  workspace_bytes, _stream(stream)), "linear_w4a8")
+
+
+def quantize_activations(x, M, K, group, a_q, a_scale, A, x_dtype=F16, stream=None) -> None:
+    _check(lib.mnnllm_quantize_activations(_ptr(x), x_dtype, M, K, group, _ptr(a_q), _ptr(a_scale), _ptr(A),
+                                           _stream(stream)), "quantize_activations")
+
+
+def debug_w4a8_partials(x, packed, P, a_q, a_scale, A, M, N, K, group, x_dtype=F16, stream=None) -> None:
+    _check(lib.mnnllm_debug_w4a8_partials(_ptr(x), x_dtype, _ptr(packed), _ptr(P), _ptr(a_q), _ptr(a_scale), _ptr(A),
+                                          M, N, K, group, _stream(stream)), "debug_w4a8_partials")
+
+
+def read_status(stream=None) -> int:
+    """Synchronises the stream and returns the device status word (0 = no bounded wait gave up)."""
+    detail = _c.c_uint32(0)
+    st = lib.mnnllm_read_status(_stream(stream), _c.byref(detail))
+    if st not in (0, 5):
+        raise MnnllmError(st, "read_status")
+    return int(detail.value)

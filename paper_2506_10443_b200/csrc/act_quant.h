@@ -1,0 +1,14 @@
+// Launch wrapper of the per-token int8 activation quantiser (internal to the library).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/mnnllm.h"
+
+namespace mnnllm {
+
+// x [M, K] (fp16 or bf16) -> a_q int8 [M, K], a_scale fp32 [M], A int32 [M, K / group].
+cudaError_t act_quant_launch(const void* x, int x_dtype, int M, int K, int group, int8_t* a_q, float* a_scale,
+                             int32_t* A, cudaStream_t stream);
+
+}  // namespace mnnllm

@@ -1,0 +1,208 @@
+// C-ABI entry points of the weight-only (W4A16 / W8A16) decode path: argument checks, the launch
+// plan (how rows and k-chunks are spread over warps, CTAs and clusters) and the kernel launches.
+#include <cuda_fp16.h>
+
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+
+#include "common.h"
+#include "gemv.h"
+
+namespace mnnllm {
+
+__device__ uint32_t g_status_word = 0;
+
+static int g_cc_major[64];
+static bool g_cc_known[64];
+static uint32_t* g_status_ptr[64];
+
+int device_is_supported() {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+    if (!g_cc_known[dev]) {
+        int major = 0;
+        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return 0;
+        g_cc_major[dev] = major;
+        g_cc_known[dev] = true;
+    }
+    return g_cc_major[dev] == 10;
+}
+
+uint32_t* status_word_ptr() {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    if (!g_status_ptr[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_status_word) != cudaSuccess) return nullptr;
+        g_status_ptr[dev] = (uint32_t*)p;
+    }
+    return g_status_ptr[dev];
+}
+
+namespace {
+
+struct Plan {
+    int CS, WC, SR, RBI, stages;
+};
+
+// How the quanta (16 rows x 512 k) of a launch are spread: WC warps of a CTA take different
+// k-chunks, SR groups of warps take different row blocks, a cluster of CS CTAs splits K further
+// when there are too few row blocks to occupy the GPU, and each warp walks RBI row blocks per
+// k-chunk so that the activation fragments it builds are reused.
+Plan make_plan(int nb_total, int nc_max, int group, int MP, int bits = 4) {
+    Plan p;
+    p.CS = 1;
+    while (p.CS < 8 && nb_total * p.CS < 120 && p.CS * 2 <= nc_max) p.CS *= 2;
+    p.WC = (nc_max + p.CS - 1) / p.CS;
+    if (p.WC > kGemvMaxWarps) p.WC = kGemvMaxWarps;
+    p.SR = kGemvMaxWarps / p.WC;
+    while (p.SR > 1 && nb_total * p.CS < kNumSMs * p.SR) --p.SR;
+    p.RBI = nb_total / (p.SR * kNumSMs);
+    p.RBI = p.RBI < 1 ? 1 : (p.RBI > kGemvMaxRBI ? kGemvMaxRBI : p.RBI);
+    p.stages = 3;
+    if (const char* env = std::getenv("MNNLLM_GEMV_PLAN")) {  // tuning override: "CS,WC,SR,RBI,stages"
+        int v[5];
+        if (std::sscanf(env, "%d,%d,%d,%d,%d", &v[0], &v[1], &v[2], &v[3], &v[4]) == 5) {
+            if (v[0] >= 1 && v[0] <= 8) p.CS = v[0];
+            if (v[1] >= 1 && v[1] <= kGemvMaxWarps) p.WC = v[1];
+            if (v[2] >= 1 && v[1] * v[2] <= kGemvMaxWarps) p.SR = v[2];
+            if (v[3] >= 1 && v[3] <= kGemvMaxRBI) p.RBI = v[3];
+            if (v[4] >= 1 && v[4] <= kGemvMaxStages) p.stages = v[4];
+        }
+    }
+    auto smem = [&](int st) {
+        return bits == 4 ? gemv_w4a16_smem(group, MP, p.WC * p.SR, p.SR, st) : gemv_w8a16_smem(p.WC * p.SR, p.SR, st);
+    };
+    while (p.stages > 1 && smem(p.stages) > 220 * 1024) --p.stages;
+    return p;
+}
+
+int check_problem(const mnnllm_w4a16_problem& q, int M) {
+    if (!q.x || !q.packed || !q.y || M < 1 || q.N < 1 || q.K < 1) return MNNLLM_ERR_INVALID_ARG;
+    if ((q.group != 64 && q.group != 128) || q.K % q.group != 0) return MNNLLM_ERR_UNSUPPORTED;
+    if (q.y_dtype != MNNLLM_F16 && q.y_dtype != MNNLLM_BF16 && q.y_dtype != MNNLLM_F32) return MNNLLM_ERR_UNSUPPORTED;
+    if (((uintptr_t)q.x & 15) || ((uintptr_t)q.y & 15) || ((uintptr_t)q.packed & 127)) return MNNLLM_ERR_ALIGNMENT;
+    return MNNLLM_OK;
+}
+
+int run_batch(const mnnllm_w4a16_problem* problems, int count, int M, cudaStream_t stream) {
+    if (!problems || count < 1 || count > MNNLLM_MAX_BATCH) return MNNLLM_ERR_INVALID_ARG;
+    const int group = problems[0].group;
+    for (int i = 0; i < count; ++i) {
+        const int st = check_problem(problems[i], M);
+        if (st != MNNLLM_OK) return st;
+        if (problems[i].group != group) return MNNLLM_ERR_UNSUPPORTED;
+    }
+    if (!device_is_supported()) return MNNLLM_ERR_UNSUPPORTED;
+    uint32_t* status = status_word_ptr();
+    if (!status) return MNNLLM_ERR_CUDA;
+
+    int nb_total = 0, nc_max = 0;
+    for (int i = 0; i < count; ++i) {
+        const W4Geometry g = w4_geometry(problems[i].N, problems[i].K, group);
+        nb_total += g.n_row_blocks;
+        nc_max = g.n_chunks > nc_max ? g.n_chunks : nc_max;
+    }
+    // tokens are processed in passes of at most 8 (one pass over the weights each)
+    for (int m0 = 0; m0 < M; m0 += 8) {
+        const int m = (M - m0) < 8 ? (M - m0) : 8;
+        const int MP = m <= 1 ? 1 : (m <= 2 ? 2 : (m <= 4 ? 4 : 8));
+        const Plan plan = make_plan(nb_total, nc_max, group, MP);
+        GemvLaunch L;
+        std::memset(&L, 0, sizeof(L));
+        L.count = count; L.M = m; L.WC = plan.WC; L.SR = plan.SR; L.stages = plan.stages;
+        int clusters = 0;
+        for (int i = 0; i < count; ++i) {
+            const mnnllm_w4a16_problem& q = problems[i];
+            const W4Geometry g = w4_geometry(q.N, q.K, group);
+            GemvProblem& P = L.prob[i];
+            const size_t ybytes = q.y_dtype == MNNLLM_F32 ? 4 : 2;
+            P.packed = (const uint8_t*)q.packed;
+            P.x = (const __half*)q.x + (size_t)m0 * q.K;
+            P.y = (uint8_t*)q.y + (size_t)m0 * q.N * ybytes;
+            P.N = q.N; P.K = q.K;
+            P.NB = g.n_row_blocks; P.NC = g.n_chunks; P.NS = g.n_slabs;
+            P.RBI = plan.RBI;
+            P.cluster_begin = clusters;
+            P.y_dtype = q.y_dtype;
+            P.row_block_bytes = g.row_block_bytes;
+            clusters += (g.n_row_blocks + plan.SR * plan.RBI - 1) / (plan.SR * plan.RBI);
+        }
+        if (gemv_w4a16_launch(L, group, MP, clusters, plan.CS, status, stream) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return MNNLLM_ERR_CUDA;
+        }
+    }
+    return MNNLLM_OK;
+}
+
+}  // namespace
+}  // namespace mnnllm
+
+using namespace mnnllm;
+
+extern "C" {
+
+int mnnllm_device_supported(void) { return device_is_supported(); }
+
+int mnnllm_read_status(void* stream, uint32_t* detail) {
+    if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return MNNLLM_ERR_CUDA;
+    uint32_t* p = status_word_ptr();
+    if (!p) return MNNLLM_ERR_CUDA;
+    uint32_t v = 0, zero = 0;
+    if (cudaMemcpy(&v, p, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return MNNLLM_ERR_CUDA;
+    if (v && cudaMemcpy(p, &zero, 4, cudaMemcpyHostToDevice) != cudaSuccess) return MNNLLM_ERR_CUDA;
+    if (detail) *detail = v;
+    return v ? MNNLLM_ERR_TIMEOUT : MNNLLM_OK;
+}
+
+int mnnllm_linear_w4a16_batch(const mnnllm_w4a16_problem* problems, int count, int M, void* stream) {
+    return run_batch(problems, count, M, (cudaStream_t)stream);
+}
+
+int mnnllm_linear_w8a16(const void* x, const void* packed, void* y, int M, int N, int K, int y_dtype, void* stream) {
+    if (!x || !packed || !y || M < 1 || N < 1 || K < 1) return MNNLLM_ERR_INVALID_ARG;
+    if (K % kSlabK8 != 0) return MNNLLM_ERR_UNSUPPORTED;
+    if (y_dtype != MNNLLM_F16 && y_dtype != MNNLLM_BF16 && y_dtype != MNNLLM_F32) return MNNLLM_ERR_UNSUPPORTED;
+    if (((uintptr_t)x & 15) || ((uintptr_t)y & 15) || ((uintptr_t)packed & 127)) return MNNLLM_ERR_ALIGNMENT;
+    if (!device_is_supported()) return MNNLLM_ERR_UNSUPPORTED;
+    uint32_t* status = status_word_ptr();
+    if (!status) return MNNLLM_ERR_CUDA;
+    const W8Geometry g = w8_geometry(N, K);
+    const Plan plan = make_plan(g.n_row_blocks, g.n_chunks, 0, 8, 8);
+    const size_t ybytes = y_dtype == MNNLLM_F32 ? 4 : 2;
+    for (int m0 = 0; m0 < M; m0 += 8) {
+        GemvLaunch L;
+        std::memset(&L, 0, sizeof(L));
+        L.count = 1; L.M = (M - m0) < 8 ? (M - m0) : 8; L.WC = plan.WC; L.SR = plan.SR; L.stages = plan.stages;
+        GemvProblem& P = L.prob[0];
+        P.packed = (const uint8_t*)packed;
+        P.x = (const __half*)x + (size_t)m0 * K;
+        P.y = (uint8_t*)y + (size_t)m0 * N * ybytes;
+        P.N = N; P.K = K; P.NB = g.n_row_blocks; P.NC = g.n_chunks; P.NS = g.n_slabs;
+        P.RBI = plan.RBI; P.cluster_begin = 0; P.y_dtype = y_dtype;
+        P.row_block_bytes = g.row_block_bytes; P.table_offset = g.table_offset;
+        const int clusters = (g.n_row_blocks + plan.SR * plan.RBI - 1) / (plan.SR * plan.RBI);
+        if (gemv_w8a16_launch(L, clusters, plan.CS, status, (cudaStream_t)stream) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return MNNLLM_ERR_CUDA;
+        }
+    }
+    return MNNLLM_OK;
+}
+
+int mnnllm_linear_w4a16_ex(const void* x, const void* packed, void* y, int M, int N, int K, int group, int x_dtype,
+                           int y_dtype, void* stream) {
+    if (x_dtype != MNNLLM_F16) return x_dtype == MNNLLM_BF16 || x_dtype == MNNLLM_F32 ? MNNLLM_ERR_UNSUPPORTED
+                                                                                     : MNNLLM_ERR_INVALID_ARG;
+    mnnllm_w4a16_problem p;
+    p.x = x; p.packed = packed; p.y = y; p.N = N; p.K = K; p.group = group; p.y_dtype = y_dtype;
+    return run_batch(&p, 1, M, (cudaStream_t)stream);
+}
+
+int mnnllm_linear_w4a16(const void* x, const void* packed, void* y, int M, int N, int K, int group, void* stream) {
+    return mnnllm_linear_w4a16_ex(x, packed, y, M, N, K, group, MNNLLM_F16, MNNLLM_F16, stream);
+}
+
+}  // extern "C"

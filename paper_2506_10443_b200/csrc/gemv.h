@@ -1,0 +1,44 @@
+// Host/device interface of the decode GEMV kernels (internal to the library).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/mnnllm.h"
+#include "layout.h"
+
+namespace mnnllm {
+
+constexpr int kGemvMaxWarps = 8;    // warps per CTA
+constexpr int kGemvMaxStages = 4;   // ring slots per warp
+constexpr int kGemvMaxRBI = 8;      // 16-row blocks a warp walks through per k-chunk
+constexpr int kNumSMs = 148;
+
+struct GemvProblem {
+    const uint8_t* packed;  // start of the packed buffer (header included)
+    const __half* x;        // [M, K]
+    void* y;                // [M, N]
+    int N, K;
+    int NB, NC, NS;         // 16-row blocks, 512-k chunks, slabs per row
+    int RBI;                // row blocks per warp and chunk
+    int cluster_begin;      // first cluster of this problem in the launch
+    int y_dtype;
+    unsigned long long row_block_bytes;
+    unsigned long long table_offset;  // W8: per-row (scale, zero) table, from the buffer start
+};
+
+struct GemvLaunch {
+    GemvProblem prob[MNNLLM_MAX_BATCH];
+    int count;
+    int M;       // tokens (<= MP of the instantiation)
+    int WC, SR;  // warps per CTA = WC (k-chunk lanes) * SR (row-block lanes)
+    int stages;
+};
+
+size_t gemv_w4a16_smem(int group, int MP, int W, int SR, int S);
+cudaError_t gemv_w4a16_launch(const GemvLaunch& L, int group, int MP, int n_clusters, int CS, uint32_t* status,
+                              cudaStream_t stream);
+
+size_t gemv_w8a16_smem(int W, int SR, int S);
+cudaError_t gemv_w8a16_launch(const GemvLaunch& L, int n_clusters, int CS, uint32_t* status, cudaStream_t stream);
+
+}  // namespace mnnllm
