@@ -44,12 +44,31 @@ namespace {
 
 struct Plan {
     int CS, WC, SR, RBI, stages;
+    int clusters;  // total clusters of the launch (persistent: about one resident set)
 };
+
+// Resident CTAs per SM, asked of the runtime once per configuration and cached.
+int cached_occupancy(int bits, int group, int MP, int W, int SR, int S) {
+    struct Entry { int key[6]; int occ; };
+    static Entry cache[64];
+    static int n_cached = 0;
+    const int key[6] = {bits, group, MP, W, SR, S};
+    for (int i = 0; i < n_cached; ++i)
+        if (!std::memcmp(cache[i].key, key, sizeof(key))) return cache[i].occ;
+    int occ = bits == 4 ? gemv_w4a16_occupancy(group, MP, W, SR, S) : gemv_w8a16_occupancy(W, SR, S);
+    if (occ < 1) occ = 1;
+    if (n_cached < 64) {
+        std::memcpy(cache[n_cached].key, key, sizeof(key));
+        cache[n_cached++].occ = occ;
+    }
+    return occ;
+}
 
 // How the quanta (16 rows x 512 k) of a launch are spread: WC warps of a CTA take different
 // k-chunks, SR groups of warps take different row blocks, a cluster of CS CTAs splits K further
-// when there are too few row blocks to occupy the GPU, and each warp walks RBI row blocks per
-// k-chunk so that the activation fragments it builds are reused.
+// when there are too few row blocks to occupy the GPU.  The grid is persistent: about as many
+// CTAs as fit on the GPU at once, each walking an even share of the row blocks in rounds of
+// SR * RBI blocks, so that the activation fragments a warp builds are reused RBI times.
 Plan make_plan(int nb_total, int nc_max, int group, int MP, int bits = 4) {
     Plan p;
     p.CS = 1;
@@ -58,24 +77,49 @@ Plan make_plan(int nb_total, int nc_max, int group, int MP, int bits = 4) {
     if (p.WC > kGemvMaxWarps) p.WC = kGemvMaxWarps;
     p.SR = kGemvMaxWarps / p.WC;
     while (p.SR > 1 && nb_total * p.CS < kNumSMs * p.SR) --p.SR;
-    p.RBI = nb_total / (p.SR * kNumSMs);
-    p.RBI = p.RBI < 1 ? 1 : (p.RBI > kGemvMaxRBI ? kGemvMaxRBI : p.RBI);
     p.stages = 3;
-    if (const char* env = std::getenv("MNNLLM_GEMV_PLAN")) {  // tuning override: "CS,WC,SR,RBI,stages"
-        int v[5];
-        if (std::sscanf(env, "%d,%d,%d,%d,%d", &v[0], &v[1], &v[2], &v[3], &v[4]) == 5) {
+    p.RBI = 0;
+    int forced_clusters = 0;
+    if (const char* env = std::getenv("MNNLLM_GEMV_PLAN")) {  // tuning override: "CS,WC,SR,RBI,stages[,clusters]"
+        int v[6] = {0, 0, 0, 0, 0, 0};
+        if (std::sscanf(env, "%d,%d,%d,%d,%d,%d", &v[0], &v[1], &v[2], &v[3], &v[4], &v[5]) >= 5) {
             if (v[0] >= 1 && v[0] <= 8) p.CS = v[0];
             if (v[1] >= 1 && v[1] <= kGemvMaxWarps) p.WC = v[1];
             if (v[2] >= 1 && v[1] * v[2] <= kGemvMaxWarps) p.SR = v[2];
             if (v[3] >= 1 && v[3] <= kGemvMaxRBI) p.RBI = v[3];
             if (v[4] >= 1 && v[4] <= kGemvMaxStages) p.stages = v[4];
+            if (v[5] >= 1) forced_clusters = v[5];
         }
     }
     auto smem = [&](int st) {
         return bits == 4 ? gemv_w4a16_smem(group, MP, p.WC * p.SR, p.SR, st) : gemv_w8a16_smem(p.WC * p.SR, p.SR, st);
     };
     while (p.stages > 1 && smem(p.stages) > 220 * 1024) --p.stages;
+    const int occ = cached_occupancy(bits, group, MP, p.WC * p.SR, p.SR, p.stages);
+    int clusters = kNumSMs * occ / p.CS;
+    const int max_useful = (nb_total + p.SR - 1) / p.SR;  // at least SR row blocks per cluster
+    if (clusters > max_useful) clusters = max_useful;
+    if (forced_clusters) clusters = forced_clusters;
+    if (clusters < 1) clusters = 1;
+    p.clusters = clusters;
+    if (p.RBI == 0) {
+        p.RBI = (nb_total + clusters * p.SR - 1) / (clusters * p.SR);
+        p.RBI = p.RBI < 1 ? 1 : (p.RBI > kGemvMaxRBI ? kGemvMaxRBI : p.RBI);
+    }
     return p;
+}
+
+// Splits the launch's clusters over the problems in proportion to their row blocks (at least one each).
+void share_clusters(const int* nb, int count, int total, int SR, int* out) {
+    int nb_total = 0;
+    for (int i = 0; i < count; ++i) nb_total += nb[i];
+    for (int i = 0; i < count; ++i) {
+        long long want = ((long long)total * nb[i] + nb_total / 2) / nb_total;
+        const int cap = (nb[i] + SR - 1) / SR;
+        if (want > cap) want = cap;
+        if (want < 1) want = 1;
+        out[i] = (int)want;
+    }
 }
 
 int check_problem(const mnnllm_w4a16_problem& q, int M) {
@@ -111,8 +155,10 @@ int run_batch(const mnnllm_w4a16_problem* problems, int count, int M, cudaStream
         const Plan plan = make_plan(nb_total, nc_max, group, MP);
         GemvLaunch L;
         std::memset(&L, 0, sizeof(L));
-        L.count = count; L.M = m; L.WC = plan.WC; L.SR = plan.SR; L.stages = plan.stages;
-        int clusters = 0;
+        L.count = count; L.M = m; L.WC = plan.WC; L.SR = plan.SR; L.RBI = plan.RBI; L.stages = plan.stages;
+        int clusters = 0, nbs[MNNLLM_MAX_BATCH], ncl[MNNLLM_MAX_BATCH];
+        for (int i = 0; i < count; ++i) nbs[i] = w4_geometry(problems[i].N, problems[i].K, group).n_row_blocks;
+        share_clusters(nbs, count, plan.clusters, plan.SR, ncl);
         for (int i = 0; i < count; ++i) {
             const mnnllm_w4a16_problem& q = problems[i];
             const W4Geometry g = w4_geometry(q.N, q.K, group);
@@ -123,11 +169,11 @@ int run_batch(const mnnllm_w4a16_problem* problems, int count, int M, cudaStream
             P.y = (uint8_t*)q.y + (size_t)m0 * q.N * ybytes;
             P.N = q.N; P.K = q.K;
             P.NB = g.n_row_blocks; P.NC = g.n_chunks; P.NS = g.n_slabs;
-            P.RBI = plan.RBI;
             P.cluster_begin = clusters;
+            P.n_clusters = ncl[i];
             P.y_dtype = q.y_dtype;
             P.row_block_bytes = g.row_block_bytes;
-            clusters += (g.n_row_blocks + plan.SR * plan.RBI - 1) / (plan.SR * plan.RBI);
+            clusters += ncl[i];
         }
         if (gemv_w4a16_launch(L, group, MP, clusters, plan.CS, status, stream) != cudaSuccess) {
             (void)cudaGetLastError();
@@ -175,15 +221,16 @@ int mnnllm_linear_w8a16(const void* x, const void* packed, void* y, int M, int N
     for (int m0 = 0; m0 < M; m0 += 8) {
         GemvLaunch L;
         std::memset(&L, 0, sizeof(L));
-        L.count = 1; L.M = (M - m0) < 8 ? (M - m0) : 8; L.WC = plan.WC; L.SR = plan.SR; L.stages = plan.stages;
+        L.count = 1; L.M = (M - m0) < 8 ? (M - m0) : 8; L.WC = plan.WC; L.SR = plan.SR; L.RBI = plan.RBI;
+        L.stages = plan.stages;
         GemvProblem& P = L.prob[0];
         P.packed = (const uint8_t*)packed;
         P.x = (const __half*)x + (size_t)m0 * K;
         P.y = (uint8_t*)y + (size_t)m0 * N * ybytes;
         P.N = N; P.K = K; P.NB = g.n_row_blocks; P.NC = g.n_chunks; P.NS = g.n_slabs;
-        P.RBI = plan.RBI; P.cluster_begin = 0; P.y_dtype = y_dtype;
+        P.cluster_begin = 0; P.n_clusters = plan.clusters; P.y_dtype = y_dtype;
         P.row_block_bytes = g.row_block_bytes; P.table_offset = g.table_offset;
-        const int clusters = (g.n_row_blocks + plan.SR * plan.RBI - 1) / (plan.SR * plan.RBI);
+        const int clusters = plan.clusters;
         if (gemv_w8a16_launch(L, clusters, plan.CS, status, (cudaStream_t)stream) != cudaSuccess) {
             (void)cudaGetLastError();
             return MNNLLM_ERR_CUDA;

@@ -8,7 +8,7 @@
 
 namespace mnnllm {
 
-constexpr int kGemvMaxWarps = 8;    // warps per CTA
+constexpr int kGemvMaxWarps = 7;    // warps per CTA (7 * 32 threads leave 144 registers each at 2 CTAs per SM)
 constexpr int kGemvMaxStages = 4;   // ring slots per warp
 constexpr int kGemvMaxRBI = 8;      // 16-row blocks a warp walks through per k-chunk
 constexpr int kNumSMs = 148;
@@ -19,8 +19,8 @@ struct GemvProblem {
     void* y;                // [M, N]
     int N, K;
     int NB, NC, NS;         // 16-row blocks, 512-k chunks, slabs per row
-    int RBI;                // row blocks per warp and chunk
     int cluster_begin;      // first cluster of this problem in the launch
+    int n_clusters;         // clusters that share this problem's row blocks evenly
     int y_dtype;
     unsigned long long row_block_bytes;
     unsigned long long table_offset;  // W8: per-row (scale, zero) table, from the buffer start
@@ -31,14 +31,18 @@ struct GemvLaunch {
     int count;
     int M;       // tokens (<= MP of the instantiation)
     int WC, SR;  // warps per CTA = WC (k-chunk lanes) * SR (row-block lanes)
+    int RBI;     // row blocks a warp walks per k-chunk and round
     int stages;
 };
 
 size_t gemv_w4a16_smem(int group, int MP, int W, int SR, int S);
+// resident CTAs per SM for this configuration (queries the runtime; 0 on error)
+int gemv_w4a16_occupancy(int group, int MP, int W, int SR, int S);
 cudaError_t gemv_w4a16_launch(const GemvLaunch& L, int group, int MP, int n_clusters, int CS, uint32_t* status,
                               cudaStream_t stream);
 
 size_t gemv_w8a16_smem(int W, int SR, int S);
+int gemv_w8a16_occupancy(int W, int SR, int S);
 cudaError_t gemv_w8a16_launch(const GemvLaunch& L, int n_clusters, int CS, uint32_t* status, cudaStream_t stream);
 
 }  // namespace mnnllm

@@ -51,8 +51,50 @@ __device__ __forceinline__ void store_out(void* y, int dtype, size_t idx, float 
     else reinterpret_cast<float*>(y)[idx] = v;
 }
 
+// MMAs of one quantum.  FULL: the chunk has all 8 slabs, so the loop is branch-free and the loads
+// and logic ops of different slabs can be interleaved.  Accumulator tile `set` collects GPS groups;
+// with few tiles the four MMAs of a slab go to separate banks (summed afterwards) to keep the
+// dependent-MMA chains short.
+template <int GROUP, int MP, bool FULL>
+__device__ __forceinline__ void quantum_mma(const uint4* __restrict__ slabs, int lane, int ns,
+                                            const uint32_t (&B)[8][4][2], float (&D)[Cfg<GROUP, MP>::NSETS][4]) {
+    using C = Cfg<GROUP, MP>;
+    constexpr int NBANK = C::NSETS == 1 ? 2 : 1;
+    constexpr uint32_t LO = 0x000F000Fu, HI = 0x00F000F0u, M1024 = 0x64006400u, M64 = 0x54005400u;
+    float acc[C::NSETS][NBANK][4];
+#pragma unroll
+    for (int s = 0; s < C::NSETS; ++s)
+#pragma unroll
+        for (int b = 0; b < NBANK; ++b) acc[s][b][0] = acc[s][b][1] = acc[s][b][2] = acc[s][b][3] = 0.f;
+#pragma unroll
+    for (int sl = 0; sl < 8; ++sl) {
+        if (FULL || sl < ns) {
+            const uint4 w = slabs[sl * 32 + lane];
+            const int set = (sl / C::SPG) / C::GPS;
+            const uint32_t x8 = w.x >> 8, z8 = w.z >> 8, y8 = w.y >> 8, w8 = w.w >> 8;
+            mma_m16n8k16_f16(acc[set][0 % NBANK], lop3_and_or(w.x, LO, M1024), lop3_and_or(w.z, LO, M1024),
+                             lop3_and_or(w.x, HI, M64), lop3_and_or(w.z, HI, M64), B[sl][0][0], B[sl][0][1]);
+            mma_m16n8k16_f16(acc[set][1 % NBANK], lop3_and_or(x8, LO, M1024), lop3_and_or(z8, LO, M1024),
+                             lop3_and_or(x8, HI, M64), lop3_and_or(z8, HI, M64), B[sl][1][0], B[sl][1][1]);
+            mma_m16n8k16_f16(acc[set][2 % NBANK], lop3_and_or(w.y, LO, M1024), lop3_and_or(w.w, LO, M1024),
+                             lop3_and_or(w.y, HI, M64), lop3_and_or(w.w, HI, M64), B[sl][2][0], B[sl][2][1]);
+            mma_m16n8k16_f16(acc[set][3 % NBANK], lop3_and_or(y8, LO, M1024), lop3_and_or(w8, LO, M1024),
+                             lop3_and_or(y8, HI, M64), lop3_and_or(w8, HI, M64), B[sl][3][0], B[sl][3][1]);
+        }
+    }
+#pragma unroll
+    for (int s = 0; s < C::NSETS; ++s)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            float v = acc[s][0][i];
+#pragma unroll
+            for (int b = 1; b < NBANK; ++b) v += acc[s][b][i];
+            D[s][i] = v;
+        }
+}
+
 template <int GROUP, int MP>
-__global__ void __launch_bounds__(kGemvMaxWarps * 32, 1)
+__global__ void __launch_bounds__(kGemvMaxWarps * 32, (MP <= 2 ? 2 : 1))
 gemv_w4a16_kernel(const __grid_constant__ GemvLaunch L, uint32_t* __restrict__ status) {
     using C = Cfg<GROUP, MP>;
     extern __shared__ __align__(128) uint8_t smem[];
@@ -61,7 +103,7 @@ gemv_w4a16_kernel(const __grid_constant__ GemvLaunch L, uint32_t* __restrict__ s
     const int r = lane >> 2, c = lane & 3;
     const int CS = (int)cluster_nctarank(), rank = (int)cluster_ctarank();
     const int cluster_id = blockIdx.x / CS;
-    const int W = L.WC * L.SR, S = L.stages;
+    const int W = L.WC * L.SR, S = L.stages, SR = L.SR, RBI = L.RBI;
 
     int pi = 0;
     while (pi + 1 < L.count && cluster_id >= L.prob[pi + 1].cluster_begin) ++pi;
@@ -69,27 +111,31 @@ gemv_w4a16_kernel(const __grid_constant__ GemvLaunch L, uint32_t* __restrict__ s
     const int cl = cluster_id - P.cluster_begin;
     const int wc = warp % L.WC, sr = warp / L.WC;
 
-    // shared memory carve-up (all offsets multiples of 128 B)
+    // shared memory carve-up
     uint8_t* ring = smem + (size_t)warp * S * C::QB;
-    float* corr = reinterpret_cast<float*>(smem + (size_t)W * S * C::QB) + warp * C::CORR_FLOATS;
-    float* part_all = reinterpret_cast<float*>(smem + (size_t)W * S * C::QB) + W * C::CORR_FLOATS;
-    float* part = part_all + warp * C::PART_FLOATS;
-    float* red = part_all + W * C::PART_FLOATS;  // [SR][RBI][MP][16]
-    uint64_t* bars = reinterpret_cast<uint64_t*>(red + L.SR * C::PART_FLOATS) + warp * kGemvMaxStages;
+    float* fbase = reinterpret_cast<float*>(smem + (size_t)W * S * C::QB);
+    float* corr = fbase + warp * C::CORR_FLOATS;
+    float* part_all = fbase + W * C::CORR_FLOATS;            // [W][2][RBI][MP][16]
+    float* red = part_all + W * 2 * C::PART_FLOATS;          // [2][SR][RBI][MP][16]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(red + 2 * SR * C::PART_FLOATS) + warp * kGemvMaxStages;
 
-    // this warp's work: chunks j = rank*WC + wc + t*CS*WC, row blocks rb = rb0 + it*SR
-    const int rb0 = cl * (L.SR * P.RBI) + sr;
-    int rbi_eff = 0;
-    if (rb0 < P.NB) {
-        rbi_eff = (P.NB - rb0 + L.SR - 1) / L.SR;
-        rbi_eff = rbi_eff < P.RBI ? rbi_eff : P.RBI;
-    }
+    // this cluster's rows: an even share of the problem's 16-row blocks, walked in rounds of SR*RBI
+    const int rb_begin = (int)((long long)P.NB * cl / P.n_clusters);
+    const int rb_end = (int)((long long)P.NB * (cl + 1) / P.n_clusters);
+    const int per_round = SR * RBI;
+    const int n_rounds = (rb_end - rb_begin + per_round - 1) / per_round;
+    // this warp's k-chunks: j = j0 + t * jstride
     const int jstride = CS * L.WC;
     const int j0 = rank * L.WC + wc;
     const int T = j0 < P.NC ? (P.NC - j0 + jstride - 1) / jstride : 0;
-    const int Q = T * rbi_eff;
-    const uint32_t full_chunk_bytes = (uint32_t)C::QB;
     const int last_ns = P.NS - 8 * (P.NC - 1);  // slabs in the last chunk
+
+    auto nit_of = [&](int rd) {  // row blocks of round rd that fall to this warp's sub-range
+        const int first = rb_begin + rd * per_round + sr;
+        if (first >= rb_end || T == 0) return 0;
+        const int n = (rb_end - first + SR - 1) / SR;
+        return n < RBI ? n : RBI;
+    };
 
     if (lane == 0) {
         for (int s = 0; s < S; ++s) mbar_init(&bars[s], 1);
@@ -98,23 +144,44 @@ gemv_w4a16_kernel(const __grid_constant__ GemvLaunch L, uint32_t* __restrict__ s
     fence_proxy_async_smem();
     __syncwarp();
 
-    auto issue = [&](int q) {  // lane 0 only
-        const int t = q / rbi_eff, it = q - t * rbi_eff;
-        const int j = j0 + t * jstride;
-        const int rb = rb0 + it * L.SR;
-        const int ns = (j == P.NC - 1) ? last_ns : 8;
-        const uint32_t bytes = (uint32_t)(ns * kSlabBytes + 16 * (ns / C::SPG) * 4);
-        const uint8_t* src = P.packed + kHeaderBytes + (size_t)rb * P.row_block_bytes + (size_t)j * full_chunk_bytes;
-        const int slot = q % S;
-        mbar_arrive_expect_tx(&bars[slot], bytes);
-        bulk_g2s(ring + (size_t)slot * C::QB, src, bytes, &bars[slot]);
+    // ---- producer side (lane 0): walks (round, chunk, row block) in the order of consumption ----
+    // A slot is refilled right after the warp has read it (the __syncwarp before the refill orders
+    // the reads of all lanes before the bulk copy is issued).
+    int i_rd = 0, i_t = 0, i_it = 0, i_nit = nit_of(0), i_slot = 0;
+    while (i_rd < n_rounds && i_nit == 0) { ++i_rd; i_nit = i_rd < n_rounds ? nit_of(i_rd) : 0; }
+    const uint8_t* const body = P.packed + kHeaderBytes;
+    const size_t it_stride = (size_t)SR * P.row_block_bytes;
+    auto src_of = [&](int rd, int t) {
+        return body + (size_t)(rb_begin + rd * per_round + sr) * P.row_block_bytes + (size_t)(j0 + t * jstride) * C::QB;
+    };
+    auto bytes_of = [&](int t) {
+        const int ns = (j0 + t * jstride == P.NC - 1) ? last_ns : 8;
+        return (uint32_t)(ns * kSlabBytes + 16 * (ns / C::SPG) * 4);
+    };
+    const uint8_t* i_src = i_rd < n_rounds ? src_of(i_rd, 0) : body;
+    uint32_t i_bytes = bytes_of(0);
+    auto issue_next = [&]() {
+        if (i_rd >= n_rounds) return;
+        mbar_arrive_expect_tx(&bars[i_slot], i_bytes);
+        bulk_g2s(ring + (size_t)i_slot * C::QB, i_src, i_bytes, &bars[i_slot]);
+        i_slot = (i_slot + 1 == S) ? 0 : i_slot + 1;
+        i_src += it_stride;
+        if (++i_it == i_nit) {
+            i_it = 0;
+            if (++i_t == T) {
+                i_t = 0;
+                do { ++i_rd; i_nit = i_rd < n_rounds ? nit_of(i_rd) : 0; } while (i_rd < n_rounds && i_nit == 0);
+            }
+            if (i_rd < n_rounds) {
+                i_src = src_of(i_rd, i_t);
+                i_bytes = bytes_of(i_t);
+            }
+        }
     };
 
     pdl_launch_dependents();
-    if (lane == 0) {
-        const int pre = Q < S ? Q : S;
-        for (int q = 0; q < pre; ++q) issue(q);
-    }
+    if (lane == 0)
+        for (int s = 0; s < S; ++s) issue_next();
     // everything above touched only weights; the activations may come from the previous kernel
     pdl_wait();
 
@@ -122,200 +189,205 @@ gemv_w4a16_kernel(const __grid_constant__ GemvLaunch L, uint32_t* __restrict__ s
     uint32_t B[8][4][2];
     float C1[C::NSETS][2], C2[C::NSETS][2];
     bool dead = false;
+    int cur_j = -1, slot = 0;
+    uint32_t phase = 0;
+    const int wc_used = (P.NC - rank * L.WC) < L.WC ? (P.NC - rank * L.WC) : L.WC;  // warps that own a chunk
 
-    for (int q = 0; q < Q; ++q) {
-        const int t = q / rbi_eff, it = q - t * rbi_eff;
-        const int j = j0 + t * jstride;
-        const int ns = (j == P.NC - 1) ? last_ns : 8;
-        const int ng = ns / C::SPG;
+    for (int rd = 0; rd < n_rounds; ++rd) {
+        const int nit = nit_of(rd);
+        float* part = part_all + (warp * 2 + (rd & 1)) * C::PART_FLOATS;
+        if (nit > 0)
+            for (int t = 0; t < T; ++t) {
+                const int j = j0 + t * jstride;
+                const int ns = (j == P.NC - 1) ? last_ns : 8;
+                const int ng = ns / C::SPG;
 
-        if (it == 0) {
-            // ---- new k-chunk: activations -> B fragments, group sums -> correction terms ----
-            const __half* xk = P.x + (size_t)j * kChunkK;
+                if (j != cur_j) {
+                    cur_j = j;
+                    // ---- new k-chunk: activations -> B fragments, group sums -> correction terms ----
+                    const __half* xk = P.x + (size_t)j * kChunkK;
 #pragma unroll
-            for (int sl = 0; sl < 8; ++sl) {
-                uint4 u0 = make_uint4(0, 0, 0, 0), u1 = u0;
-                const int gi = sl / C::SPG;
-                const bool mine = (sl < ns) && (tokB < L.M) && (gsB == gi % C::GPS);
-                if (mine) {
-                    const uint4* px = reinterpret_cast<const uint4*>(xk + (size_t)tokB * P.K + sl * kSlabK4 + 16 * c);
-                    u0 = px[0];
-                    u1 = px[1];
+                    for (int sl = 0; sl < 8; ++sl) {
+                        uint4 u0 = make_uint4(0, 0, 0, 0), u1 = u0;
+                        const int gi = sl / C::SPG;
+                        const bool mine = (sl < ns) && (tokB < L.M) && (gsB == gi % C::GPS);
+                        if (mine) {
+                            const uint4* px =
+                                reinterpret_cast<const uint4*>(xk + (size_t)tokB * P.K + sl * kSlabK4 + 16 * c);
+                            u0 = px[0];
+                            u1 = px[1];
+                        }
+                        B[sl][0][0] = __byte_perm(u0.x, u0.y, 0x5410);
+                        B[sl][0][1] = __byte_perm(u0.z, u0.w, 0x5410);
+                        B[sl][1][0] = __byte_perm(u0.x, u0.y, 0x7632);
+                        B[sl][1][1] = __byte_perm(u0.z, u0.w, 0x7632);
+                        B[sl][2][0] = __byte_perm(u1.x, u1.y, 0x5410);
+                        B[sl][2][1] = __byte_perm(u1.z, u1.w, 0x5410);
+                        B[sl][3][0] = __byte_perm(u1.x, u1.y, 0x7632);
+                        B[sl][3][1] = __byte_perm(u1.z, u1.w, 0x7632);
+                    }
+                    __syncwarp();  // the previous chunk's correction terms are no longer read
+#pragma unroll
+                    for (int i = 0; i < C::NSETS; ++i) {
+                        const int gi = gsB + C::GPS * i;
+                        float lo = 0.f, hi = 0.f;
+                        if (gi < ng && tokB < L.M) {
+#pragma unroll
+                            for (int sp = 0; sp < C::SPG; ++sp) {
+                                const uint4* px = reinterpret_cast<const uint4*>(
+                                    xk + (size_t)tokB * P.K + (gi * C::SPG + sp) * kSlabK4 + 16 * c);
+                                const uint4 u0 = px[0], u1 = px[1];
+                                float2 f;
+                                f = h2f2(u0.x); lo += f.x + f.y;
+                                f = h2f2(u0.y); lo += f.x + f.y;
+                                f = h2f2(u1.x); lo += f.x + f.y;
+                                f = h2f2(u1.y); lo += f.x + f.y;
+                                f = h2f2(u0.z); hi += f.x + f.y;
+                                f = h2f2(u0.w); hi += f.x + f.y;
+                                f = h2f2(u1.z); hi += f.x + f.y;
+                                f = h2f2(u1.w); hi += f.x + f.y;
+                            }
+                        }
+                        lo += __shfl_xor_sync(0xffffffffu, lo, 1);
+                        hi += __shfl_xor_sync(0xffffffffu, hi, 1);
+                        lo += __shfl_xor_sync(0xffffffffu, lo, 2);
+                        hi += __shfl_xor_sync(0xffffffffu, hi, 2);
+                        if (c == 0 && gi < C::GC) {
+                            corr[(tokB * C::GC + gi) * 2 + 0] = 1024.f * lo + 64.f * hi;
+                            corr[(tokB * C::GC + gi) * 2 + 1] = lo + hi;
+                        }
+                    }
+                    __syncwarp();
+#pragma unroll
+                    for (int s = 0; s < C::NSETS; ++s)
+#pragma unroll
+                        for (int e = 0; e < 2; ++e) {
+                            const int col = 2 * c + e;
+                            const int gi = s * C::GPS + col / MP;
+                            const bool ok = gi < C::GC;
+                            C1[s][e] = ok ? corr[((col % MP) * C::GC + gi) * 2 + 0] : 0.f;
+                            C2[s][e] = ok ? corr[((col % MP) * C::GC + gi) * 2 + 1] : 0.f;
+                        }
                 }
-                B[sl][0][0] = __byte_perm(u0.x, u0.y, 0x5410);
-                B[sl][0][1] = __byte_perm(u0.z, u0.w, 0x5410);
-                B[sl][1][0] = __byte_perm(u0.x, u0.y, 0x7632);
-                B[sl][1][1] = __byte_perm(u0.z, u0.w, 0x7632);
-                B[sl][2][0] = __byte_perm(u1.x, u1.y, 0x5410);
-                B[sl][2][1] = __byte_perm(u1.z, u1.w, 0x5410);
-                B[sl][3][0] = __byte_perm(u1.x, u1.y, 0x7632);
-                B[sl][3][1] = __byte_perm(u1.z, u1.w, 0x7632);
-            }
-            __syncwarp();  // the previous chunk's correction terms are no longer read
+
+                for (int it = 0; it < nit; ++it) {
+                    // ---- wait for this quantum's bulk copy ----
+                    if (!dead && !mbar_wait_bounded(&bars[slot], phase, kMaxPolls)) {
+                        dead = true;
+                        if (lane == 0) atomicOr(status, 0x100u | (uint32_t)pi);
+                    }
+                    const uint8_t* qp = ring + (size_t)slot * C::QB;
+                    const uint4* slabs = reinterpret_cast<const uint4*>(qp);
+
+                    float D[C::NSETS][4];
+                    if (ns == 8) quantum_mma<GROUP, MP, true>(slabs, lane, 8, B, D);
+                    else quantum_mma<GROUP, MP, false>(slabs, lane, ns, B, D);
+
+                    // ---- rescale: column (2c + e) of tile s is (token, group) = (col % MP, s*GPS + col / MP) ----
+                    float out[2][2] = {{0.f, 0.f}, {0.f, 0.f}};  // [row half h][column e]
+                    auto rescale = [&](const int ngc) {
+                        const uint32_t* table = reinterpret_cast<const uint32_t*>(qp + (size_t)ngc * C::SPG * kSlabBytes);
 #pragma unroll
-            for (int i = 0; i < C::NSETS; ++i) {
-                const int gi = gsB + C::GPS * i;
-                float lo = 0.f, hi = 0.f;
-                if (gi < ng && tokB < L.M) {
+                        for (int s = 0; s < C::NSETS; ++s)
 #pragma unroll
-                    for (int sp = 0; sp < C::SPG; ++sp) {
-                        const uint4* px = reinterpret_cast<const uint4*>(
-                            xk + (size_t)tokB * P.K + (gi * C::SPG + sp) * kSlabK4 + 16 * c);
-                        const uint4 u0 = px[0], u1 = px[1];
-                        float2 f;
-                        f = h2f2(u0.x); lo += f.x + f.y;
-                        f = h2f2(u0.y); lo += f.x + f.y;
-                        f = h2f2(u1.x); lo += f.x + f.y;
-                        f = h2f2(u1.y); lo += f.x + f.y;
-                        f = h2f2(u0.z); hi += f.x + f.y;
-                        f = h2f2(u0.w); hi += f.x + f.y;
-                        f = h2f2(u1.z); hi += f.x + f.y;
-                        f = h2f2(u1.w); hi += f.x + f.y;
+                            for (int e = 0; e < 2; ++e) {
+                                const int gi = s * C::GPS + (2 * c + e) / MP;
+                                const bool ok = gi < ngc;
+                                const int gic = ok ? gi : 0;
+#pragma unroll
+                                for (int h = 0; h < 2; ++h) {
+                                    const float2 sz = h2f2(table[(r + 8 * h) * ngc + gic]);
+                                    const float v = sz.x * ((D[s][2 * h + e] - C1[s][e]) - sz.y * C2[s][e]);
+                                    out[h][e] += ok ? v : 0.f;
+                                }
+                            }
+                    };
+                    if (ns == 8) rescale(C::GC); else rescale(ng);
+                    // the slot has been read: release and refill it before the (register-only) tail
+                    __syncwarp();
+                    if (lane == 0) issue_next();
+                    slot = (slot + 1 == S) ? 0 : slot + 1;
+                    phase ^= (slot == 0) ? 1u : 0u;
+
+                    // sum the columns that belong to the same token
+                    if (MP == 1) { out[0][0] += out[0][1]; out[1][0] += out[1][1]; }
+#pragma unroll
+                    for (int h = 0; h < 2; ++h)
+#pragma unroll
+                        for (int e = 0; e < 2; ++e) {
+                            if (MP <= 2) out[h][e] += __shfl_xor_sync(0xffffffffu, out[h][e], 1);
+                            if (MP <= 4) out[h][e] += __shfl_xor_sync(0xffffffffu, out[h][e], 2);
+                        }
+                    // writers: MP=1: c==0 writes token 0 (e=0); MP=2: c==0 writes tokens e; MP=4: c<2
+                    // writes tokens 2c+e; MP=8: every lane writes tokens 2c+e
+                    const bool writer = (MP == 8) || (MP == 4 && c < 2) || (MP <= 2 && c == 0);
+                    if (writer) {
+#pragma unroll
+                        for (int e = 0; e < (MP == 1 ? 1 : 2); ++e) {
+                            const int tok = (2 * c + e) % MP;
+#pragma unroll
+                            for (int h = 0; h < 2; ++h) {
+                                float* dst = part + (it * MP + tok) * 16 + r + 8 * h;
+                                *dst = (t == 0) ? out[h][e] : (*dst + out[h][e]);
+                            }
+                        }
                     }
                 }
-                lo += __shfl_xor_sync(0xffffffffu, lo, 1);
-                hi += __shfl_xor_sync(0xffffffffu, hi, 1);
-                lo += __shfl_xor_sync(0xffffffffu, lo, 2);
-                hi += __shfl_xor_sync(0xffffffffu, hi, 2);
-                if (c == 0 && gi < C::GC) {
-                    corr[(tokB * C::GC + gi) * 2 + 0] = 1024.f * lo + 64.f * hi;
-                    corr[(tokB * C::GC + gi) * 2 + 1] = lo + hi;
-                }
             }
-            __syncwarp();
-#pragma unroll
-            for (int s = 0; s < C::NSETS; ++s)
-#pragma unroll
-                for (int e = 0; e < 2; ++e) {
-                    const int col = 2 * c + e;
-                    const int gi = s * C::GPS + col / MP;
-                    const bool ok = gi < C::GC;
-                    C1[s][e] = ok ? corr[((col % MP) * C::GC + gi) * 2 + 0] : 0.f;
-                    C2[s][e] = ok ? corr[((col % MP) * C::GC + gi) * 2 + 1] : 0.f;
-                }
-        }
 
-        // ---- wait for this quantum's bulk copy ----
-        const int slot = q % S;
-        if (!dead && !mbar_wait_bounded(&bars[slot], (uint32_t)((q / S) & 1), kMaxPolls)) {
-            dead = true;
-            if (lane == 0) atomicOr(status, 0x100u | (uint32_t)pi);
-        }
-        const uint8_t* qp = ring + (size_t)slot * C::QB;
-        const uint4* slabs = reinterpret_cast<const uint4*>(qp);
-
-        float D[C::NSETS][4];
-#pragma unroll
-        for (int s = 0; s < C::NSETS; ++s) D[s][0] = D[s][1] = D[s][2] = D[s][3] = 0.f;
-
-#pragma unroll
-        for (int sl = 0; sl < 8; ++sl) {
-            if (sl < ns) {
-                const uint4 w = slabs[sl * 32 + lane];
-                constexpr uint32_t LO = 0x000F000Fu, HI = 0x00F000F0u, M1024 = 0x64006400u, M64 = 0x54005400u;
-                const int set = (sl / C::SPG) / C::GPS;
-                mma_m16n8k16_f16(D[set], lop3_and_or(w.x, LO, M1024), lop3_and_or(w.z, LO, M1024),
-                                 lop3_and_or(w.x, HI, M64), lop3_and_or(w.z, HI, M64), B[sl][0][0], B[sl][0][1]);
-                const uint32_t x8 = w.x >> 8, z8 = w.z >> 8;
-                mma_m16n8k16_f16(D[set], lop3_and_or(x8, LO, M1024), lop3_and_or(z8, LO, M1024),
-                                 lop3_and_or(x8, HI, M64), lop3_and_or(z8, HI, M64), B[sl][1][0], B[sl][1][1]);
-                mma_m16n8k16_f16(D[set], lop3_and_or(w.y, LO, M1024), lop3_and_or(w.w, LO, M1024),
-                                 lop3_and_or(w.y, HI, M64), lop3_and_or(w.w, HI, M64), B[sl][2][0], B[sl][2][1]);
-                const uint32_t y8 = w.y >> 8, w8 = w.w >> 8;
-                mma_m16n8k16_f16(D[set], lop3_and_or(y8, LO, M1024), lop3_and_or(w8, LO, M1024),
-                                 lop3_and_or(y8, HI, M64), lop3_and_or(w8, HI, M64), B[sl][3][0], B[sl][3][1]);
+        // ---- end of round: sum over the warps (k-chunks) of this CTA, then over the cluster ----
+        __syncthreads();
+        const int n_out = per_round * MP * 16;
+        float* red_rd = red + (rd & 1) * SR * C::PART_FLOATS;
+        for (int o = threadIdx.x; o < n_out; o += blockDim.x) {
+            const int row = o & 15, tok = (o >> 4) % MP, it = (o / (16 * MP)) % RBI, s_r = o / (16 * MP * RBI);
+            const int rb = rb_begin + rd * per_round + it * SR + s_r;
+            float acc = 0.f;
+            if (rb < rb_end)
+                for (int w = 0; w < wc_used; ++w)
+                    acc += part_all[((s_r * L.WC + w) * 2 + (rd & 1)) * C::PART_FLOATS + (it * MP + tok) * 16 + row];
+            if (CS == 1) {
+                const int n = rb * 16 + row;
+                if (rb < rb_end && n < P.N && tok < L.M) store_out(P.y, P.y_dtype, (size_t)tok * P.N + n, acc);
+            } else {
+                red_rd[o] = acc;
             }
         }
-
-        // ---- rescale: column (2c + e) of tile s is (token, group) = (col % MP, s*GPS + col / MP) ----
-        const uint32_t* table = reinterpret_cast<const uint32_t*>(qp + (size_t)ns * kSlabBytes);
-        float out[2][2] = {{0.f, 0.f}, {0.f, 0.f}};  // [row half h][column e]
-#pragma unroll
-        for (int s = 0; s < C::NSETS; ++s)
-#pragma unroll
-            for (int e = 0; e < 2; ++e) {
-                const int gi = s * C::GPS + (2 * c + e) / MP;
-                if (gi < ng) {
-#pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        const float2 sz = h2f2(table[(r + 8 * h) * ng + gi]);
-                        out[h][e] += sz.x * ((D[s][2 * h + e] - C1[s][e]) - sz.y * C2[s][e]);
-                    }
+        if (CS > 1) {
+            cluster_sync();
+            for (int o = threadIdx.x * CS + rank; o < n_out; o += blockDim.x * CS) {
+                const int row = o & 15, tok = (o >> 4) % MP, it = (o / (16 * MP)) % RBI, s_r = o / (16 * MP * RBI);
+                const int rb = rb_begin + rd * per_round + it * SR + s_r;
+                const int n = rb * 16 + row;
+                if (rb < rb_end && n < P.N && tok < L.M) {
+                    float acc = 0.f;
+                    for (int cr = 0; cr < CS; ++cr) acc += ld_dsmem_f32(red_rd + o, (uint32_t)cr);
+                    store_out(P.y, P.y_dtype, (size_t)tok * P.N + n, acc);
                 }
             }
-        // sum the columns that belong to the same token
-        if (MP == 1) { out[0][0] += out[0][1]; out[1][0] += out[1][1]; }
-#pragma unroll
-        for (int h = 0; h < 2; ++h)
-#pragma unroll
-            for (int e = 0; e < 2; ++e) {
-                if (MP <= 2) out[h][e] += __shfl_xor_sync(0xffffffffu, out[h][e], 1);
-                if (MP <= 4) out[h][e] += __shfl_xor_sync(0xffffffffu, out[h][e], 2);
-            }
-        // writers: MP=1: c==0 writes token 0 (e=0); MP=2: c==0 writes tokens e; MP=4: c<2 writes
-        // tokens 2c+e; MP=8: every lane writes tokens 2c+e
-        {
-            const bool writer = (MP == 8) || (MP == 4 && c < 2) || (MP <= 2 && c == 0);
-            if (writer) {
-#pragma unroll
-                for (int e = 0; e < (MP == 1 ? 1 : 2); ++e) {
-                    const int tok = (2 * c + e) % MP;
-#pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        float* dst = part + (it * MP + tok) * 16 + r + 8 * h;
-                        *dst = (t == 0) ? out[h][e] : (*dst + out[h][e]);
-                    }
-                }
-            }
-        }
-
-        // ---- release the slot and refill it ----
-        __syncwarp();
-        if (lane == 0 && q + S < Q) {
-            fence_proxy_async_smem();
-            issue(q + S);
         }
     }
-
-    // ---- sum over the warps (k-chunks) of this CTA, then over the CTAs of the cluster ----
-    __syncthreads();
-    const int n_out = L.SR * P.RBI * MP * 16;
-    const int wc_used = (P.NC - rank * L.WC) < L.WC ? (P.NC - rank * L.WC) : L.WC;  // warps that had a chunk
-    for (int o = threadIdx.x; o < n_out; o += blockDim.x) {
-        const int row = o & 15, tok = (o >> 4) % MP, it = (o / (16 * MP)) % P.RBI, s_r = o / (16 * MP * P.RBI);
-        float acc = 0.f;
-        const int rb = cl * (L.SR * P.RBI) + s_r + it * L.SR;
-        if (rb < P.NB)
-            for (int w = 0; w < wc_used; ++w)
-                acc += part_all[(s_r * L.WC + w) * C::PART_FLOATS + (it * MP + tok) * 16 + row];
-        if (CS == 1) {
-            const int n = rb * 16 + row;
-            if (rb < P.NB && n < P.N && tok < L.M) store_out(P.y, P.y_dtype, (size_t)tok * P.N + n, acc);
-        } else {
-            red[o] = acc;
-        }
-    }
-    if (CS > 1) {
-        cluster_sync();
-        for (int o = threadIdx.x * CS + rank; o < n_out; o += blockDim.x * CS) {
-            const int row = o & 15, tok = (o >> 4) % MP, it = (o / (16 * MP)) % P.RBI, s_r = o / (16 * MP * P.RBI);
-            const int rb = cl * (L.SR * P.RBI) + s_r + it * L.SR;
-            const int n = rb * 16 + row;
-            if (rb < P.NB && n < P.N && tok < L.M) {
-                float acc = 0.f;
-                for (int cr = 0; cr < CS; ++cr) acc += ld_dsmem_f32(red + o, (uint32_t)cr);
-                store_out(P.y, P.y_dtype, (size_t)tok * P.N + n, acc);
-            }
-        }
-        cluster_sync();  // peers may still be reading this CTA's shared memory
-    }
+    if (CS > 1) cluster_sync();  // peers may still be reading this CTA's shared memory
 }
 
 template <int GROUP, int MP>
 size_t smem_bytes(int W, int SR, int S) {
     using C = Cfg<GROUP, MP>;
-    return (size_t)W * S * C::QB + (size_t)W * C::CORR_FLOATS * 4 + (size_t)W * C::PART_FLOATS * 4 +
-           (size_t)SR * C::PART_FLOATS * 4 + (size_t)W * kGemvMaxStages * 8;
+    return (size_t)W * S * C::QB + (size_t)W * C::CORR_FLOATS * 4 + (size_t)W * 2 * C::PART_FLOATS * 4 +
+           (size_t)2 * SR * C::PART_FLOATS * 4 + (size_t)W * kGemvMaxStages * 8;
+}
+
+// Raises the kernel's dynamic shared memory limit when a launch needs more than any before it.
+template <int GROUP, int MP>
+cudaError_t ensure_smem(size_t smem) {
+    static size_t configured = 0;  // per instantiation
+    if (smem > configured) {
+        cudaError_t e = cudaFuncSetAttribute(gemv_w4a16_kernel<GROUP, MP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)smem);
+        if (e != cudaSuccess) return e;
+        configured = smem;
+    }
+    return cudaSuccess;
 }
 
 template <int GROUP, int MP>
@@ -323,12 +395,7 @@ cudaError_t launch_one(const GemvLaunch& L, int n_clusters, int CS, uint32_t* st
     const int W = L.WC * L.SR;
     const size_t smem = smem_bytes<GROUP, MP>(W, L.SR, L.stages);
     auto kern = gemv_w4a16_kernel<GROUP, MP>;
-    static size_t configured = 0;  // per instantiation
-    if (smem > configured) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        configured = smem;
-    }
+    if (cudaError_t e = ensure_smem<GROUP, MP>(smem); e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(n_clusters * CS));
     cfg.blockDim = dim3((unsigned)(W * 32));
@@ -346,7 +413,25 @@ cudaError_t launch_one(const GemvLaunch& L, int n_clusters, int CS, uint32_t* st
     return cudaLaunchKernelEx(&cfg, kern, L, status);
 }
 
+template <int GROUP, int MP>
+int occupancy_of(int W, int SR, int S) {
+    int n = 0;
+    const size_t smem = smem_bytes<GROUP, MP>(W, SR, S);
+    auto kern = gemv_w4a16_kernel<GROUP, MP>;
+    if (ensure_smem<GROUP, MP>(smem) != cudaSuccess) return 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kern, W * 32, smem) != cudaSuccess) return 0;
+    return n;
+}
+
 }  // namespace
+
+int gemv_w4a16_occupancy(int group, int MP, int W, int SR, int S) {
+#define MNN_CASE(G, P) if (group == G && MP == P) return occupancy_of<G, P>(W, SR, S);
+    MNN_CASE(64, 1) MNN_CASE(64, 2) MNN_CASE(64, 4) MNN_CASE(64, 8)
+    MNN_CASE(128, 1) MNN_CASE(128, 2) MNN_CASE(128, 4) MNN_CASE(128, 8)
+#undef MNN_CASE
+    return 0;
+}
 
 size_t gemv_w4a16_smem(int group, int MP, int W, int SR, int S) {
     if (group == 64) {
