@@ -1,0 +1,389 @@
+#!/usr/bin/env python
+"""Benchmark of the weight-quantised linear stack on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+One step = one pass of the whole linear stack of the workload over one batch of synthetic input
+(decode: one token through all 28 layers x 7 linears).  Rank 0 prints ONE JSON line.  With N > 1
+(launched by torchrun) every rank runs an independent replica on its own GPU: the path has no
+exchange step, so there is no collective on the data path.
+
+`--impl reference` times the CPU oracle (a deliberately plain program) on the host cores instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+METRIC = "decode W4 GEMV GB/s"
+UNIT = "GB/s"
+FALLBACK_HBM_GBS = 6650.0
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel from the committed
+# ncu capture (profiles/), keyed by workload; None when no capture matches the current kernel.
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return json.load(f), "measured"
+    return {"hbm_gbs": FALLBACK_HBM_GBS}, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU through NVML while the benchmark runs."""
+
+    def __init__(self, torch_device_index: int, period_s: float = 0.02):
+        self.period = period_s
+        self.samples = []  # (t, sm_mhz, reasons bitmask)
+        self.ok = False
+        self.sm_max = None
+        self._stop = threading.Event()
+        try:
+            import pynvml
+            import torch
+
+            pynvml.nvmlInit()
+            uuid = str(torch.cuda.get_device_properties(torch_device_index).uuid)
+            handle = None
+            for i in range(pynvml.nvmlDeviceGetCount()):
+                h = pynvml.nvmlDeviceGetHandleByIndex(i)
+                u = pynvml.nvmlDeviceGetUUID(h)
+                u = u.decode() if isinstance(u, bytes) else u
+                if uuid in u:
+                    handle = h
+                    break
+            if handle is None:
+                handle = pynvml.nvmlDeviceGetHandleByIndex(torch_device_index)
+            self.nv, self.h = pynvml, handle
+            self.sm_max = int(pynvml.nvmlDeviceGetMaxClockInfo(handle, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception as e:  # NVML missing: the line says so instead of inventing clocks
+            self.err = repr(e)
+        self.thread = threading.Thread(target=self._run, daemon=True)
+
+    def _reasons(self):
+        nv = self.nv
+        for name in ("nvmlDeviceGetCurrentClocksEventReasons", "nvmlDeviceGetCurrentClocksThrottleReasons"):
+            f = getattr(nv, name, None)
+            if f is not None:
+                try:
+                    return int(f(self.h))
+                except Exception:
+                    pass
+        return 0
+
+    def _run(self):
+        while not self._stop.is_set():
+            try:
+                mhz = int(self.nv.nvmlDeviceGetClockInfo(self.h, self.nv.NVML_CLOCK_SM))
+                self.samples.append((time.perf_counter(), mhz, self._reasons()))
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def start(self):
+        if self.ok:
+            self.thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self.ok:
+            self.thread.join(timeout=2)
+
+    def summary(self, t0: float, t1: float):
+        if not self.ok:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "note": "NVML unavailable"}
+        inside = [s for s in self.samples if t0 <= s[0] <= t1]
+        note = "sampled inside the timed region"
+        if not inside:  # region shorter than the sampling period: take every sample under load
+            inside = self.samples[1:] or self.samples
+            note = "timed region shorter than the sampling period; samples cover warm-up + timed + e2e loops"
+        bits = 0
+        for s in inside:
+            bits |= s[2]
+        names = {
+            0x1: "gpu_idle", 0x2: "applications_clocks_setting", 0x4: "sw_power_cap", 0x8: "hw_slowdown",
+            0x10: "sync_boost", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+            0x80: "hw_power_brake_slowdown", 0x100: "display_clock_setting",
+        }
+        reasons = [n for b, n in names.items() if bits & b and n != "gpu_idle"]
+        mhz = sorted(s[1] for s in inside)
+        return {"sm_mhz": mhz[len(mhz) // 2] if mhz else None, "sm_max_mhz": self.sm_max, "reasons": reasons,
+                "samples": len(inside), "note": note}
+
+
+# --------------------------------------------------------------------------------------------------
+# workloads
+# --------------------------------------------------------------------------------------------------
+WORKLOADS = {
+    # name: (model key, config number of the workload list, tokens per step)
+    "decode_qwen2_1p5b_w4a16_g64": ("QWEN2_1P5B", 2, 1),
+    "decode_qwen2_7b_w4a16_g64": ("QWEN2_7B", 4, 1),
+}
+DEFAULT_WORKLOAD = "decode_qwen2_1p5b_w4a16_g64"
+
+
+def oracle_stack_pass(model, config, M, group, max_seconds, max_layers):
+    """Times the CPU oracle's W4A16 linear, layer by layer, until `max_seconds` have been spent or
+    `max_layers` layers are done.  Returns (algorithmic bytes processed, seconds, layers, threads)."""
+    import oracle
+    from paper_2506_10443_b200 import inputs
+    from paper_2506_10443_b200.workloads import linear_bytes
+
+    done_bytes, spent, layers = 0, 0.0, 0
+    for l in range(max_layers):
+        for lin in inputs.stack(model):
+            W = inputs.weights(inputs.seed_for(config, l, lin.matrix_id, 0), lin.N, lin.K)
+            q, s, z = oracle.quantize_w4(W, group)          # offline step, not timed
+            x = inputs.activations(inputs.seed_for(config, l, lin.matrix_id, 1), M, lin.K).astype(np.float32)
+            t = time.perf_counter()
+            oracle.linear_wa16(x, q, s, z, group)
+            spent += time.perf_counter() - t
+            done_bytes += linear_bytes(lin.N, lin.K, group, M)
+        layers += 1
+        if spent >= max_seconds:
+            break
+    return done_bytes, spent, layers, oracle.num_threads()
+
+
+def run_reference(args):
+    """The reference arm: the CPU oracle as it stands, on the host cores, same metric and config.
+    Each step is a bounded sample of the workload sized from a calibration pass so that the whole
+    run (warm-up + steps) stays within about two minutes of oracle time."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    from paper_2506_10443_b200 import inputs
+    from paper_2506_10443_b200.workloads import linear_bytes
+
+    model_key, config, M = WORKLOADS[args.workload]
+    model = getattr(inputs, model_key)
+    group = 64
+    linears = inputs.stack(model)
+    layer_bytes = sum(linear_bytes(t.N, t.K, group, M) for t in linears)
+
+    def prepared(layer, frac):
+        out = []
+        for lin in linears:
+            rows = lin.N if frac >= 1.0 else max(1, int(np.ceil(frac * lin.N)))
+            W = inputs.weights(inputs.seed_for(config, layer, lin.matrix_id, 0), lin.N, lin.K)[:rows]
+            q, s, z = oracle.quantize_w4(W, group)   # offline step, not timed
+            x = inputs.activations(inputs.seed_for(config, layer, lin.matrix_id, 1), M, lin.K).astype(np.float32)
+            out.append((x, q, s, z, linear_bytes(rows, lin.K, group, M)))
+        return out
+
+    # calibration: 2 % of the rows of layer 0
+    cal = prepared(0, 0.02)
+    t = time.perf_counter()
+    for x, q, s, z, _ in cal:
+        oracle.linear_wa16(x, q, s, z, group)
+    rate = sum(c[4] for c in cal) / max(time.perf_counter() - t, 1e-6)   # bytes per second
+    budget = min(2.0, 120.0 / max(args.steps + args.warmup, 1))
+    frac = rate * budget / layer_bytes
+    if frac >= 1.0:
+        n_layers = min(model["layers"], int(frac))
+        sample = [p for l in range(n_layers) for p in prepared(l, 1.0)]
+        what = "%d of %d layers (7 linears each), %d token, per step" % (n_layers, model["layers"], M)
+    else:
+        sample = prepared(0, frac)
+        what = "first %.1f %% of the rows of each of the 7 linears of layer 0, %d token, per step" % (100 * frac, M)
+    step_bytes = sum(p[4] for p in sample)
+
+    def step():
+        for x, q, s, z, _ in sample:
+            oracle.linear_wa16(x, q, s, z, group)
+
+    for _ in range(args.warmup):
+        step()
+    t = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    total_s = time.perf_counter() - t
+    value = step_bytes * args.steps / total_s / 1e9
+    threads = oracle.num_threads()
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total_s / max(args.steps, 1),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": args.workload, "sample": what, "algorithmic_bytes_per_step": step_bytes},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": what},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def run_ours(args):
+    import torch
+
+    from paper_2506_10443_b200 import binding as B   # raises if the CUDA library is missing
+    from paper_2506_10443_b200 import inputs
+    from paper_2506_10443_b200.workloads import LinearStack
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a GPU: there is no CPU path")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    if not B.device_supported():
+        raise SystemExit("the kernels are built for compute capability 10.x only")
+
+    model_key, config, M = WORKLOADS[args.workload]
+    model = getattr(inputs, model_key)
+    stack = LinearStack(model, config, M, 64)   # every rank: an independent replica of the workload
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # one untimed pass resolves per-device state (function attributes, symbol addresses), then capture
+    stack.run_w4a16()
+    assert B.read_status() == 0
+    graph = None
+    if not args.no_graph:
+        graph = torch.cuda.CUDAGraph()
+        cap = torch.cuda.Stream()
+        cap.wait_stream(stream)
+        with torch.cuda.graph(graph, stream=cap):
+            stack.run_w4a16(cap)
+        torch.cuda.synchronize()
+
+    def step():
+        if graph is not None:
+            graph.replay()
+        else:
+            stack.run_w4a16()
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = time.perf_counter()
+    ev0.record()
+    for _ in range(args.steps):
+        step()
+    ev1.record()
+    barrier()
+    t1 = time.perf_counter()
+    ms = ev0.elapsed_time(ev1)
+    assert B.read_status() == 0
+
+    # end to end: the step's activations come from pinned host memory, its outputs go back to it
+    e2e_steps = max(1, min(args.steps, 500))
+    for _ in range(3):
+        stack.xin.copy_(stack.xin_host, non_blocking=True)
+        step()
+        stack.yout_host.copy_(stack.yout, non_blocking=True)
+        torch.cuda.synchronize()
+    barrier()
+    ee0, ee1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ee0.record()
+    for _ in range(e2e_steps):
+        stack.xin.copy_(stack.xin_host, non_blocking=True)
+        step()
+        stack.yout_host.copy_(stack.yout, non_blocking=True)
+        stream.synchronize()   # the host reads the result of every step
+    ee1.record()
+    barrier()
+    e2e_ms = ee0.elapsed_time(ee1)
+    sampler.stop()
+
+    if dist is not None:
+        t = torch.tensor([ms, e2e_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms, e2e_ms = float(t[0]), float(t[1])
+
+    if rank == 0:
+        peaks, peaks_kind = measured_peaks()
+        step_bytes = stack.algorithmic_bytes_w4a16
+        ms_per_step = ms / args.steps
+        gbs_one = step_bytes / (ms_per_step * 1e-3) / 1e9          # one replica
+        value = gbs_one * world
+        e2e_value = step_bytes * world / (e2e_ms / e2e_steps * 1e-3) / 1e9
+        launches = stack.launches_per_step_w4a16
+        peak = float(peaks["hbm_gbs"])
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {
+                "workload": args.workload, "tokens_per_step": M, "group": 64, "layers": stack.n_layers,
+                "linears_per_layer": 7, "weight_bytes": stack.weight_bytes, "algorithmic_bytes_per_step": step_bytes,
+                "l2": "weights of one step (%.0f MB) exceed L2 (126 MB); no flush" % (stack.weight_bytes / 1e6),
+                "cuda_graph": graph is not None, "parallelism": "replicas only" if world > 1 else "single GPU",
+            },
+            "tokens_per_s": M * world / (ms_per_step * 1e-3),
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(stack.xin_host.numel() * 2),
+                    "d2h_bytes_per_step": int(stack.yout_host.numel() * 2), "steps": e2e_steps,
+                    "ms_per_step": e2e_ms / e2e_steps},
+            "gpu_launches": launches * args.steps,
+            "clocks": sampler.summary(t0, t1),
+            "roofline": {
+                "bound": "hbm", "kernel": "gemv_w4a16_kernel", "achieved": gbs_one, "peak": peak, "unit": "GB/s",
+                "frac": gbs_one / peak, "peak_source": "of " + peaks_kind,
+                "launches_per_step": launches, "avg_launch_us": 1e3 * ms_per_step / launches,
+                "algorithmic_bytes_per_launch": step_bytes / launches,
+                "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(args.workload),
+            },
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            b, s, layers, threads = oracle_stack_pass(model, config, M, 64, args.cpu_seconds, model["layers"])
+            line["cpu_baseline"] = {
+                "value": b / s / 1e9, "unit": UNIT, "cores": threads, "kind": "oracle",
+                "sample": "%d of %d layers, %d token, %.1f s of oracle time" % (layers, model["layers"], M, s),
+            }
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
+    ap.add_argument("--no-graph", action="store_true", help="issue the launches directly instead of replaying a CUDA graph")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-seconds", type=float, default=10.0, help="oracle time budget of the cpu_baseline leg")
+    args = ap.parse_args()
+    if args.steps is None:
+        args.steps = 3000 if args.impl == "ours" else 5
+    if args.warmup is None:
+        args.warmup = 50 if args.impl == "ours" else 3
+    args.steps = max(args.steps, 1)
+    args.warmup = max(args.warmup, 3)
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

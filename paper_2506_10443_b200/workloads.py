@@ -1,0 +1,117 @@
+"""Device-resident synthetic workloads shaped like the paper's evaluation models (Section 6): the
+linear layers of a decoder stack, packed once ("weights are determined when the model is loaded",
+Section 5.1) and then driven token by token (decode) or prompt by prompt (prefill).
+
+Only plumbing lives here: seeded arrays from ``inputs`` are packed with the library's host packer,
+copied to the GPU, and the launches of one step are issued through the C ABI.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+from typing import Dict, List, Optional, Tuple
+
+import numpy as np
+import torch
+
+from . import binding as B
+from . import inputs
+
+# which linears of a decoder layer read the same activations: (q, k, v), (o), (gate, up), (down)
+_INPUT_OF = {"q": 0, "k": 0, "v": 0, "o": 1, "gate": 2, "up": 2, "down": 3}
+_INPUT_SEED_ID = {0: 0, 1: 3, 2: 4, 3: 6}
+
+
+def w4_bytes(N: int, K: int, group: int) -> int:
+    """Bytes of codes plus fp16 (scale, zero) pairs of an [N, K] matrix."""
+    return N * K // 2 + N * (K // group) * 4
+
+
+def linear_bytes(N: int, K: int, group: int, M: int, y_bytes: int = 2) -> int:
+    """Bytes the W4A16 linear has to move: packed weights once, activations in, outputs out."""
+    return w4_bytes(N, K, group) + 2 * M * K + y_bytes * M * N
+
+
+@dataclass
+class _Layer:
+    packed: Dict[str, torch.Tensor] = field(default_factory=dict)
+    x_off: Dict[int, Tuple[int, int]] = field(default_factory=dict)   # input id -> (offset, K) in halfs
+    y_off: Dict[str, Tuple[int, int]] = field(default_factory=dict)   # linear -> (offset, N) in halfs
+
+
+class LinearStack:
+    """All linears of ``layers`` decoder layers of ``model`` for ``M`` tokens.
+
+    ``xin`` holds every layer's four input activations back to back ([M, K] each), ``yout`` every
+    linear's output ([M, N] each); ``xin_host`` / ``yout_host`` are pinned mirrors for end-to-end
+    timing.  ``run_w4a16`` issues the decode launches of one step: per layer one batched launch
+    for q, k, v (same input), one for o, one batched for gate and up, one for down.
+    """
+
+    def __init__(self, model: dict, config: int, M: int, group: int = 64, layers: Optional[int] = None,
+                 outliers: bool = False, device: str = "cuda"):
+        self.model, self.config, self.M, self.group = model, config, M, group
+        self.n_layers = model["layers"] if layers is None else layers
+        self.linears = inputs.stack(model)
+        self.device = torch.device(device)
+        xs: List[np.ndarray] = []
+        x_total = y_total = 0
+        self.layers: List[_Layer] = []
+        self.weight_bytes = 0
+        self.algorithmic_bytes_w4a16 = 0
+        self.ops = 0
+        for l in range(self.n_layers):
+            L = _Layer()
+            for lin in self.linears:
+                W = inputs.weights(inputs.seed_for(config, l, lin.matrix_id, 0), lin.N, lin.K)
+                L.packed[lin.name] = torch.from_numpy(B.pack_w4(W, group)).to(self.device)
+                del W
+                iid = _INPUT_OF[lin.name]
+                if iid not in L.x_off:
+                    x = inputs.activations(inputs.seed_for(config, l, _INPUT_SEED_ID[iid], 1), M, lin.K,
+                                           outliers=outliers)
+                    L.x_off[iid] = (x_total, lin.K)
+                    xs.append(x.reshape(-1))
+                    x_total += M * lin.K
+                L.y_off[lin.name] = (y_total, lin.N)
+                y_total += M * lin.N
+                self.weight_bytes += w4_bytes(lin.N, lin.K, group)
+                self.algorithmic_bytes_w4a16 += linear_bytes(lin.N, lin.K, group, M)
+                self.ops += 2 * M * lin.N * lin.K
+            self.layers.append(L)
+        self.xin_host = torch.from_numpy(np.concatenate(xs)).pin_memory()
+        self.xin = self.xin_host.to(self.device)
+        self.yout = torch.zeros(y_total, dtype=torch.float16, device=self.device)
+        self.yout_host = torch.empty(y_total, dtype=torch.float16).pin_memory()
+        self._launches = None
+
+    # ---- views ----
+    def x_view(self, layer: int, name: str) -> torch.Tensor:
+        off, K = self.layers[layer].x_off[_INPUT_OF[name]]
+        return self.xin[off:off + self.M * K].view(self.M, K)
+
+    def y_view(self, layer: int, name: str) -> torch.Tensor:
+        off, N = self.layers[layer].y_off[name]
+        return self.yout[off:off + self.M * N].view(self.M, N)
+
+    # ---- decode ----
+    def _decode_launches(self):
+        if self._launches is None:
+            out = []
+            for l, L in enumerate(self.layers):
+                for names in (("q", "k", "v"), ("o",), ("gate", "up"), ("down",)):
+                    probs = []
+                    for name in names:
+                        lin = next(t for t in self.linears if t.name == name)
+                        probs.append(dict(x=self.x_view(l, name), packed=L.packed[name], y=self.y_view(l, name),
+                                          N=lin.N, K=lin.K, group=self.group, y_dtype=B.F16))
+                    out.append(B.make_batch(probs))
+            self._launches = out
+        return self._launches
+
+    @property
+    def launches_per_step_w4a16(self) -> int:
+        return 4 * self.n_layers * ((self.M + 7) // 8)
+
+    def run_w4a16(self, stream=None) -> None:
+        for arr in self._decode_launches():
+            B.linear_w4a16_batch(arr, self.M, stream)
