@@ -21,6 +21,7 @@ SOURCES = [
     "gemv_w4a16.cu",
     "gemv_w8a16.cu",
     "act_quant.cu",
+    "gemm_w4a8.cu",
     "api_w4a8.cu",
 ]
 

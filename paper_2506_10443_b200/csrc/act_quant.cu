@@ -4,6 +4,10 @@
 // and, for the zero-point correction of the asymmetric weights, the group sums A[m,g] = sum a_q.
 // One CTA per token; the row is read twice (the second read hits L2).  HBM-bound and tiny next to
 // the GEMM it feeds.
+//
+// For the GEMM's tensor-core evaluation of the zero-point term sum_g (s z)[n,g] * A[m,g] the group
+// sums are also written as fp16 quadruples (64h, l, 64h, l) with A = 64h + l, h = round(A / 64),
+// l in [-32, 31]: both parts are exact in fp16 (|A| <= 127 * 128), so the term loses nothing.
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
@@ -41,7 +45,7 @@ __device__ __forceinline__ void widen8<__nv_bfloat16>(const uint4& v, float (&f)
 template <typename T>
 __global__ void __launch_bounds__(kThreads) act_quant_kernel(const T* __restrict__ x, int K, int group,
                                                              int8_t* __restrict__ a_q, float* __restrict__ a_scale,
-                                                             int32_t* __restrict__ A) {
+                                                             int32_t* __restrict__ A, uint2* __restrict__ AC, int G4) {
     __shared__ float warp_max[kThreads / 32];
     ptx::pdl_launch_dependents();
     ptx::pdl_wait();
@@ -70,6 +74,8 @@ __global__ void __launch_bounds__(kThreads) act_quant_kernel(const T* __restrict
     const int lanes_per_group = group / 8;  // 8 or 16 consecutive lanes share a group
     uint2* out = reinterpret_cast<uint2*>(a_q + (size_t)m * K);
     const int G = K / group;
+    if (AC != nullptr)  // groups that only pad the row to a multiple of four
+        for (int g = G + threadIdx.x; g < G4; g += kThreads) AC[(size_t)m * G4 + g] = make_uint2(0u, 0u);
     for (int v0 = 0; v0 < nvec; v0 += kThreads) {
         const int v = v0 + threadIdx.x;
         int sum = 0;
@@ -98,7 +104,16 @@ __global__ void __launch_bounds__(kThreads) act_quant_kernel(const T* __restrict
         if (lanes_per_group == 16) sum += __shfl_xor_sync(0xffffffffu, sum, 8);
         if (v < nvec && (threadIdx.x % lanes_per_group) == 0) {
             const int g = v / lanes_per_group;
-            if (g < G) A[(size_t)m * G + g] = sum;
+            if (g < G) {
+                if (A != nullptr) A[(size_t)m * G + g] = sum;
+                if (AC != nullptr) {
+                    const int h = (sum + 32) >> 6;  // floor((sum + 32) / 64)
+                    const int l = sum - 64 * h;
+                    const __half2 hl = __floats2half2_rn((float)(64 * h), (float)l);
+                    const uint32_t bits = *reinterpret_cast<const uint32_t*>(&hl);
+                    AC[(size_t)m * G4 + g] = make_uint2(bits, bits);
+                }
+            }
         }
     }
 }
@@ -106,7 +121,9 @@ __global__ void __launch_bounds__(kThreads) act_quant_kernel(const T* __restrict
 }  // namespace
 
 cudaError_t act_quant_launch(const void* x, int x_dtype, int M, int K, int group, int8_t* a_q, float* a_scale,
-                             int32_t* A, cudaStream_t stream) {
+                             int32_t* A, void* AC, cudaStream_t stream) {
+    const int G4 = (K / group + 3) / 4 * 4;
+    uint2* ac = reinterpret_cast<uint2*>(AC);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)M);
     cfg.blockDim = dim3(kThreads);
@@ -117,9 +134,10 @@ cudaError_t act_quant_launch(const void* x, int x_dtype, int M, int K, int group
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     if (x_dtype == MNNLLM_F16)
-        return cudaLaunchKernelEx(&cfg, act_quant_kernel<__half>, (const __half*)x, K, group, a_q, a_scale, A);
+        return cudaLaunchKernelEx(&cfg, act_quant_kernel<__half>, (const __half*)x, K, group, a_q, a_scale, A, ac,
+                                  G4);
     return cudaLaunchKernelEx(&cfg, act_quant_kernel<__nv_bfloat16>, (const __nv_bfloat16*)x, K, group, a_q, a_scale,
-                              A);
+                              A, ac, G4);
 }
 
 }  // namespace mnnllm

@@ -1,11 +1,14 @@
-// C-ABI entry points of the W4A8 prefill path.
+// C-ABI entry points of the W4A8 prefill path: argument checks, workspace carve-up, and the two
+// launches (activation quantiser, then the tensor-core GEMM).
 #include "act_quant.h"
 #include "common.h"
+#include "gemm_w4a8.h"
 #include "layout.h"
 
 using namespace mnnllm;
 
 namespace {
+
 int check_xq(const void* x, int x_dtype, int M, int K, int group) {
     if (!x || M < 1 || K < 1) return MNNLLM_ERR_INVALID_ARG;
     if (x_dtype != MNNLLM_F16 && x_dtype != MNNLLM_BF16) return MNNLLM_ERR_UNSUPPORTED;
@@ -13,6 +16,23 @@ int check_xq(const void* x, int x_dtype, int M, int K, int group) {
     if ((uintptr_t)x & 15) return MNNLLM_ERR_ALIGNMENT;
     return MNNLLM_OK;
 }
+
+size_t round256(size_t v) { return (v + 255) & ~(size_t)255; }
+
+// workspace: a_q int8 [M, K] | a_scale fp32 [M] | fp16 group-sum quadruples [M, G4] x 8 bytes
+struct Workspace {
+    size_t a_q, a_scale, ac, total;
+};
+Workspace workspace_layout(int M, int K, int group) {
+    Workspace w;
+    const size_t G4 = (size_t)(K / group + 3) / 4 * 4;
+    w.a_q = 0;
+    w.a_scale = round256((size_t)M * K);
+    w.ac = w.a_scale + round256((size_t)M * 4);
+    w.total = w.ac + round256((size_t)M * G4 * 8);
+    return w;
+}
+
 }  // namespace
 
 extern "C" {
@@ -24,20 +44,75 @@ int mnnllm_quantize_activations(const void* x, int x_dtype, int M, int K, int gr
     if (!a_q || !a_scale || !A) return MNNLLM_ERR_INVALID_ARG;
     if (((uintptr_t)a_q & 15) || ((uintptr_t)a_scale & 3) || ((uintptr_t)A & 3)) return MNNLLM_ERR_ALIGNMENT;
     if (!device_is_supported()) return MNNLLM_ERR_UNSUPPORTED;
-    if (act_quant_launch(x, x_dtype, M, K, group, a_q, a_scale, A, (cudaStream_t)stream) != cudaSuccess) {
+    if (act_quant_launch(x, x_dtype, M, K, group, a_q, a_scale, A, nullptr, (cudaStream_t)stream) != cudaSuccess) {
         (void)cudaGetLastError();
         return MNNLLM_ERR_CUDA;
     }
     return MNNLLM_OK;
 }
 
-size_t mnnllm_workspace_size_w4a8(int M, int N, int K, int group) { return 0; }
-int mnnllm_linear_w4a8(const void*, const void*, void*, int, int, int, int, int, int, void*, size_t, void*) {
-    return MNNLLM_ERR_UNSUPPORTED;
+size_t mnnllm_workspace_size_w4a8(int M, int N, int K, int group) {
+    if (M < 1 || N < 1 || K < 1 || (group != 64 && group != 128) || K % group != 0) return 0;
+    return workspace_layout(M, K, group).total;
 }
-int mnnllm_debug_w4a8_partials(const void*, int, const void*, int32_t*, int8_t*, float*, int32_t*, int, int, int, int,
-                               void*) {
-    return MNNLLM_ERR_UNSUPPORTED;
+
+int mnnllm_linear_w4a8(const void* x, const void* packed, void* y, int M, int N, int K, int group, int x_dtype,
+                       int y_dtype, void* workspace, size_t workspace_bytes, void* stream) {
+    const int st = check_xq(x, x_dtype, M, K, group);
+    if (st != MNNLLM_OK) return st;
+    if (!packed || !y || N < 1) return MNNLLM_ERR_INVALID_ARG;
+    if (y_dtype != MNNLLM_F16 && y_dtype != MNNLLM_BF16 && y_dtype != MNNLLM_F32) return MNNLLM_ERR_UNSUPPORTED;
+    if (((uintptr_t)y & 15) || ((uintptr_t)packed & 127)) return MNNLLM_ERR_ALIGNMENT;
+    const Workspace w = workspace_layout(M, K, group);
+    if (!workspace || workspace_bytes < w.total) return MNNLLM_ERR_WORKSPACE;
+    if ((uintptr_t)workspace & 255) return MNNLLM_ERR_ALIGNMENT;
+    if (!device_is_supported()) return MNNLLM_ERR_UNSUPPORTED;
+    uint32_t* status = status_word_ptr();
+    if (!status) return MNNLLM_ERR_CUDA;
+
+    uint8_t* ws = (uint8_t*)workspace;
+    int8_t* a_q = (int8_t*)(ws + w.a_q);
+    float* a_scale = (float*)(ws + w.a_scale);
+    void* ac = ws + w.ac;
+    if (act_quant_launch(x, x_dtype, M, K, group, a_q, a_scale, nullptr, ac, (cudaStream_t)stream) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return MNNLLM_ERR_CUDA;
+    }
+    GemmW4A8Args a;
+    a.packed = packed; a.a_q = a_q; a.a_scale = a_scale; a.AC = ac; a.y = y; a.P = nullptr;
+    a.M = M; a.N = N; a.K = K; a.group = group; a.y_dtype = y_dtype;
+    const cudaError_t e = gemm_w4a8_launch(a, status, (cudaStream_t)stream);
+    if (e != cudaSuccess) {
+        (void)cudaGetLastError();
+        return e == cudaErrorNotSupported ? MNNLLM_ERR_UNSUPPORTED : MNNLLM_ERR_CUDA;
+    }
+    return MNNLLM_OK;
+}
+
+int mnnllm_debug_w4a8_partials(const void* x, int x_dtype, const void* packed, int32_t* P, int8_t* a_q, float* a_scale,
+                               int32_t* A, int M, int N, int K, int group, void* stream) {
+    const int st = check_xq(x, x_dtype, M, K, group);
+    if (st != MNNLLM_OK) return st;
+    if (!packed || !P || !a_q || !a_scale || !A || N < 1) return MNNLLM_ERR_INVALID_ARG;
+    if (((uintptr_t)a_q & 15) || ((uintptr_t)a_scale & 3) || ((uintptr_t)A & 3) || ((uintptr_t)P & 3) ||
+        ((uintptr_t)packed & 127))
+        return MNNLLM_ERR_ALIGNMENT;
+    if (!device_is_supported()) return MNNLLM_ERR_UNSUPPORTED;
+    uint32_t* status = status_word_ptr();
+    if (!status) return MNNLLM_ERR_CUDA;
+    if (act_quant_launch(x, x_dtype, M, K, group, a_q, a_scale, A, nullptr, (cudaStream_t)stream) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return MNNLLM_ERR_CUDA;
+    }
+    GemmW4A8Args a;
+    a.packed = packed; a.a_q = a_q; a.a_scale = a_scale; a.AC = nullptr; a.y = nullptr; a.P = P;
+    a.M = M; a.N = N; a.K = K; a.group = group; a.y_dtype = MNNLLM_F32;
+    const cudaError_t e = gemm_w4a8_launch(a, status, (cudaStream_t)stream);
+    if (e != cudaSuccess) {
+        (void)cudaGetLastError();
+        return e == cudaErrorNotSupported ? MNNLLM_ERR_UNSUPPORTED : MNNLLM_ERR_CUDA;
+    }
+    return MNNLLM_OK;
 }
 
 }  // extern "C"

@@ -1,0 +1,462 @@
+// Prefill W4A8 linear (Section 4.2: activations quantised to int8 so that integer matrix
+// instructions can be used; Section 5.1 for the operand shapes):
+//     P[m,n,g] = sum_{k in g} a_q[m,k] * q[n,k]                       int32, exact
+//     y[m,n]   = a_scale[m] * ( sum_g s[n,g] * P[m,n,g]  -  sum_g (s z)[n,g] * A[m,g] )
+//
+// One CTA computes a tile of 128 weight rows x 128 tokens.  The weights are the M side of the MMA,
+// so that a tensor-memory lane is one output channel n and its per-group scale is a per-thread
+// scalar in the drain.  Warp roles (14 warps):
+//   warp 0      producer: TMA loads of the int8 activation tile (128 tokens x 128 k, 128B swizzle)
+//               and of the fp16 group-sum quadruples that feed the zero-point MMA
+//   warp 1      allocates tensor memory, issues tcgen05.mma (kind::i8 into one of two int32
+//               accumulators per group; kind::f16 for the zero-point term) and the commits
+//   warps 2-5   unpack: packed int4 codes (global, coalesced 16-byte loads, register prefetch three
+//               stages ahead) -> int8 K-major tile in the 128B-swizzled layout the MMA reads; the
+//               row's fp32 scale for the drain; (s z) split into fp16 hi + lo for the zero-point MMA
+//   warps 6-13  drain: every group's 128 x 128 int32 partial tile leaves tensor memory
+//               (tcgen05.ld), is converted and accumulated as acc += s * P in registers while the
+//               MMA fills the other accumulator; epilogue applies the zero-point term and a_scale.
+// The zero-point term is a rank-G product, evaluated on the tensor cores without loss:
+//   (s z) = hi + lo (fp16 each; s and z are fp16, so the product has 22 significant bits),
+//   A     = 64 h + l (both exact in fp16), four fp16 products per group, fp32 accumulation in a
+//   third tensor-memory region; 4 groups fill one K = 16 MMA.
+// Every wait is bounded: on a time-out the CTA records a code in the status word and all roles
+// leave their loops, tensor memory is released and the kernel returns.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
+#include "gemm_w4a8.h"
+#include "layout.h"
+#include "ptx.cuh"
+
+namespace mnnllm {
+
+using namespace ptx;
+
+namespace {
+
+constexpr int kTileN = 128;   // weight rows per CTA tile (MMA M)
+constexpr int kTileT = 128;   // tokens per CTA tile (MMA N)
+constexpr int kStageK = 128;  // k per pipeline stage (one 128-byte swizzle row of int8)
+constexpr int kStages = 4;
+constexpr int kScaleSlots = 2 * kStages + 2;  // groups whose scales may be live at once
+constexpr int kPrefetch = 3;                  // stages of packed codes held in registers ahead of use
+constexpr int kThreads = 14 * 32;
+constexpr int kUnpackWarp0 = 2, kDrainWarp0 = 6;
+constexpr uint32_t kMaxPolls = 1u << 22;
+constexpr uint32_t kTmemCols = 512;           // 2 x 128 int32 accumulators + 128 fp32 zero-point term
+constexpr uint32_t kColCorr = 256;
+
+constexpr int kStageBytes = kTileN * kStageK;  // 16 KiB, int8
+constexpr int kCorrBytes = 128 * 32;           // 128 rows x 16 fp16
+
+struct Smem {
+    static constexpr int wq = 0;
+    static constexpr int aq = wq + kStages * kStageBytes;
+    static constexpr int ca = aq + kStages * kStageBytes;
+    static constexpr int cb = ca + 2 * kCorrBytes;
+    static constexpr int scale = cb + 2 * kCorrBytes;
+    static constexpr int bars = scale + kScaleSlots * kTileN * 4;
+    static constexpr int n_bars = 2 * kStages + 2 + 2 + 2 + 2 + 1;
+    static constexpr int misc = bars + n_bars * 8;
+    static constexpr int total = misc + 16;
+};
+constexpr size_t kSmemBytes = Smem::total + 1024;  // slack to align the base to 1024 bytes
+
+struct Params {
+    const uint8_t* packed;
+    const float* a_scale;
+    void* y;
+    int32_t* P;
+    int M, N, K, G;
+    int n_row_blocks, n_slabs, n_stages;
+    int y_dtype;
+    unsigned long long row_block_bytes, chunk_bytes;
+};
+
+// K-major operand tile whose rows are 128 bytes, 128B swizzle: 8-row groups are 1024 bytes apart.
+__device__ __forceinline__ uint64_t desc_sw128(uint32_t smem_addr) {
+    return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+// K-major operand tile whose rows are 32 bytes, 32B swizzle: 8-row groups are 256 bytes apart.
+__device__ __forceinline__ uint64_t desc_sw32(uint32_t smem_addr) {
+    return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | (1ull << 16) | (16ull << 32) | (1ull << 46) | (6ull << 61);
+}
+// instruction descriptors: D format (bits 4-5), A/B formats (7-9, 10-12), both K-major, N >> 3 at
+// bit 17, M >> 4 at bit 24
+constexpr uint32_t kIdescI8 = (2u << 4) | (1u << 7) | (1u << 10) | ((kTileT >> 3) << 17) | ((kTileN >> 4) << 24);
+constexpr uint32_t kIdescF16 = (1u << 4) | (0u << 7) | (0u << 10) | ((kTileT >> 3) << 17) | ((kTileN >> 4) << 24);
+
+__device__ __forceinline__ void store_y(void* y, int dtype, size_t idx, float v) {
+    if (dtype == MNNLLM_F16) reinterpret_cast<__half*>(y)[idx] = __float2half_rn(v);
+    else if (dtype == MNNLLM_BF16) reinterpret_cast<__nv_bfloat16*>(y)[idx] = __float2bfloat16_rn(v);
+    else reinterpret_cast<float*>(y)[idx] = v;
+}
+
+template <int GROUP, bool PARTIALS>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ CUtensorMap tm_ac,
+                 const __grid_constant__ Params p, uint32_t* __restrict__ status) {
+    constexpr int GPS = kStageK / GROUP;  // groups per stage (2 or 1)
+    constexpr int SPB = 4 / GPS;          // stages per block of four groups (zero-point MMA cadence)
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + Smem::bars);
+    uint64_t* ab_full = bars;
+    uint64_t* ab_empty = ab_full + kStages;
+    uint64_t* tm_full = ab_empty + kStages;
+    uint64_t* tm_empty = tm_full + 2;
+    uint64_t* c_full = tm_empty + 2;
+    uint64_t* c_empty = c_full + 2;
+    uint64_t* corr_done = c_empty + 2;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + Smem::misc);
+    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + Smem::misc + 4);
+    float* scale_ring = reinterpret_cast<float*>(smem + Smem::scale);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n0 = blockIdx.x * kTileN, m0 = blockIdx.y * kTileT;
+    const int n_stages = p.n_stages, G = p.G;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < kStages; ++i) { mbar_init(&ab_full[i], 5); mbar_init(&ab_empty[i], 1); }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&tm_full[i], 1); mbar_init(&tm_empty[i], 8);
+            mbar_init(&c_full[i], 5); mbar_init(&c_empty[i], 1);
+        }
+        mbar_init(corr_done, 1);
+        *abort_flag = 0;
+        fence_mbar_init();
+        prefetch_tensormap(&tm_act);
+        if (!PARTIALS) prefetch_tensormap(&tm_ac);
+    }
+    if (warp == 1) {
+        tmem_alloc(tmem_slot, kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    // a failed wait marks the CTA as aborted; every role then leaves its loop
+    auto wait = [&](uint64_t* bar, uint32_t parity, uint32_t code) -> bool {
+        if (mbar_wait_bounded(bar, parity, kMaxPolls)) return true;
+        if (*abort_flag == 0) {
+            *abort_flag = 1;
+            atomicOr(status, 0x200u | code);
+        }
+        return false;
+    };
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ producer (TMA)
+        for (int st = 0; st < n_stages && !*abort_flag; ++st) {
+            const int slot = st % kStages, round = st / kStages;
+            if (!wait(&ab_empty[slot], (round & 1) ^ 1, 1)) break;
+            if (lane == 0) {
+                mbar_arrive_expect_tx(&ab_full[slot], kTileT * kStageK);
+                tma_load_2d(smem + Smem::aq + slot * kStageBytes, &tm_act, st * kStageK, m0, &ab_full[slot]);
+            }
+            if (!PARTIALS && st % SPB == 0) {
+                const int cblk = st / SPB, cslot = cblk & 1;
+                if (!wait(&c_empty[cslot], ((cblk >> 1) & 1) ^ 1, 2)) break;
+                if (lane == 0) {
+                    mbar_arrive_expect_tx(&c_full[cslot], kTileT * 32);
+                    tma_load_2d(smem + Smem::cb + cslot * kCorrBytes, &tm_ac, cblk * 16, m0, &c_full[cslot]);
+                }
+            }
+            __syncwarp();
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issue
+        int gcount = 0, ccount = 0;
+        const uint32_t wq_addr = smem_u32(smem + Smem::wq), aq_addr = smem_u32(smem + Smem::aq);
+        bool ok = true;
+        for (int st = 0; st < n_stages && ok && !*abort_flag; ++st) {
+            const int slot = st % kStages, round = st / kStages;
+            if (!wait(&ab_full[slot], round & 1, 3)) break;
+            tc_fence_after_sync();
+            const int ngr = (G - st * GPS) < GPS ? (G - st * GPS) : GPS;
+            for (int gi = 0; gi < ngr; ++gi) {
+                const int b = gcount & 1;
+                if (!wait(&tm_empty[b], ((gcount >> 1) & 1) ^ 1, 4)) { ok = false; break; }
+                tc_fence_after_sync();
+                if (lane == 0) {
+                    const uint64_t da = desc_sw128(wq_addr + slot * kStageBytes);
+                    const uint64_t db = desc_sw128(aq_addr + slot * kStageBytes);
+#pragma unroll
+                    for (int kk = 0; kk < GROUP / 32; ++kk) {
+                        const uint64_t adv = (uint64_t)((gi * GROUP + kk * 32) >> 4);
+                        mma_i8_ss(tmem_base + b * kTileT, da + adv, db + adv, kIdescI8, kk > 0);
+                    }
+                    mma_commit(&tm_full[b]);
+                }
+                __syncwarp();
+                ++gcount;
+            }
+            if (!ok) break;
+            if (lane == 0) mma_commit(&ab_empty[slot]);
+            if (!PARTIALS && ((gcount & 3) == 0 || st == n_stages - 1)) {
+                const int cslot = ccount & 1;
+                if (!wait(&c_full[cslot], (ccount >> 1) & 1, 5)) break;
+                tc_fence_after_sync();
+                if (lane == 0) {
+                    mma_f16_ss(tmem_base + kColCorr, desc_sw32(smem_u32(smem + Smem::ca + cslot * kCorrBytes)),
+                               desc_sw32(smem_u32(smem + Smem::cb + cslot * kCorrBytes)), kIdescF16, ccount > 0);
+                    mma_commit(&c_empty[cslot]);
+                }
+                ++ccount;
+            }
+            __syncwarp();
+        }
+        if (!PARTIALS && lane == 0) mma_commit(corr_done);
+        __syncwarp();
+    } else if (warp < kDrainWarp0) {
+        // ------------------------------------------------------------------ unpack
+        const int u = threadIdx.x - kUnpackWarp0 * 32;  // 0..127 = row of the tile this thread owns for scales
+        const int wu = u >> 5;
+        const int rb0 = n0 / kRowsPerBlock;
+        const uint8_t* body = p.packed + kHeaderBytes;
+        auto load_codes = [&](int st, uint4 (&e)[4]) {
+            const int j = st >> 2;
+            const int ns_chunk = (p.n_slabs - 8 * j) < 8 ? (p.n_slabs - 8 * j) : 8;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int sidx = i * 4 + wu;
+                const int rb = rb0 + (sidx >> 1), sl = (st & 3) * 2 + (sidx & 1);
+                e[i] = make_uint4(0, 0, 0, 0);
+                if (st < n_stages && rb < p.n_row_blocks && sl < ns_chunk)
+                    e[i] = __ldg(reinterpret_cast<const uint4*>(body + (size_t)rb * p.row_block_bytes +
+                                                                (size_t)j * p.chunk_bytes + (size_t)sl * kSlabBytes) + lane);
+            }
+        };
+        auto load_sz = [&](int st, uint32_t (&sz)[GPS]) {
+            const int j = st >> 2;
+            const int ns_chunk = (p.n_slabs - 8 * j) < 8 ? (p.n_slabs - 8 * j) : 8;
+            const int ng = ns_chunk * kSlabK4 / GROUP;
+            const int rb = rb0 + (u >> 4), r16 = u & 15;
+#pragma unroll
+            for (int gi = 0; gi < GPS; ++gi) {
+                const int gc = (st & 3) * GPS + gi;
+                sz[gi] = 0;
+                if (st < n_stages && rb < p.n_row_blocks && gc < ng)
+                    sz[gi] = __ldg(reinterpret_cast<const uint32_t*>(body + (size_t)rb * p.row_block_bytes +
+                                                                     (size_t)j * p.chunk_bytes +
+                                                                     (size_t)ns_chunk * kSlabBytes) + r16 * ng + gc);
+            }
+        };
+        uint4 e0[4], e1[4], e2[4];
+        uint32_t z0[GPS], z1[GPS], z2[GPS];
+        load_codes(0, e0); load_sz(0, z0);
+        load_codes(1, e1); load_sz(1, z1);
+        load_codes(2, e2); load_sz(2, z2);
+        static_assert(kPrefetch == 3, "the register ring below holds three stages");
+        bool ok = true;
+        for (int st = 0; st < n_stages && ok && !*abort_flag; ++st) {
+            const int slot = st % kStages, round = st / kStages;
+            uint4 cur[4];
+            uint32_t zc[GPS];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) { cur[i] = e0[i]; e0[i] = e1[i]; e1[i] = e2[i]; }
+#pragma unroll
+            for (int i = 0; i < GPS; ++i) { zc[i] = z0[i]; z0[i] = z1[i]; z1[i] = z2[i]; }
+            load_codes(st + kPrefetch, e2);
+            load_sz(st + kPrefetch, z2);
+            if (!wait(&ab_empty[slot], (round & 1) ^ 1, 6)) break;
+
+            // scales for the drain, (s z) halves for the zero-point MMA: this thread's row u
+#pragma unroll
+            for (int gi = 0; gi < GPS; ++gi) {
+                const int g = st * GPS + gi;
+                if (g >= G) break;
+                const __half2 h2 = *reinterpret_cast<const __half2*>(&zc[gi]);
+                const float s = __low2float(h2), z = __high2float(h2);
+                scale_ring[(g % kScaleSlots) * kTileN + u] = s;
+                if (!PARTIALS) {
+                    const int pos = g & 3, cblk = g >> 2, cslot = cblk & 1;
+                    if (pos == 0 && !wait(&c_empty[cslot], ((cblk >> 1) & 1) ^ 1, 7)) { ok = false; break; }
+                    const float szf = s * z;  // exact: 11-bit x 11-bit significands
+                    const __half hi = __float2half_rn(szf);
+                    const __half lo = __float2half_rn(szf - __half2float(hi));
+                    const uint32_t hh = (uint32_t)__half_as_ushort(hi) * 0x00010001u;
+                    const uint32_t ll = (uint32_t)__half_as_ushort(lo) * 0x00010001u;
+                    uint8_t* tile = smem + Smem::ca + cslot * kCorrBytes;
+                    const int rowoff = (u >> 3) * 256 + (u & 7) * 32, sw = (u & 7) >> 2;
+                    *reinterpret_cast<uint2*>(tile + rowoff + (((pos >> 1) ^ sw) << 4) + (pos & 1) * 8) = make_uint2(hh, ll);
+                    if (pos == 3 || g == G - 1) {
+                        for (int q = pos + 1; q < 4; ++q)
+                            *reinterpret_cast<uint2*>(tile + rowoff + (((q >> 1) ^ sw) << 4) + (q & 1) * 8) = make_uint2(0u, 0u);
+                        fence_proxy_async_smem();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&c_full[cslot]);
+                    }
+                }
+            }
+            if (!ok) break;
+
+            // codes -> int8, 128B-swizzled K-major rows
+            uint8_t* wq = smem + Smem::wq + slot * kStageBytes;
+            const int r = lane >> 2, c = lane & 3;
+            constexpr uint32_t M4 = 0x0F0F0F0Fu;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int sidx = i * 4 + wu;
+                const int R0 = (sidx >> 1) * 16 + r;          // rows R0 and R0 + 8 of the tile
+                const int kc = (sidx & 1) * 4 + c;            // 16-byte chunk of the 128-byte row
+                const uint32_t off = (uint32_t)(R0 >> 3) * 1024u + (uint32_t)r * 128u + (uint32_t)((kc ^ r) << 4);
+                const uint4 w = cur[i];
+                *reinterpret_cast<uint4*>(wq + off) = make_uint4(w.x & M4, (w.x >> 4) & M4, w.y & M4, (w.y >> 4) & M4);
+                *reinterpret_cast<uint4*>(wq + off + 1024u) = make_uint4(w.z & M4, (w.z >> 4) & M4, w.w & M4, (w.w >> 4) & M4);
+            }
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&ab_full[slot]);
+        }
+    } else {
+        // ------------------------------------------------------------------ drain + epilogue
+        const int q4 = warp & 3;                      // tensor-memory lane quarter this warp may read
+        const int half = (warp - kDrainWarp0) >> 2;   // which 64 token columns
+        const int nl = q4 * 32 + lane, n = n0 + nl;
+        const uint32_t lane_base = tmem_base + ((uint32_t)(q4 * 32) << 16);
+        float acc[64];
+#pragma unroll
+        for (int i = 0; i < 64; ++i) acc[i] = 0.f;
+        bool ok = true;
+        for (int g = 0; g < G && !*abort_flag; ++g) {
+            const int b = g & 1;
+            if (!wait(&tm_full[b], (g >> 1) & 1, 8)) { ok = false; break; }
+            tc_fence_after_sync();
+            const float sf = scale_ring[(g % kScaleSlots) * kTileN + nl];
+#pragma unroll
+            for (int cc = 0; cc < 2; ++cc) {
+                uint32_t v[32];
+                tmem_ld_x32(lane_base + b * kTileT + half * 64 + cc * 32, v);
+                tmem_ld_wait();
+                if (PARTIALS) {
+                    if (n < p.N)
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            const int m = m0 + half * 64 + cc * 32 + j;
+                            if (m < p.M) p.P[((size_t)m * p.N + n) * G + g] = (int32_t)v[j];
+                        }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) acc[cc * 32 + j] = fmaf(sf, (float)(int32_t)v[j], acc[cc * 32 + j]);
+                }
+            }
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&tm_empty[b]);
+        }
+        if (!PARTIALS && ok && !*abort_flag && wait(corr_done, 0, 9)) {
+            tc_fence_after_sync();
+#pragma unroll
+            for (int cc = 0; cc < 2; ++cc) {
+                uint32_t v[32];
+                tmem_ld_x32(lane_base + kColCorr + half * 64 + cc * 32, v);
+                tmem_ld_wait();
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    const int m = m0 + half * 64 + cc * 32 + j;
+                    if (m < p.M && n < p.N) {
+                        const float val = __ldg(p.a_scale + m) * (acc[cc * 32 + j] - __uint_as_float(v[j]));
+                        store_y(p.y, p.y_dtype, (size_t)m * p.N + n, val);
+                    }
+                }
+            }
+        }
+    }
+
+    // ---- teardown: after an abort give copies in flight time to land before the CTA goes away ----
+    if (*abort_flag) {
+        const long long t0 = clock64();
+        while (clock64() - t0 < 400000) {}
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem_base, kTmemCols);
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)ptr;
+    }
+    return fn;
+}
+
+template <int GROUP, bool PARTIALS>
+cudaError_t launch(const CUtensorMap& tm_act, const CUtensorMap& tm_ac, const Params& p, dim3 grid, uint32_t* status,
+                   cudaStream_t stream) {
+    static bool configured = false;
+    auto kern = gemm_w4a8_kernel<GROUP, PARTIALS>;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    kern<<<grid, kThreads, kSmemBytes, stream>>>(tm_act, tm_ac, p, status);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t gemm_w4a8_launch(const GemmW4A8Args& a, uint32_t* status, cudaStream_t stream) {
+    EncodeTiledFn enc = encode_fn();
+    if (!enc) return cudaErrorNotSupported;
+    const W4Geometry geo = w4_geometry(a.N, a.K, a.group);
+    const bool partials = a.P != nullptr;
+
+    CUtensorMap tm_act, tm_ac;
+    {
+        const cuuint64_t dims[2] = {(cuuint64_t)a.K, (cuuint64_t)a.M};
+        const cuuint64_t strides[1] = {(cuuint64_t)a.K};
+        const cuuint32_t box[2] = {(cuuint32_t)kStageK, (cuuint32_t)kTileT};
+        const cuuint32_t estr[2] = {1, 1};
+        if (enc(&tm_act, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, (void*)a.a_q, dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return cudaErrorInvalidValue;
+    }
+    if (!partials) {
+        const int G4 = (geo.G + 3) / 4 * 4;
+        const cuuint64_t dims[2] = {(cuuint64_t)G4 * 4, (cuuint64_t)a.M};
+        const cuuint64_t strides[1] = {(cuuint64_t)G4 * 8};
+        const cuuint32_t box[2] = {16, (cuuint32_t)kTileT};
+        const cuuint32_t estr[2] = {1, 1};
+        if (enc(&tm_ac, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, (void*)a.AC, dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_32B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return cudaErrorInvalidValue;
+    } else {
+        tm_ac = tm_act;  // never read in the partials form
+    }
+
+    Params p;
+    p.packed = (const uint8_t*)a.packed;
+    p.a_scale = a.a_scale;
+    p.y = a.y;
+    p.P = a.P;
+    p.M = a.M; p.N = a.N; p.K = a.K; p.G = geo.G;
+    p.n_row_blocks = geo.n_row_blocks; p.n_slabs = geo.n_slabs;
+    p.n_stages = (a.K + kStageK - 1) / kStageK;
+    p.y_dtype = a.y_dtype;
+    p.row_block_bytes = geo.row_block_bytes; p.chunk_bytes = geo.chunk_bytes;
+    const dim3 grid((unsigned)((a.N + kTileN - 1) / kTileN), (unsigned)((a.M + kTileT - 1) / kTileT));
+    if (a.group == 64)
+        return partials ? launch<64, true>(tm_act, tm_ac, p, grid, status, stream)
+                        : launch<64, false>(tm_act, tm_ac, p, grid, status, stream);
+    return partials ? launch<128, true>(tm_act, tm_ac, p, grid, status, stream)
+                    : launch<128, false>(tm_act, tm_ac, p, grid, status, stream);
+}
+
+}  // namespace mnnllm
