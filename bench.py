@@ -25,9 +25,9 @@ if ROOT not in sys.path:
 
 import numpy as np  # noqa: E402
 
-METRIC = "decode W4 GEMV GB/s"
-UNIT = "GB/s"
 FALLBACK_HBM_GBS = 6650.0
+FALLBACK_BF16_TFLOPS = 1590.0        # burst; about 1400 sustained
+INT8_OVER_BF16 = 2.0                 # nominal dense tensor-rate ratio (4.5 POPS int8 : 2.25 PFLOPS bf16)
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel from the committed
 # ncu capture (profiles/), keyed by workload; None when no capture matches the current kernel.
@@ -39,7 +39,8 @@ def measured_peaks():
     if os.path.exists(path):
         with open(path) as f:
             return json.load(f), "measured"
-    return {"hbm_gbs": FALLBACK_HBM_GBS}, "fallback"
+    return {"hbm_gbs": FALLBACK_HBM_GBS, "bf16_tflops": FALLBACK_BF16_TFLOPS,
+            "bf16_tflops_sustained": 1400.0}, "fallback"
 
 
 class ClockSampler:
@@ -128,84 +129,106 @@ class ClockSampler:
 # --------------------------------------------------------------------------------------------------
 # workloads
 # --------------------------------------------------------------------------------------------------
+def _wl(model, config, M, kind):
+    return {"model": model, "config": config, "M": M, "kind": kind}
+
+
 WORKLOADS = {
-    # name: (model key, config number of the workload list, tokens per step)
-    "decode_qwen2_1p5b_w4a16_g64": ("QWEN2_1P5B", 2, 1),
-    "decode_qwen2_7b_w4a16_g64": ("QWEN2_7B", 4, 1),
+    # decode: one token through the stack, W4A16, HBM-bound; prefill: a prompt of M tokens, W4A8
+    "decode_qwen2_1p5b_w4a16_g64": _wl("QWEN2_1P5B", 2, 1, "decode"),
+    "decode_qwen2_7b_w4a16_g64": _wl("QWEN2_7B", 4, 1, "decode"),
+    "prefill_qwen2_1p5b_w4a8_g64_m64": _wl("QWEN2_1P5B", 3, 64, "prefill"),
+    "prefill_qwen2_1p5b_w4a8_g64_m256": _wl("QWEN2_1P5B", 3, 256, "prefill"),
+    "prefill_qwen2_1p5b_w4a8_g64_m1024": _wl("QWEN2_1P5B", 3, 1024, "prefill"),
+    "prefill_qwen2_7b_w4a8_g64_m512": _wl("QWEN2_7B", 4, 512, "prefill"),
 }
 DEFAULT_WORKLOAD = "decode_qwen2_1p5b_w4a16_g64"
+GROUP = 64
 
 
-def oracle_stack_pass(model, config, M, group, max_seconds, max_layers):
-    """Times the CPU oracle's W4A16 linear, layer by layer, until `max_seconds` have been spent or
-    `max_layers` layers are done.  Returns (algorithmic bytes processed, seconds, layers, threads)."""
-    import oracle
-    from paper_2506_10443_b200 import inputs
+def metric_of(kind):
+    """(metric, unit, dtype): decode is graded on bytes moved, prefill on integer operations."""
+    if kind == "decode":
+        return "decode W4 GEMV GB/s", "GB/s", "f32"
+    return "prefill W4A8 TOPS", "TOPS", "int8"
+
+
+def units_of_linear(kind, N, K, M):
+    """Algorithmic work of one linear in the metric's unit x 1e9 (bytes) or x 1e12 (int8 ops)."""
     from paper_2506_10443_b200.workloads import linear_bytes
 
-    done_bytes, spent, layers = 0, 0.0, 0
-    for l in range(max_layers):
-        for lin in inputs.stack(model):
-            W = inputs.weights(inputs.seed_for(config, l, lin.matrix_id, 0), lin.N, lin.K)
-            q, s, z = oracle.quantize_w4(W, group)          # offline step, not timed
-            x = inputs.activations(inputs.seed_for(config, l, lin.matrix_id, 1), M, lin.K).astype(np.float32)
-            t = time.perf_counter()
-            oracle.linear_wa16(x, q, s, z, group)
-            spent += time.perf_counter() - t
-            done_bytes += linear_bytes(lin.N, lin.K, group, M)
-        layers += 1
-        if spent >= max_seconds:
-            break
-    return done_bytes, spent, layers, oracle.num_threads()
+    return linear_bytes(N, K, GROUP, M) if kind == "decode" else 2 * M * N * K
+
+
+def scale_of(kind):
+    return 1e9 if kind == "decode" else 1e12
+
+
+def oracle_linear(kind, x, q, s, z):
+    import oracle
+
+    if kind == "decode":
+        return oracle.linear_wa16(x, q, s, z, GROUP)
+    return oracle.linear_w4a8(x, q, s, z, GROUP)
+
+
+def oracle_prepare(wl, model, layer, frac):
+    """Oracle inputs of one layer (rows [0, frac*N) of every linear): quantised offline, untimed."""
+    import oracle
+    from paper_2506_10443_b200 import inputs
+
+    out = []
+    for lin in inputs.stack(model):
+        rows = lin.N if frac >= 1.0 else max(1, int(np.ceil(frac * lin.N)))
+        W = inputs.weights(inputs.seed_for(wl["config"], layer, lin.matrix_id, 0), lin.N, lin.K)[:rows]
+        q, s, z = oracle.quantize_w4(W, GROUP)
+        x = inputs.activations(inputs.seed_for(wl["config"], layer, lin.matrix_id, 1), wl["M"], lin.K,
+                               outliers=wl["kind"] == "prefill").astype(np.float32)
+        out.append((x, q, s, z, units_of_linear(wl["kind"], rows, lin.K, wl["M"])))
+    return out
+
+
+def oracle_sample(wl, model, seconds):
+    """A sample of the workload sized so that one oracle pass over it takes about `seconds`:
+    whole layers if they fit, else the first rows of every linear of layer 0."""
+    import oracle
+    from paper_2506_10443_b200 import inputs
+
+    layer_units = sum(units_of_linear(wl["kind"], t.N, t.K, wl["M"]) for t in inputs.stack(model))
+    cal = oracle_prepare(wl, model, 0, 0.02 if wl["kind"] == "decode" else 0.002)
+    t = time.perf_counter()
+    for x, q, s, z, _ in cal:
+        oracle_linear(wl["kind"], x, q, s, z)
+    rate = sum(c[4] for c in cal) / max(time.perf_counter() - t, 1e-6)
+    frac = rate * seconds / layer_units
+    if frac >= 1.0:
+        n_layers = min(model["layers"], int(frac))
+        sample = [p for l in range(n_layers) for p in oracle_prepare(wl, model, l, 1.0)]
+        what = "%d of %d layers (7 linears each), %d token(s)" % (n_layers, model["layers"], wl["M"])
+    else:
+        sample = oracle_prepare(wl, model, 0, frac)
+        what = "first %.2f %% of the rows of each of the 7 linears of layer 0, %d token(s)" % (100 * frac, wl["M"])
+    return sample, what, oracle.num_threads()
 
 
 def run_reference(args):
     """The reference arm: the CPU oracle as it stands, on the host cores, same metric and config.
     Each step is a bounded sample of the workload sized from a calibration pass so that the whole
     run (warm-up + steps) stays within about two minutes of oracle time."""
-    rank = int(os.environ.get("RANK", "0"))
-    if rank != 0:
+    if int(os.environ.get("RANK", "0")) != 0:
         return
-    import oracle
     from paper_2506_10443_b200 import inputs
-    from paper_2506_10443_b200.workloads import linear_bytes
 
-    model_key, config, M = WORKLOADS[args.workload]
-    model = getattr(inputs, model_key)
-    group = 64
-    linears = inputs.stack(model)
-    layer_bytes = sum(linear_bytes(t.N, t.K, group, M) for t in linears)
-
-    def prepared(layer, frac):
-        out = []
-        for lin in linears:
-            rows = lin.N if frac >= 1.0 else max(1, int(np.ceil(frac * lin.N)))
-            W = inputs.weights(inputs.seed_for(config, layer, lin.matrix_id, 0), lin.N, lin.K)[:rows]
-            q, s, z = oracle.quantize_w4(W, group)   # offline step, not timed
-            x = inputs.activations(inputs.seed_for(config, layer, lin.matrix_id, 1), M, lin.K).astype(np.float32)
-            out.append((x, q, s, z, linear_bytes(rows, lin.K, group, M)))
-        return out
-
-    # calibration: 2 % of the rows of layer 0
-    cal = prepared(0, 0.02)
-    t = time.perf_counter()
-    for x, q, s, z, _ in cal:
-        oracle.linear_wa16(x, q, s, z, group)
-    rate = sum(c[4] for c in cal) / max(time.perf_counter() - t, 1e-6)   # bytes per second
+    wl = WORKLOADS[args.workload]
+    model = getattr(inputs, wl["model"])
+    metric, unit, _ = metric_of(wl["kind"])
     budget = min(2.0, 120.0 / max(args.steps + args.warmup, 1))
-    frac = rate * budget / layer_bytes
-    if frac >= 1.0:
-        n_layers = min(model["layers"], int(frac))
-        sample = [p for l in range(n_layers) for p in prepared(l, 1.0)]
-        what = "%d of %d layers (7 linears each), %d token, per step" % (n_layers, model["layers"], M)
-    else:
-        sample = prepared(0, frac)
-        what = "first %.1f %% of the rows of each of the 7 linears of layer 0, %d token, per step" % (100 * frac, M)
-    step_bytes = sum(p[4] for p in sample)
+    sample, what, threads = oracle_sample(wl, model, budget)
+    step_units = sum(p[4] for p in sample)
 
     def step():
         for x, q, s, z, _ in sample:
-            oracle.linear_wa16(x, q, s, z, group)
+            oracle_linear(wl["kind"], x, q, s, z)
 
     for _ in range(args.warmup):
         step()
@@ -213,15 +236,15 @@ def run_reference(args):
     for _ in range(args.steps):
         step()
     total_s = time.perf_counter() - t
-    value = step_bytes * args.steps / total_s / 1e9
-    threads = oracle.num_threads()
+    value = step_units * args.steps / total_s / scale_of(wl["kind"])
+    what += ", per step"
     line = {
-        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "impl": "reference", "metric": metric, "value": value, "unit": unit, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total_s / max(args.steps, 1),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": args.workload, "sample": what, "algorithmic_bytes_per_step": step_bytes},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": what},
-        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "config": {"workload": args.workload, "sample": what, "algorithmic_units_per_step": step_units},
+        "cpu_baseline": {"value": value, "unit": unit, "cores": threads, "kind": "oracle", "sample": what},
+        "e2e": {"value": value, "unit": unit, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
     print(json.dumps(line), flush=True)
@@ -249,9 +272,15 @@ def run_ours(args):
     if not B.device_supported():
         raise SystemExit("the kernels are built for compute capability 10.x only")
 
-    model_key, config, M = WORKLOADS[args.workload]
-    model = getattr(inputs, model_key)
-    stack = LinearStack(model, config, M, 64)   # every rank: an independent replica of the workload
+    wl = WORKLOADS[args.workload]
+    kind, M = wl["kind"], wl["M"]
+    model = getattr(inputs, wl["model"])
+    metric, unit, dtype = metric_of(kind)
+    # every rank: an independent replica of the workload
+    stack = LinearStack(model, wl["config"], M, GROUP, outliers=kind == "prefill")
+    run = stack.run_w4a16 if kind == "decode" else stack.run_w4a8
+    launches = stack.launches_per_step_w4a16 if kind == "decode" else stack.launches_per_step_w4a8
+    step_units = stack.algorithmic_bytes_w4a16 if kind == "decode" else stack.ops
     stream = torch.cuda.current_stream()
 
     def barrier():
@@ -260,7 +289,7 @@ def run_ours(args):
         torch.cuda.synchronize()
 
     # one untimed pass resolves per-device state (function attributes, symbol addresses), then capture
-    stack.run_w4a16()
+    run()
     assert B.read_status() == 0
     graph = None
     if not args.no_graph:
@@ -268,14 +297,14 @@ def run_ours(args):
         cap = torch.cuda.Stream()
         cap.wait_stream(stream)
         with torch.cuda.graph(graph, stream=cap):
-            stack.run_w4a16(cap)
+            run(cap)
         torch.cuda.synchronize()
 
     def step():
         if graph is not None:
             graph.replay()
         else:
-            stack.run_w4a16()
+            run()
 
     sampler = ClockSampler(local_rank)
     sampler.start()
@@ -320,42 +349,53 @@ def run_ours(args):
 
     if rank == 0:
         peaks, peaks_kind = measured_peaks()
-        step_bytes = stack.algorithmic_bytes_w4a16
         ms_per_step = ms / args.steps
-        gbs_one = step_bytes / (ms_per_step * 1e-3) / 1e9          # one replica
-        value = gbs_one * world
-        e2e_value = step_bytes * world / (e2e_ms / e2e_steps * 1e-3) / 1e9
-        launches = stack.launches_per_step_w4a16
-        peak = float(peaks["hbm_gbs"])
+        one = step_units / (ms_per_step * 1e-3) / scale_of(kind)          # one replica
+        value = one * world
+        e2e_value = step_units * world / (e2e_ms / e2e_steps * 1e-3) / scale_of(kind)
+        if kind == "decode":
+            roof = {"bound": "hbm", "kernel": "gemv_w4a16_kernel", "achieved": one, "peak": float(peaks["hbm_gbs"]),
+                    "unit": "GB/s", "peak_source": "HBM copy rate, of " + peaks_kind}
+            l2 = "weights of one step (%.0f MB) exceed L2 (126 MB); no flush" % (stack.weight_bytes / 1e6)
+        else:
+            peak = float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])) * INT8_OVER_BF16
+            roof = {"bound": "tensor", "kernel": "gemm_w4a8_kernel", "achieved": one, "peak": peak, "unit": "TOP/s",
+                    "peak_source": "sustained cuBLAS bf16 rate x 2 (nominal int8:bf16 ratio), of " + peaks_kind,
+                    "frac_of_nominal_4500": one / 4500.0,
+                    "note": "the timed region also holds the activation-quantiser launches (HBM-bound, small)"}
+            l2 = "weights + activations of one step (%.0f MB) exceed L2 (126 MB); no flush" % (
+                (stack.weight_bytes + 2 * stack.xin.numel() + 2 * stack.yout.numel()) / 1e6)
+        roof.update({"frac": roof["achieved"] / roof["peak"], "launches_per_step": launches,
+                     "avg_launch_us": 1e3 * ms_per_step / launches,
+                     "algorithmic_units_per_launch": step_units / launches,
+                     "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(args.workload)})
         line = {
-            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "metric": metric, "value": value, "unit": unit, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "vs_baseline": None, "dtype": dtype, "data": "synthetic",
             "config": {
-                "workload": args.workload, "tokens_per_step": M, "group": 64, "layers": stack.n_layers,
-                "linears_per_layer": 7, "weight_bytes": stack.weight_bytes, "algorithmic_bytes_per_step": step_bytes,
-                "l2": "weights of one step (%.0f MB) exceed L2 (126 MB); no flush" % (stack.weight_bytes / 1e6),
-                "cuda_graph": graph is not None, "parallelism": "replicas only" if world > 1 else "single GPU",
+                "workload": args.workload, "tokens_per_step": M, "group": GROUP, "layers": stack.n_layers,
+                "linears_per_layer": 7, "weight_bytes": stack.weight_bytes, "algorithmic_units_per_step": step_units,
+                "l2": l2, "cuda_graph": graph is not None,
+                "parallelism": "replicas only" if world > 1 else "single GPU",
             },
             "tokens_per_s": M * world / (ms_per_step * 1e-3),
-            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(stack.xin_host.numel() * 2),
+            "e2e": {"value": e2e_value, "unit": unit, "h2d_bytes_per_step": int(stack.xin_host.numel() * 2),
                     "d2h_bytes_per_step": int(stack.yout_host.numel() * 2), "steps": e2e_steps,
                     "ms_per_step": e2e_ms / e2e_steps},
             "gpu_launches": launches * args.steps,
             "clocks": sampler.summary(t0, t1),
-            "roofline": {
-                "bound": "hbm", "kernel": "gemv_w4a16_kernel", "achieved": gbs_one, "peak": peak, "unit": "GB/s",
-                "frac": gbs_one / peak, "peak_source": "of " + peaks_kind,
-                "launches_per_step": launches, "avg_launch_us": 1e3 * ms_per_step / launches,
-                "algorithmic_bytes_per_launch": step_bytes / launches,
-                "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(args.workload),
-            },
+            "roofline": roof,
         }
         if world == 1 and not args.no_cpu_baseline:
-            b, s, layers, threads = oracle_stack_pass(model, config, M, 64, args.cpu_seconds, model["layers"])
+            sample, what, threads = oracle_sample(wl, model, args.cpu_seconds)
+            t = time.perf_counter()
+            for x, q, s, z, _ in sample:
+                oracle_linear(kind, x, q, s, z)
+            spent = time.perf_counter() - t
             line["cpu_baseline"] = {
-                "value": b / s / 1e9, "unit": UNIT, "cores": threads, "kind": "oracle",
-                "sample": "%d of %d layers, %d token, %.1f s of oracle time" % (layers, model["layers"], M, s),
+                "value": sum(p[4] for p in sample) / spent / scale_of(kind), "unit": unit, "cores": threads,
+                "kind": "oracle", "sample": "%s, %.1f s of oracle time" % (what, spent),
             }
         print(json.dumps(line), flush=True)
     if dist is not None:
@@ -373,10 +413,11 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=10.0, help="oracle time budget of the cpu_baseline leg")
     args = ap.parse_args()
+    decode = WORKLOADS[args.workload]["kind"] == "decode"
     if args.steps is None:
-        args.steps = 3000 if args.impl == "ours" else 5
+        args.steps = (3000 if decode else 100) if args.impl == "ours" else 5
     if args.warmup is None:
-        args.warmup = 50 if args.impl == "ours" else 3
+        args.warmup = (50 if decode else 5) if args.impl == "ours" else 3
     args.steps = max(args.steps, 1)
     args.warmup = max(args.warmup, 3)
     if args.impl == "reference":

@@ -48,7 +48,7 @@ class LinearStack:
     """
 
     def __init__(self, model: dict, config: int, M: int, group: int = 64, layers: Optional[int] = None,
-                 outliers: bool = False, device: str = "cuda"):
+                 outliers: bool = False, device: str = "cuda", weights_from: "Optional[LinearStack]" = None):
         self.model, self.config, self.M, self.group = model, config, M, group
         self.n_layers = model["layers"] if layers is None else layers
         self.linears = inputs.stack(model)
@@ -62,9 +62,12 @@ class LinearStack:
         for l in range(self.n_layers):
             L = _Layer()
             for lin in self.linears:
-                W = inputs.weights(inputs.seed_for(config, l, lin.matrix_id, 0), lin.N, lin.K)
-                L.packed[lin.name] = torch.from_numpy(B.pack_w4(W, group)).to(self.device)
-                del W
+                if weights_from is not None:   # same packed weights, other activations
+                    L.packed[lin.name] = weights_from.layers[l].packed[lin.name]
+                else:
+                    W = inputs.weights(inputs.seed_for(config, l, lin.matrix_id, 0), lin.N, lin.K)
+                    L.packed[lin.name] = torch.from_numpy(B.pack_w4(W, group)).to(self.device)
+                    del W
                 iid = _INPUT_OF[lin.name]
                 if iid not in L.x_off:
                     x = inputs.activations(inputs.seed_for(config, l, _INPUT_SEED_ID[iid], 1), M, lin.K,
@@ -83,6 +86,7 @@ class LinearStack:
         self.yout = torch.zeros(y_total, dtype=torch.float16, device=self.device)
         self.yout_host = torch.empty(y_total, dtype=torch.float16).pin_memory()
         self._launches = None
+        self._workspace = None
 
     # ---- views ----
     def x_view(self, layer: int, name: str) -> torch.Tensor:
@@ -115,3 +119,19 @@ class LinearStack:
     def run_w4a16(self, stream=None) -> None:
         for arr in self._decode_launches():
             B.linear_w4a16_batch(arr, self.M, stream)
+
+    # ---- prefill ----
+    @property
+    def launches_per_step_w4a8(self) -> int:
+        return 2 * 7 * self.n_layers   # activation quantiser + GEMM per linear
+
+    def run_w4a8(self, stream=None) -> None:
+        """One prefill step: every linear of every layer as quantise-activations + W4A8 GEMM."""
+        if self._workspace is None:
+            need = max(B.workspace_size_w4a8(self.M, t.N, t.K, self.group) for t in self.linears)
+            self._workspace = torch.empty(need, dtype=torch.uint8, device=self.device)
+        ws, nbytes = self._workspace, self._workspace.numel()
+        for l, L in enumerate(self.layers):
+            for lin in self.linears:
+                B.linear_w4a8(self.x_view(l, lin.name), L.packed[lin.name], self.y_view(l, lin.name), self.M, lin.N,
+                              lin.K, self.group, ws, nbytes, stream=stream)

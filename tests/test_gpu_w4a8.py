@@ -1,0 +1,122 @@
+"""GPU parity of the prefill W4A8 path against the CPU oracle, through the C ABI: the int32 group
+partials bit for bit, the outputs within 2e-3."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2506_10443_b200 import binding as B
+from paper_2506_10443_b200 import inputs
+from gpu_util import assert_bf16_within_1ulp, assert_close, dev, quantized
+
+pytestmark = pytest.mark.gpu
+
+
+def run_w4a8(x, packed, M, N, K, group, y_dtype=B.F16, x_dtype=B.F16):
+    tdt = {B.F16: torch.float16, B.BF16: torch.bfloat16, B.F32: torch.float32}[y_dtype]
+    nbytes = B.workspace_size_w4a8(M, N, K, group)
+    assert nbytes > 0
+    ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    y = torch.full((M, N), float("nan"), dtype=tdt, device="cuda")
+    B.linear_w4a8(x, dev(packed), y, M, N, K, group, ws, nbytes, x_dtype=x_dtype, y_dtype=y_dtype)
+    assert B.read_status() == 0
+    return y.float().cpu().numpy()
+
+
+@pytest.mark.parametrize("M,N,K,group", [
+    (1, 16, 64, 64),         # one group, one row block
+    (5, 40, 192, 64),        # K = 1.5 stages: a stage with a single group
+    (130, 200, 320, 64),     # ragged in M, N and K against the 128 x 128 x 128 tiles
+    (64, 256, 1536, 64),     # k/v projection, shortest prompt
+    (33, 130, 1024, 128),    # group 128
+    (96, 48, 8960, 64),      # the down projection's K: a partial last 512-k chunk
+    (3, 300, 3584, 128),
+])
+def test_group_partials_bit_exact(M, N, K, group):
+    W, packed, (q, s, z) = quantized(M + 3 * N + K, N, K, group)
+    x = inputs.activations(M + N + K, M, K, outliers=True)
+    G = K // group
+    P = torch.full((M, N, G), -7777, dtype=torch.int32, device="cuda")
+    a_q = torch.empty((M, K), dtype=torch.int8, device="cuda")
+    a_scale = torch.empty((M,), dtype=torch.float32, device="cuda")
+    A = torch.empty((M, G), dtype=torch.int32, device="cuda")
+    B.debug_w4a8_partials(dev(x), dev(packed), P, a_q, a_scale, A, M, N, K, group)
+    assert B.read_status() == 0
+    aq0, as0, A0 = oracle.act_quant(x.astype(np.float32), group)
+    assert (a_q.cpu().numpy() == aq0).all()
+    assert (A.cpu().numpy() == A0).all()
+    assert (a_scale.cpu().numpy().view(np.uint32) == as0.view(np.uint32)).all()
+    assert (P.cpu().numpy() == oracle.group_partials(aq0, q, group)).all()
+
+
+@pytest.mark.parametrize("M,N,K,group", [
+    (1, 16, 64, 64),
+    (5, 40, 192, 64),
+    (130, 200, 320, 64),
+    (64, 1536, 1536, 64),     # q/o projection, prompt of 64
+    (256, 256, 1536, 64),     # k/v projection, prompt of 256
+    (256, 512, 8960, 64),     # down projection rows, long K
+    (300, 1000, 448, 64),     # G = 7: the last zero-point block holds three groups
+    (77, 130, 1024, 128),
+    (512, 384, 3584, 128),
+])
+def test_w4a8_matches_oracle(M, N, K, group):
+    W, packed, (q, s, z) = quantized(2 * M + N + K, N, K, group)
+    x = inputs.activations(M + 2 * N + K, M, K, outliers=True)
+    y = run_w4a8(dev(x), packed, M, N, K, group, B.F32)
+    assert_close(y, oracle.linear_w4a8(x.astype(np.float32), q, s, z, group))
+
+
+def test_w4a8_output_and_input_dtypes():
+    M, N, K, group = 70, 272, 1536, 64
+    W, packed, (q, s, z) = quantized(11, N, K, group)
+    x = inputs.activations(12, M, K, outliers=True)
+    ref = oracle.linear_w4a8(x.astype(np.float32), q, s, z, group)
+    y32 = run_w4a8(dev(x), packed, M, N, K, group, B.F32)
+    assert_close(y32, ref, 2e-4)
+    assert_close(run_w4a8(dev(x), packed, M, N, K, group, B.F16), ref)
+    assert_bf16_within_1ulp(run_w4a8(dev(x), packed, M, N, K, group, B.BF16), y32.astype(np.float64))
+    xb = inputs.activations(13, M, K, outliers=True, dtype="bf16")
+    yb = run_w4a8(dev(inputs.bf16_bits(xb)).view(torch.bfloat16), packed, M, N, K, group, B.F32, x_dtype=B.BF16)
+    assert_close(yb, oracle.linear_w4a8(xb, q, s, z, group))
+
+
+def test_w4a8_unusual_zero_points():
+    # groups that do not straddle zero (negative and large zero points), a constant group and an
+    # all-zero token: the zero-point term must stay exact
+    rng = np.random.default_rng(5)
+    M, N, K, group = 40, 64, 512, 64
+    W = rng.normal(0, 0.02, (N, K)).astype(np.float32)
+    W[:16] += 0.3
+    W[16:32] -= 0.25
+    W[32, :64] = 0.125
+    x = inputs.activations(21, M, K, outliers=True)
+    x[7] = 0
+    packed = B.pack_w4(W, group)
+    q, s, z = oracle.quantize_w4(W, group)
+    y = run_w4a8(dev(x), packed, M, N, K, group, B.F32)
+    assert_close(y, oracle.linear_w4a8(x.astype(np.float32), q, s, z, group))
+    assert (y[7] == 0).all()
+
+
+def test_w4a8_deterministic():
+    M, N, K, group = 200, 640, 1536, 64
+    W, packed, _ = quantized(31, N, K, group)
+    xd = dev(inputs.activations(32, M, K, outliers=True))
+    a = run_w4a8(xd, packed, M, N, K, group)
+    b = run_w4a8(xd, packed, M, N, K, group)
+    assert (a == b).all()
+
+
+def test_w4a8_argument_errors_on_gpu():
+    t = torch.empty(1 << 16, dtype=torch.uint8, device="cuda")
+    p = t.data_ptr()
+    need = B.workspace_size_w4a8(4, 16, 64, 64)
+    assert need > 0 and B.workspace_size_w4a8(4, 16, 96, 64) == 0
+    f = B.lib.mnnllm_linear_w4a8
+    assert f(p, p, p, 4, 16, 64, 64, B.F16, B.F16, p, need - 1, None) == 6       # workspace too small
+    assert f(p, p, p, 4, 16, 64, 64, B.F16, B.F16, None, need, None) == 6
+    assert f(p, p, p, 4, 16, 64, 64, B.F16, B.F16, p + 16, need, None) == 3      # workspace alignment
+    assert f(p, p, p, 4, 16, 64, 32, B.F16, B.F16, p, need, None) == 2
+    assert f(p, p, p, 4, 16, 64, 64, B.F32, B.F16, p, need, None) == 2
+    assert f(None, p, p, 4, 16, 64, 64, B.F16, B.F16, p, need, None) == 1
