@@ -5,17 +5,25 @@
 //
 // One CTA computes a tile of 128 weight rows x 128 tokens.  The weights are the M side of the MMA,
 // so that a tensor-memory lane is one output channel n and its per-group scale is a per-thread
-// scalar in the drain.  Warp roles (14 warps):
-//   warp 0      producer: TMA loads of the int8 activation tile (128 tokens x 128 k, 128B swizzle)
-//               and of the fp16 group-sum quadruples that feed the zero-point MMA
-//   warp 1      allocates tensor memory, issues tcgen05.mma (kind::i8 into one of two int32
+// scalar in the drain.  Warp roles (15 warps):
+//   warp 0      producer: TMA loads of the packed int4 codes (the packed buffer seen as a 2-D tensor
+//               [row block][bytes]: one box of 8 row blocks x 1 KiB per stage; issuing one small bulk
+//               copy per row block instead costs ~75 cycles each and starves the pipeline) and of
+//               each 512-k chunk's (scale, zero) tables into shared-memory rings; TMA loads of the
+//               int8 activation tile (128 tokens x 128 k, 128B swizzle) and of the fp16 group-sum
+//               quadruples that feed the zero-point MMA
+//   warp 1      allocates tensor memory, issues tcgen05.mma (kind::i8 into one of three int32
 //               accumulators per group; kind::f16 for the zero-point term) and the commits
-//   warps 2-5   unpack: packed int4 codes (global, coalesced 16-byte loads, register prefetch three
-//               stages ahead) -> int8 K-major tile in the 128B-swizzled layout the MMA reads; the
-//               row's fp32 scale for the drain; (s z) split into fp16 hi + lo for the zero-point MMA
+//   warps 2-5   unpack: packed int4 codes (shared-memory ring) -> int8 K-major tile in the
+//               128B-swizzled layout the MMA reads
+//   warp 14     scales: each (row, group) pair of the stage: the fp32 scale for the drain; (s z)
+//               split into fp16 hi + lo for the zero-point MMA (a separate warp, because these
+//               conversion chains would otherwise sit on the unpack warps' critical path)
 //   warps 6-13  drain: every group's 128 x 128 int32 partial tile leaves tensor memory
-//               (tcgen05.ld), is converted and accumulated as acc += s * P in registers while the
-//               MMA fills the other accumulator; epilogue applies the zero-point term and a_scale.
+//               (tcgen05.ld), is converted (integer add of a float bit pattern + float subtract: the
+//               cvt instruction runs at 16 lanes per clock per SM and would bound the kernel) and
+//               accumulated as acc += s * P in registers while the
+//               MMA fills the other accumulators; epilogue applies the zero-point term and a_scale.
 // The zero-point term is a rank-G product, evaluated on the tensor cores without loss:
 //   (s z) = hi + lo (fp16 each; s and z are fp16, so the product has 22 significant bits),
 //   A     = 64 h + l (both exact in fp16), four fp16 products per group, fp32 accumulation in a
@@ -40,25 +48,32 @@ constexpr int kTileN = 128;   // weight rows per CTA tile (MMA M)
 constexpr int kTileT = 128;   // tokens per CTA tile (MMA N)
 constexpr int kStageK = 128;  // k per pipeline stage (one 128-byte swizzle row of int8)
 constexpr int kStages = 4;
-constexpr int kScaleSlots = 2 * kStages + 2;  // groups whose scales may be live at once
-constexpr int kPrefetch = 3;                  // stages of packed codes held in registers ahead of use
-constexpr int kThreads = 14 * 32;
-constexpr int kUnpackWarp0 = 2, kDrainWarp0 = 6;
+constexpr int kScaleSlots = 2 * kStages + 4;  // groups whose scales may be live at once (ring + accumulators + 1)
+constexpr int kPkStages = 6;                  // ring of packed-code stages (8 KiB each)
+constexpr int kPkLead = 2;                    // stages the packed ring is produced ahead of the activations
+constexpr int kTabSlots = 3;                  // ring of per-chunk (scale, zero) tables (8 row blocks x 512 B)
+constexpr int kThreads = 15 * 32;
+constexpr int kUnpackWarp0 = 2, kDrainWarp0 = 6, kScaleWarp = 14;
 constexpr uint32_t kMaxPolls = 1u << 22;
-constexpr uint32_t kTmemCols = 512;           // 2 x 128 int32 accumulators + 128 fp32 zero-point term
-constexpr uint32_t kColCorr = 256;
+constexpr int kAcc = 3;                       // int32 group accumulators in tensor memory (128 columns each)
+constexpr uint32_t kTmemCols = 512;           // 3 x 128 int32 accumulators + 128 fp32 zero-point term
+constexpr uint32_t kColCorr = kAcc * 128;
 
 constexpr int kStageBytes = kTileN * kStageK;  // 16 KiB, int8
 constexpr int kCorrBytes = 128 * 32;           // 128 rows x 16 fp16
+constexpr int kPkBytes = 8 * 2 * kSlabBytes;   // packed codes of a stage: 8 row blocks x 2 slabs
+constexpr int kTabBytes = 8 * 512;             // (scale, zero) tables of a chunk: 8 row blocks x 16 rows x 8 pairs
 
 struct Smem {
     static constexpr int wq = 0;
     static constexpr int aq = wq + kStages * kStageBytes;
     static constexpr int ca = aq + kStages * kStageBytes;
     static constexpr int cb = ca + 2 * kCorrBytes;
-    static constexpr int scale = cb + 2 * kCorrBytes;
+    static constexpr int pk = cb + 2 * kCorrBytes;
+    static constexpr int tab = pk + kPkStages * kPkBytes;
+    static constexpr int scale = tab + kTabSlots * kTabBytes;
     static constexpr int bars = scale + kScaleSlots * kTileN * 4;
-    static constexpr int n_bars = 2 * kStages + 2 + 2 + 2 + 2 + 1;
+    static constexpr int n_bars = 2 * kStages + 2 * kAcc + 2 + 2 + 1 + 2 * kPkStages + 2 * kTabSlots;
     static constexpr int misc = bars + n_bars * 8;
     static constexpr int total = misc + 16;
 };
@@ -97,6 +112,7 @@ __device__ __forceinline__ void store_y(void* y, int dtype, size_t idx, float v)
 template <int GROUP, bool PARTIALS>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ CUtensorMap tm_ac,
+                 const __grid_constant__ CUtensorMap tm_pk, const __grid_constant__ CUtensorMap tm_tab,
                  const __grid_constant__ Params p, uint32_t* __restrict__ status) {
     constexpr int GPS = kStageK / GROUP;  // groups per stage (2 or 1)
     constexpr int SPB = 4 / GPS;          // stages per block of four groups (zero-point MMA cadence)
@@ -106,10 +122,14 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
     uint64_t* ab_full = bars;
     uint64_t* ab_empty = ab_full + kStages;
     uint64_t* tm_full = ab_empty + kStages;
-    uint64_t* tm_empty = tm_full + 2;
-    uint64_t* c_full = tm_empty + 2;
+    uint64_t* tm_empty = tm_full + kAcc;
+    uint64_t* c_full = tm_empty + kAcc;
     uint64_t* c_empty = c_full + 2;
     uint64_t* corr_done = c_empty + 2;
+    uint64_t* pk_full = corr_done + 1;
+    uint64_t* pk_empty = pk_full + kPkStages;
+    uint64_t* tab_full = pk_empty + kPkStages;
+    uint64_t* tab_empty = tab_full + kTabSlots;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + Smem::misc);
     volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + Smem::misc + 4);
     float* scale_ring = reinterpret_cast<float*>(smem + Smem::scale);
@@ -119,15 +139,17 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
     const int n_stages = p.n_stages, G = p.G;
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < kStages; ++i) { mbar_init(&ab_full[i], 5); mbar_init(&ab_empty[i], 1); }
-        for (int i = 0; i < 2; ++i) {
-            mbar_init(&tm_full[i], 1); mbar_init(&tm_empty[i], 8);
-            mbar_init(&c_full[i], 5); mbar_init(&c_empty[i], 1);
-        }
+        for (int i = 0; i < kStages; ++i) { mbar_init(&ab_full[i], 6); mbar_init(&ab_empty[i], 1); }
+        for (int i = 0; i < kAcc; ++i) { mbar_init(&tm_full[i], 1); mbar_init(&tm_empty[i], 8); }
+        for (int i = 0; i < 2; ++i) { mbar_init(&c_full[i], 2); mbar_init(&c_empty[i], 1); }
         mbar_init(corr_done, 1);
+        for (int i = 0; i < kPkStages; ++i) { mbar_init(&pk_full[i], 1); mbar_init(&pk_empty[i], 4); }
+        for (int i = 0; i < kTabSlots; ++i) { mbar_init(&tab_full[i], 1); mbar_init(&tab_empty[i], 1); }
         *abort_flag = 0;
         fence_mbar_init();
         prefetch_tensormap(&tm_act);
+        prefetch_tensormap(&tm_pk);
+        prefetch_tensormap(&tm_tab);
         if (!PARTIALS) prefetch_tensormap(&tm_ac);
     }
     if (warp == 1) {
@@ -151,19 +173,45 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
 
     if (warp == 0) {
         // ------------------------------------------------------------------ producer (TMA)
-        for (int st = 0; st < n_stages && !*abort_flag; ++st) {
-            const int slot = st % kStages, round = st / kStages;
-            if (!wait(&ab_empty[slot], (round & 1) ^ 1, 1)) break;
-            if (lane == 0) {
-                mbar_arrive_expect_tx(&ab_full[slot], kTileT * kStageK);
-                tma_load_2d(smem + Smem::aq + slot * kStageBytes, &tm_act, st * kStageK, m0, &ab_full[slot]);
+        const int rb0 = n0 / kRowsPerBlock;
+        for (int i = 0; i < n_stages + kPkLead && !*abort_flag; ++i) {
+            if (i < n_stages) {
+                // packed codes of stage i (and, at the start of a 512-k chunk, its scale/zero tables)
+                const int pslot = i % kPkStages, j = i >> 2;
+                if (!wait(&pk_empty[pslot], ((i / kPkStages) & 1) ^ 1, 10)) break;
+                const int ns_chunk = (p.n_slabs - 8 * j) < 8 ? (p.n_slabs - 8 * j) : 8;
+                const unsigned long long chunk_off = (unsigned long long)j * p.chunk_bytes;
+                // boxes are counted in full even where they run past the tensor (zero fill)
+                if ((i & 3) == 0) {
+                    const int tslot = j % kTabSlots;
+                    if (!wait(&tab_empty[tslot], ((j / kTabSlots) & 1) ^ 1, 12)) break;
+                    if (elect_one()) {
+                        mbar_arrive_expect_tx(&tab_full[tslot], kTabBytes);
+                        tma_load_2d(smem + Smem::tab + tslot * kTabBytes, &tm_tab,
+                                    (int)((chunk_off + (unsigned long long)ns_chunk * kSlabBytes) >> 2), rb0, &tab_full[tslot]);
+                    }
+                }
+                if (elect_one()) {
+                    mbar_arrive_expect_tx(&pk_full[pslot], kPkBytes);
+                    tma_load_2d(smem + Smem::pk + pslot * kPkBytes, &tm_pk,
+                                (int)((chunk_off + (unsigned long long)(i & 3) * 2 * kSlabBytes) >> 2), rb0, &pk_full[pslot]);
+                }
             }
-            if (!PARTIALS && st % SPB == 0) {
-                const int cblk = st / SPB, cslot = cblk & 1;
-                if (!wait(&c_empty[cslot], ((cblk >> 1) & 1) ^ 1, 2)) break;
-                if (lane == 0) {
-                    mbar_arrive_expect_tx(&c_full[cslot], kTileT * 32);
-                    tma_load_2d(smem + Smem::cb + cslot * kCorrBytes, &tm_ac, cblk * 16, m0, &c_full[cslot]);
+            const int st = i - kPkLead;
+            if (st >= 0) {
+                const int slot = st % kStages, round = st / kStages;
+                if (!wait(&ab_empty[slot], (round & 1) ^ 1, 1)) break;
+                if (elect_one()) {
+                    mbar_arrive_expect_tx(&ab_full[slot], kTileT * kStageK);
+                    tma_load_2d(smem + Smem::aq + slot * kStageBytes, &tm_act, st * kStageK, m0, &ab_full[slot]);
+                }
+                if (!PARTIALS && st % SPB == 0) {
+                    const int cblk = st / SPB, cslot = cblk & 1;
+                    if (!wait(&c_empty[cslot], ((cblk >> 1) & 1) ^ 1, 2)) break;
+                    if (elect_one()) {
+                        mbar_arrive_expect_tx(&c_full[cslot], kTileT * 32);
+                        tma_load_2d(smem + Smem::cb + cslot * kCorrBytes, &tm_ac, cblk * 16, m0, &c_full[cslot]);
+                    }
                 }
             }
             __syncwarp();
@@ -179,10 +227,10 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
             tc_fence_after_sync();
             const int ngr = (G - st * GPS) < GPS ? (G - st * GPS) : GPS;
             for (int gi = 0; gi < ngr; ++gi) {
-                const int b = gcount & 1;
-                if (!wait(&tm_empty[b], ((gcount >> 1) & 1) ^ 1, 4)) { ok = false; break; }
+                const int b = gcount % kAcc;
+                if (!wait(&tm_empty[b], ((gcount / kAcc) & 1) ^ 1, 4)) { ok = false; break; }
                 tc_fence_after_sync();
-                if (lane == 0) {
+                if (elect_one()) {
                     const uint64_t da = desc_sw128(wq_addr + slot * kStageBytes);
                     const uint64_t db = desc_sw128(aq_addr + slot * kStageBytes);
 #pragma unroll
@@ -196,12 +244,12 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
                 ++gcount;
             }
             if (!ok) break;
-            if (lane == 0) mma_commit(&ab_empty[slot]);
+            if (elect_one()) mma_commit(&ab_empty[slot]);
             if (!PARTIALS && ((gcount & 3) == 0 || st == n_stages - 1)) {
                 const int cslot = ccount & 1;
                 if (!wait(&c_full[cslot], (ccount >> 1) & 1, 5)) break;
                 tc_fence_after_sync();
-                if (lane == 0) {
+                if (elect_one()) {
                     mma_f16_ss(tmem_base + kColCorr, desc_sw32(smem_u32(smem + Smem::ca + cslot * kCorrBytes)),
                                desc_sw32(smem_u32(smem + Smem::cb + cslot * kCorrBytes)), kIdescF16, ccount > 0);
                     mma_commit(&c_empty[cslot]);
@@ -210,90 +258,31 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
             }
             __syncwarp();
         }
-        if (!PARTIALS && lane == 0) mma_commit(corr_done);
+        if (!PARTIALS && elect_one()) mma_commit(corr_done);
         __syncwarp();
     } else if (warp < kDrainWarp0) {
         // ------------------------------------------------------------------ unpack
-        const int u = threadIdx.x - kUnpackWarp0 * 32;  // 0..127 = row of the tile this thread owns for scales
-        const int wu = u >> 5;
-        const int rb0 = n0 / kRowsPerBlock;
-        const uint8_t* body = p.packed + kHeaderBytes;
-        auto load_codes = [&](int st, uint4 (&e)[4]) {
-            const int j = st >> 2;
-            const int ns_chunk = (p.n_slabs - 8 * j) < 8 ? (p.n_slabs - 8 * j) : 8;
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int sidx = i * 4 + wu;
-                const int rb = rb0 + (sidx >> 1), sl = (st & 3) * 2 + (sidx & 1);
-                e[i] = make_uint4(0, 0, 0, 0);
-                if (st < n_stages && rb < p.n_row_blocks && sl < ns_chunk)
-                    e[i] = __ldg(reinterpret_cast<const uint4*>(body + (size_t)rb * p.row_block_bytes +
-                                                                (size_t)j * p.chunk_bytes + (size_t)sl * kSlabBytes) + lane);
-            }
-        };
-        auto load_sz = [&](int st, uint32_t (&sz)[GPS]) {
-            const int j = st >> 2;
-            const int ns_chunk = (p.n_slabs - 8 * j) < 8 ? (p.n_slabs - 8 * j) : 8;
-            const int ng = ns_chunk * kSlabK4 / GROUP;
-            const int rb = rb0 + (u >> 4), r16 = u & 15;
-#pragma unroll
-            for (int gi = 0; gi < GPS; ++gi) {
-                const int gc = (st & 3) * GPS + gi;
-                sz[gi] = 0;
-                if (st < n_stages && rb < p.n_row_blocks && gc < ng)
-                    sz[gi] = __ldg(reinterpret_cast<const uint32_t*>(body + (size_t)rb * p.row_block_bytes +
-                                                                     (size_t)j * p.chunk_bytes +
-                                                                     (size_t)ns_chunk * kSlabBytes) + r16 * ng + gc);
-            }
-        };
-        uint4 e0[4], e1[4], e2[4];
-        uint32_t z0[GPS], z1[GPS], z2[GPS];
-        load_codes(0, e0); load_sz(0, z0);
-        load_codes(1, e1); load_sz(1, z1);
-        load_codes(2, e2); load_sz(2, z2);
-        static_assert(kPrefetch == 3, "the register ring below holds three stages");
-        bool ok = true;
-        for (int st = 0; st < n_stages && ok && !*abort_flag; ++st) {
+        const int wu = warp - kUnpackWarp0;
+        const int nrb = (p.n_row_blocks - n0 / kRowsPerBlock) < 8 ? (p.n_row_blocks - n0 / kRowsPerBlock) : 8;
+        for (int st = 0; st < n_stages && !*abort_flag; ++st) {
             const int slot = st % kStages, round = st / kStages;
+            const int pslot = st % kPkStages, j = st >> 2;
+            const int ns_chunk = (p.n_slabs - 8 * j) < 8 ? (p.n_slabs - 8 * j) : 8;
+            if (!wait(&pk_full[pslot], (st / kPkStages) & 1, 11)) break;
+            // this thread's four 16-byte entries of the stage (zero where the tile or K runs out)
             uint4 cur[4];
-            uint32_t zc[GPS];
+            {
+                const uint4* pk = reinterpret_cast<const uint4*>(smem + Smem::pk + pslot * kPkBytes);
 #pragma unroll
-            for (int i = 0; i < 4; ++i) { cur[i] = e0[i]; e0[i] = e1[i]; e1[i] = e2[i]; }
-#pragma unroll
-            for (int i = 0; i < GPS; ++i) { zc[i] = z0[i]; z0[i] = z1[i]; z1[i] = z2[i]; }
-            load_codes(st + kPrefetch, e2);
-            load_sz(st + kPrefetch, z2);
-            if (!wait(&ab_empty[slot], (round & 1) ^ 1, 6)) break;
-
-            // scales for the drain, (s z) halves for the zero-point MMA: this thread's row u
-#pragma unroll
-            for (int gi = 0; gi < GPS; ++gi) {
-                const int g = st * GPS + gi;
-                if (g >= G) break;
-                const __half2 h2 = *reinterpret_cast<const __half2*>(&zc[gi]);
-                const float s = __low2float(h2), z = __high2float(h2);
-                scale_ring[(g % kScaleSlots) * kTileN + u] = s;
-                if (!PARTIALS) {
-                    const int pos = g & 3, cblk = g >> 2, cslot = cblk & 1;
-                    if (pos == 0 && !wait(&c_empty[cslot], ((cblk >> 1) & 1) ^ 1, 7)) { ok = false; break; }
-                    const float szf = s * z;  // exact: 11-bit x 11-bit significands
-                    const __half hi = __float2half_rn(szf);
-                    const __half lo = __float2half_rn(szf - __half2float(hi));
-                    const uint32_t hh = (uint32_t)__half_as_ushort(hi) * 0x00010001u;
-                    const uint32_t ll = (uint32_t)__half_as_ushort(lo) * 0x00010001u;
-                    uint8_t* tile = smem + Smem::ca + cslot * kCorrBytes;
-                    const int rowoff = (u >> 3) * 256 + (u & 7) * 32, sw = (u & 7) >> 2;
-                    *reinterpret_cast<uint2*>(tile + rowoff + (((pos >> 1) ^ sw) << 4) + (pos & 1) * 8) = make_uint2(hh, ll);
-                    if (pos == 3 || g == G - 1) {
-                        for (int q = pos + 1; q < 4; ++q)
-                            *reinterpret_cast<uint2*>(tile + rowoff + (((q >> 1) ^ sw) << 4) + (q & 1) * 8) = make_uint2(0u, 0u);
-                        fence_proxy_async_smem();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(&c_full[cslot]);
-                    }
+                for (int i = 0; i < 4; ++i) {
+                    const int sidx = i * 4 + wu;
+                    const bool valid = (sidx >> 1) < nrb && (st & 3) * 2 + (sidx & 1) < ns_chunk;
+                    cur[i] = valid ? pk[sidx * 32 + lane] : make_uint4(0, 0, 0, 0);
                 }
             }
-            if (!ok) break;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&pk_empty[pslot]);
+            if (!wait(&ab_empty[slot], (round & 1) ^ 1, 6)) break;
 
             // codes -> int8, 128B-swizzled K-major rows
             uint8_t* wq = smem + Smem::wq + slot * kStageBytes;
@@ -313,6 +302,69 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
             __syncwarp();
             if (lane == 0) mbar_arrive(&ab_full[slot]);
         }
+    } else if (warp == kScaleWarp) {
+        // ------------------------------------------------------------------ scales and (s z) halves
+        const int nrb = (p.n_row_blocks - n0 / kRowsPerBlock) < 8 ? (p.n_row_blocks - n0 / kRowsPerBlock) : 8;
+        bool ok = true;
+        for (int st = 0; st < n_stages && ok && !*abort_flag; ++st) {
+            const int slot = st % kStages, round = st / kStages;
+            const int j = st >> 2, tslot = j % kTabSlots;
+            const int ns_chunk = (p.n_slabs - 8 * j) < 8 ? (p.n_slabs - 8 * j) : 8;
+            const int ng = ns_chunk * kSlabK4 / GROUP;
+            if ((st & 3) == 0 && !wait(&tab_full[tslot], (j / kTabSlots) & 1, 13)) break;
+            // this lane's rows: lane, lane + 32, lane + 64, lane + 96
+            uint32_t zc[4][GPS];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int row = lane + 32 * i;
+                const uint32_t* tab = reinterpret_cast<const uint32_t*>(smem + Smem::tab + tslot * kTabBytes + (row >> 4) * 512);
+#pragma unroll
+                for (int gi = 0; gi < GPS; ++gi) {
+                    const int gc = (st & 3) * GPS + gi;
+                    zc[i][gi] = ((row >> 4) < nrb && gc < ng) ? tab[(row & 15) * ng + gc] : 0u;
+                }
+            }
+            if ((st & 3) == 3 || st == n_stages - 1) {  // the chunk's table has been read in full
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&tab_empty[tslot]);
+            }
+            if (!wait(&ab_empty[slot], (round & 1) ^ 1, 14)) break;
+#pragma unroll
+            for (int gi = 0; gi < GPS; ++gi) {
+                const int g = st * GPS + gi;
+                if (g >= G) break;
+                const int pos = g & 3, cblk = g >> 2, cslot = cblk & 1;
+                if (!PARTIALS && pos == 0 && !wait(&c_empty[cslot], ((cblk >> 1) & 1) ^ 1, 7)) { ok = false; break; }
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int row = lane + 32 * i;
+                    const __half2 h2 = *reinterpret_cast<const __half2*>(&zc[i][gi]);
+                    const float s = __low2float(h2), z = __high2float(h2);
+                    scale_ring[(g % kScaleSlots) * kTileN + row] = s;
+                    if (!PARTIALS) {
+                        const float szf = s * z;  // exact: 11-bit x 11-bit significands
+                        const __half hi = __float2half_rn(szf);
+                        const __half lo = __float2half_rn(szf - __half2float(hi));
+                        const uint32_t hh = (uint32_t)__half_as_ushort(hi) * 0x00010001u;
+                        const uint32_t ll = (uint32_t)__half_as_ushort(lo) * 0x00010001u;
+                        uint8_t* tile = smem + Smem::ca + cslot * kCorrBytes;
+                        const int rowoff = (row >> 3) * 256 + (row & 7) * 32, sw = (row & 7) >> 2;
+                        *reinterpret_cast<uint2*>(tile + rowoff + (((pos >> 1) ^ sw) << 4) + (pos & 1) * 8) = make_uint2(hh, ll);
+                        if (g == G - 1)
+                            for (int q = pos + 1; q < 4; ++q)
+                                *reinterpret_cast<uint2*>(tile + rowoff + (((q >> 1) ^ sw) << 4) + (q & 1) * 8) = make_uint2(0u, 0u);
+                    }
+                }
+                if (!PARTIALS && (pos == 3 || g == G - 1)) {
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&c_full[cslot]);
+                }
+            }
+            if (!ok) break;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&ab_full[slot]);
+        }
     } else {
         // ------------------------------------------------------------------ drain + epilogue
         const int q4 = warp & 3;                      // tensor-memory lane quarter this warp may read
@@ -324,8 +376,8 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
         for (int i = 0; i < 64; ++i) acc[i] = 0.f;
         bool ok = true;
         for (int g = 0; g < G && !*abort_flag; ++g) {
-            const int b = g & 1;
-            if (!wait(&tm_full[b], (g >> 1) & 1, 8)) { ok = false; break; }
+            const int b = g % kAcc;
+            if (!wait(&tm_full[b], (g / kAcc) & 1, 8)) { ok = false; break; }
             tc_fence_after_sync();
             const float sf = scale_ring[(g % kScaleSlots) * kTileN + nl];
 #pragma unroll
@@ -341,8 +393,13 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
                             if (m < p.M) p.P[((size_t)m * p.N + n) * G + g] = (int32_t)v[j];
                         }
                 } else {
+                    // int32 -> fp32 without the conversion instruction (16 lanes per clock per SM, it
+                    // would bound the kernel): |P| < 2^22, so adding the bit pattern of 1.5 * 2^23
+                    // (ulp 1) as an integer and subtracting the same constant as a float is exact
+                    // (packed f32x2 arithmetic was measured slower here: 950 vs 520 cycles per group)
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) acc[cc * 32 + j] = fmaf(sf, (float)(int32_t)v[j], acc[cc * 32 + j]);
+                    for (int j = 0; j < 32; ++j)
+                        acc[cc * 32 + j] = fmaf(sf, __uint_as_float(v[j] + 0x4B400000u) - 12582912.0f, acc[cc * 32 + j]);
                 }
             }
             tc_fence_before_sync();
@@ -395,8 +452,8 @@ EncodeTiledFn encode_fn() {
 }
 
 template <int GROUP, bool PARTIALS>
-cudaError_t launch(const CUtensorMap& tm_act, const CUtensorMap& tm_ac, const Params& p, dim3 grid, uint32_t* status,
-                   cudaStream_t stream) {
+cudaError_t launch(const CUtensorMap& tm_act, const CUtensorMap& tm_ac, const CUtensorMap& tm_pk,
+                   const CUtensorMap& tm_tab, const Params& p, dim3 grid, uint32_t* status, cudaStream_t stream) {
     static bool configured = false;
     auto kern = gemm_w4a8_kernel<GROUP, PARTIALS>;
     if (!configured) {
@@ -404,7 +461,7 @@ cudaError_t launch(const CUtensorMap& tm_act, const CUtensorMap& tm_ac, const Pa
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    kern<<<grid, kThreads, kSmemBytes, stream>>>(tm_act, tm_ac, p, status);
+    kern<<<grid, kThreads, kSmemBytes, stream>>>(tm_act, tm_ac, tm_pk, tm_tab, p, status);
     return cudaGetLastError();
 }
 
@@ -416,7 +473,21 @@ cudaError_t gemm_w4a8_launch(const GemmW4A8Args& a, uint32_t* status, cudaStream
     const W4Geometry geo = w4_geometry(a.N, a.K, a.group);
     const bool partials = a.P != nullptr;
 
-    CUtensorMap tm_act, tm_ac;
+    CUtensorMap tm_act, tm_ac, tm_pk, tm_tab;
+    {   // the packed body as [row block][32-bit words]: codes box 8 x 1 KiB, table box 8 x 512 B
+        const cuuint64_t dims[2] = {(cuuint64_t)(geo.row_block_bytes / 4), (cuuint64_t)geo.n_row_blocks};
+        const cuuint64_t strides[1] = {(cuuint64_t)geo.row_block_bytes};
+        const cuuint32_t box_pk[2] = {2 * kSlabBytes / 4, 8}, box_tab[2] = {512 / 4, 8};
+        const cuuint32_t estr[2] = {1, 1};
+        void* body = (void*)((const uint8_t*)a.packed + kHeaderBytes);
+        if (enc(&tm_pk, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, body, dims, strides, box_pk, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS ||
+            enc(&tm_tab, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, body, dims, strides, box_tab, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return cudaErrorInvalidValue;
+    }
     {
         const cuuint64_t dims[2] = {(cuuint64_t)a.K, (cuuint64_t)a.M};
         const cuuint64_t strides[1] = {(cuuint64_t)a.K};
@@ -453,10 +524,10 @@ cudaError_t gemm_w4a8_launch(const GemmW4A8Args& a, uint32_t* status, cudaStream
     p.row_block_bytes = geo.row_block_bytes; p.chunk_bytes = geo.chunk_bytes;
     const dim3 grid((unsigned)((a.N + kTileN - 1) / kTileN), (unsigned)((a.M + kTileT - 1) / kTileT));
     if (a.group == 64)
-        return partials ? launch<64, true>(tm_act, tm_ac, p, grid, status, stream)
-                        : launch<64, false>(tm_act, tm_ac, p, grid, status, stream);
-    return partials ? launch<128, true>(tm_act, tm_ac, p, grid, status, stream)
-                    : launch<128, false>(tm_act, tm_ac, p, grid, status, stream);
+        return partials ? launch<64, true>(tm_act, tm_ac, tm_pk, tm_tab, p, grid, status, stream)
+                        : launch<64, false>(tm_act, tm_ac, tm_pk, tm_tab, p, grid, status, stream);
+    return partials ? launch<128, true>(tm_act, tm_ac, tm_pk, tm_tab, p, grid, status, stream)
+                    : launch<128, false>(tm_act, tm_ac, tm_pk, tm_tab, p, grid, status, stream);
 }
 
 }  // namespace mnnllm

@@ -123,6 +123,16 @@ __device__ __forceinline__ void mma_m16n8k16_f16(float (&d)[4], uint32_t a0, uin
 }
 
 
+// One lane of a converged warp, chosen by the hardware.  Code that issues TMA or tcgen05
+// instructions from a single thread should branch on this rather than on `lane == 0`: the compiler
+// then knows the region runs with one active lane and keeps descriptors in uniform registers
+// (measured: 207 cycles per tcgen05.mma issued under `lane == 0`, 64-128 under elect.sync).
+__device__ __forceinline__ bool elect_one() {
+    uint32_t r;
+    asm volatile("{\n\t.reg .pred P;\n\telect.sync _|P, 0xffffffff;\n\tselp.u32 %0, 1, 0, P;\n\t}" : "=r"(r));
+    return r != 0;
+}
+
 // ---- named barrier among a subset of the CTA's warps -------------------------------------------
 __device__ __forceinline__ void bar_sync(uint32_t id, uint32_t threads) {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
