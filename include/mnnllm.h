@@ -142,6 +142,31 @@ size_t mnnllm_workspace_size_w4a8(int M, int N, int K, int group);
 int mnnllm_linear_w4a8(const void* x, const void* packed, void* y, int M, int N, int K, int group,
                        int x_dtype, int y_dtype, void* workspace, size_t workspace_bytes, void* stream);
 
+/* Same computation as mnnllm_linear_w4a8 for callers that cannot allocate device memory.  (The paper
+ * has no counterpart; this is a convenience of this library.)  Some users of this code run where
+ * cudaMalloc is off limits: inside a plugin whose host application owns every allocation, in a
+ * latency-critical serving loop that forbids allocator calls after start-up, or in a process whose
+ * memory pool was sized and handed out before the library was loaded.  Such callers have nowhere
+ * to get the workspace from, so this entry point brings its own: a fixed array of
+ * MNNLLM_STATIC_SCRATCH_BYTES that is part of the library's device image.  Every GPU on which the
+ * library is loaded holds that array until the process exits.
+ *
+ *   - x, packed, y and the other arguments are exactly those of mnnllm_linear_w4a8; the caller
+ *     still owns inputs and outputs.  The call itself allocates and frees nothing.
+ *   - Limit: the activations' int8 copy (M*K bytes), their scales (4*M) and the fp16 group sums
+ *     (8 * M * ceil(K/group/4)*4), each rounded up to 256 bytes, must fit the array; a larger
+ *     problem returns MNNLLM_ERR_WORKSPACE and nothing is launched.  8 MiB covers, for example,
+ *     M = 1024 tokens at K = 3584 or M = 512 at K = 8960.
+ *   - The first call on each device looks up the array's device address (one runtime query, the
+ *     device must be current); make that first call before starting any stream capture.
+ *   - All calls on a device share the one array and it keeps whatever the last call left there.
+ *     Nothing in it has to start at zero (each call rewrites all it reads), but two calls that can
+ *     overlap on the GPU - different streams without an ordering between them - race on it and
+ *     corrupt each other's results.  Calls on one stream are safe. */
+#define MNNLLM_STATIC_SCRATCH_BYTES (8u << 20)
+int mnnllm_linear_w4a8_static(const void* x, const void* packed, void* y, int M, int N, int K, int group,
+                              int x_dtype, int y_dtype, void* stream);
+
 /* The activation quantiser alone (first kernel of the W4A8 path), writing caller-owned outputs:
  * a_q int8 [M, K], a_scale fp32 [M], A int32 [M, G]. */
 int mnnllm_quantize_activations(const void* x, int x_dtype, int M, int K, int group, int8_t* a_q,

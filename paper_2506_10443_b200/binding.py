@@ -65,6 +65,8 @@ _sig("mnnllm_linear_w8a16", _c.c_int, [_P, _P, _P, _c.c_int, _c.c_int, _c.c_int,
 _sig("mnnllm_workspace_size_w4a8", _c.c_size_t, [_c.c_int, _c.c_int, _c.c_int, _c.c_int])
 _sig("mnnllm_linear_w4a8", _c.c_int,
      [_P, _P, _P, _c.c_int, _c.c_int, _c.c_int, _c.c_int, _c.c_int, _c.c_int, _P, _c.c_size_t, _P])
+_sig("mnnllm_linear_w4a8_static", _c.c_int,
+     [_P, _P, _P, _c.c_int, _c.c_int, _c.c_int, _c.c_int, _c.c_int, _c.c_int, _P])
 _sig("mnnllm_quantize_activations", _c.c_int, [_P, _c.c_int, _c.c_int, _c.c_int, _c.c_int, _P, _P, _P, _P])
 _sig("mnnllm_debug_w4a8_partials", _c.c_int,
      [_P, _c.c_int, _P, _P, _P, _P, _P, _c.c_int, _c.c_int, _c.c_int, _c.c_int, _P])
@@ -74,7 +76,7 @@ _sig("mnnllm_device_supported", _c.c_int, [])
 EXPORTS = [
     "mnnllm_status_string", "mnnllm_packed_size_w4", "mnnllm_pack_w4", "mnnllm_unpack_w4", "mnnllm_packed_info",
     "mnnllm_packed_size_w8", "mnnllm_pack_w8", "mnnllm_unpack_w8", "mnnllm_linear_w4a16", "mnnllm_linear_w4a16_ex",
-    "mnnllm_linear_w4a16_batch", "mnnllm_linear_w8a16", "mnnllm_workspace_size_w4a8", "mnnllm_linear_w4a8",
+    "mnnllm_linear_w4a16_batch", "mnnllm_linear_w8a16", "mnnllm_workspace_size_w4a8", "mnnllm_linear_w4a8", "mnnllm_linear_w4a8_static",
     "mnnllm_quantize_activations", "mnnllm_debug_w4a8_partials", "mnnllm_read_status", "mnnllm_device_supported",
 ]
 
@@ -207,6 +209,18 @@ def linear_w4a8(x, packed, y, M, N, K, group, workspace, workspace_bytes, x_dtyp
                 stream=None) -> None:
     _check(lib.mnnllm_linear_w4a8(_ptr(x), _ptr(packed), _ptr(y), M, N, K, group, x_dtype, y_dtype, _ptr(workspace),
                                   workspace_bytes, _stream(stream)), "linear_w4a8")
+
+
+STATIC_SCRATCH_BYTES = 8 << 20
+
+
+def linear_w4a8_static(x, packed, y, M, N, K, group, x_dtype=F16, y_dtype=F16, stream=None) -> None:
+    """W4A8 linear that needs no workspace from the caller: for code that may not allocate device
+    memory.  The scratch is a fixed ``STATIC_SCRATCH_BYTES`` array inside the library; problems that
+    need more raise ``MnnllmError`` (status 6).  Calls that may overlap on the GPU share that
+    array and race; keep them on one stream."""
+    _check(lib.mnnllm_linear_w4a8_static(_ptr(x), _ptr(packed), _ptr(y), M, N, K, group, x_dtype, y_dtype,
+                                         _stream(stream)), "linear_w4a8_static")
 
 
 def quantize_activations(x, M, K, group, a_q, a_scale, A, x_dtype=F16, stream=None) -> None:

@@ -33,6 +33,26 @@ Workspace workspace_layout(int M, int K, int group) {
     return w;
 }
 
+// Scratch of mnnllm_linear_w4a8_static: lives in the library's device image, one copy on every GPU
+// that loads the library, for the lifetime of the process.  Host code may not use the symbol as an
+// address; static_scratch_ptr() asks the runtime for the device address once per device.
+static __device__ __align__(256) unsigned char g_static_scratch[MNNLLM_STATIC_SCRATCH_BYTES];
+
+void* static_scratch_ptr() {
+    static void* ptrs[64];
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    if (!ptrs[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress((void**)&p, g_static_scratch) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return nullptr;
+        }
+        ptrs[dev] = p;
+    }
+    return ptrs[dev];
+}
+
 }  // namespace
 
 extern "C" {
@@ -113,6 +133,22 @@ int mnnllm_debug_w4a8_partials(const void* x, int x_dtype, const void* packed, i
         return e == cudaErrorNotSupported ? MNNLLM_ERR_UNSUPPORTED : MNNLLM_ERR_CUDA;
     }
     return MNNLLM_OK;
+}
+
+int mnnllm_linear_w4a8_static(const void* x, const void* packed, void* y, int M, int N, int K, int group, int x_dtype,
+                              int y_dtype, void* stream) {
+    const int st = check_xq(x, x_dtype, M, K, group);
+    if (st != MNNLLM_OK) return st;
+    if (!packed || !y || N < 1) return MNNLLM_ERR_INVALID_ARG;
+    // the activations' int8 copy, scales and group sums must fit the built-in scratch
+    if (workspace_layout(M, K, group).total > (size_t)MNNLLM_STATIC_SCRATCH_BYTES) return MNNLLM_ERR_WORKSPACE;
+    if (!device_is_supported()) return MNNLLM_ERR_UNSUPPORTED;
+    void* scratch = static_scratch_ptr();
+    if (!scratch) return MNNLLM_ERR_CUDA;
+    // every byte of the scratch that the GEMM reads is written by the quantiser of the same call,
+    // so nothing left over from an earlier call needs clearing
+    return mnnllm_linear_w4a8(x, packed, y, M, N, K, group, x_dtype, y_dtype, scratch, MNNLLM_STATIC_SCRATCH_BYTES,
+                              stream);
 }
 
 }  // extern "C"
