@@ -342,10 +342,9 @@ def run_ours(args):
     e2e_ms = ee0.elapsed_time(ee1)
     sampler.stop()
 
-    if dist is not None:
-        t = torch.tensor([ms, e2e_ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms, e2e_ms = float(t[0]), float(t[1])
+    from paper_2506_10443_b200.replicas import max_over_ranks
+
+    ms, e2e_ms = max_over_ranks([ms, e2e_ms], "cuda")   # a step takes as long as its slowest replica
 
     if rank == 0:
         peaks, peaks_kind = measured_peaks()

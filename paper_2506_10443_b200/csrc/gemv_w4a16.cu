@@ -59,7 +59,7 @@ template <int GROUP, int MP, bool FULL>
 __device__ __forceinline__ void quantum_mma(const uint4* __restrict__ slabs, int lane, int ns,
                                             const uint32_t (&B)[8][4][2], float (&D)[Cfg<GROUP, MP>::NSETS][4]) {
     using C = Cfg<GROUP, MP>;
-    constexpr int NBANK = C::NSETS == 1 ? 2 : 1;
+    constexpr int NBANK = C::NSETS == 1 ? 2 : 1;  // four banks spill at the 128-register cap and run slower
     constexpr uint32_t LO = 0x000F000Fu, HI = 0x00F000F0u, M1024 = 0x64006400u, M64 = 0x54005400u;
     float acc[C::NSETS][NBANK][4];
 #pragma unroll
@@ -160,10 +160,16 @@ gemv_w4a16_kernel(const __grid_constant__ GemvLaunch L, uint32_t* __restrict__ s
     };
     const uint8_t* i_src = i_rd < n_rounds ? src_of(i_rd, 0) : body;
     uint32_t i_bytes = bytes_of(0);
+    // weights are read once per token: mark their lines evict-first so that the stream does not
+    // push the activations (written by the previous kernel, read by the next) out of L2
+    const uint64_t stream_policy = policy_evict_first();
+    // every lane keeps the (uniform) producer state; one elected lane issues the copy
     auto issue_next = [&]() {
         if (i_rd >= n_rounds) return;
-        mbar_arrive_expect_tx(&bars[i_slot], i_bytes);
-        bulk_g2s(ring + (size_t)i_slot * C::QB, i_src, i_bytes, &bars[i_slot]);
+        if (elect_one()) {
+            mbar_arrive_expect_tx(&bars[i_slot], i_bytes);
+            bulk_g2s_hint(ring + (size_t)i_slot * C::QB, i_src, i_bytes, &bars[i_slot], stream_policy);
+        }
         i_slot = (i_slot + 1 == S) ? 0 : i_slot + 1;
         i_src += it_stride;
         if (++i_it == i_nit) {
@@ -180,8 +186,7 @@ gemv_w4a16_kernel(const __grid_constant__ GemvLaunch L, uint32_t* __restrict__ s
     };
 
     pdl_launch_dependents();
-    if (lane == 0)
-        for (int s = 0; s < S; ++s) issue_next();
+    for (int s = 0; s < S; ++s) issue_next();
     // everything above touched only weights; the activations may come from the previous kernel
     pdl_wait();
 
@@ -305,7 +310,7 @@ gemv_w4a16_kernel(const __grid_constant__ GemvLaunch L, uint32_t* __restrict__ s
                     if (ns == 8) rescale(C::GC); else rescale(ng);
                     // the slot has been read: release and refill it before the (register-only) tail
                     __syncwarp();
-                    if (lane == 0) issue_next();
+                    issue_next();
                     slot = (slot + 1 == S) ? 0 : slot + 1;
                     phase ^= (slot == 0) ? 1u : 0u;
 

@@ -74,6 +74,7 @@ gemv_w8a16_kernel(const __grid_constant__ GemvLaunch L, uint32_t* __restrict__ s
 
     int i_rd = 0, i_t = 0, i_it = 0, i_nit = nit_of(0), i_slot = 0;
     while (i_rd < n_rounds && i_nit == 0) { ++i_rd; i_nit = i_rd < n_rounds ? nit_of(i_rd) : 0; }
+    const uint64_t stream_policy = policy_evict_first();  // weights are read once: keep them from displacing x in L2
     auto issue_next = [&]() {
         if (i_rd >= n_rounds) return;
         const int j = j0 + i_t * jstride;
@@ -82,7 +83,7 @@ gemv_w8a16_kernel(const __grid_constant__ GemvLaunch L, uint32_t* __restrict__ s
         const uint32_t bytes = (uint32_t)(ns * kSlabBytes);
         const uint8_t* src = P.packed + kHeaderBytes + (size_t)rb * P.row_block_bytes + (size_t)j * QB;
         mbar_arrive_expect_tx(&bars[i_slot], bytes);
-        bulk_g2s(ring + (size_t)i_slot * QB, src, bytes, &bars[i_slot]);
+        bulk_g2s_hint(ring + (size_t)i_slot * QB, src, bytes, &bars[i_slot], stream_policy);
         i_slot = (i_slot + 1 == S) ? 0 : i_slot + 1;
         if (++i_it == i_nit) {
             i_it = 0;
