@@ -5,7 +5,7 @@
 //
 // One CTA computes a tile of 128 weight rows x 128 tokens.  The weights are the M side of the MMA,
 // so that a tensor-memory lane is one output channel n and its per-group scale is a per-thread
-// scalar in the drain.  Warp roles (15 warps):
+// scalar in the drain.  Warp roles (23 warps):
 //   warp 0      producer: TMA loads of the packed int4 codes (the packed buffer seen as a 2-D tensor
 //               [row block][bytes]: one box of 8 row blocks x 1 KiB per stage; issuing one small bulk
 //               copy per row block instead costs ~75 cycles each and starves the pipeline) and of
@@ -16,10 +16,12 @@
 //               accumulators per group; kind::f16 for the zero-point term) and the commits
 //   warps 2-5   unpack: packed int4 codes (shared-memory ring) -> int8 K-major tile in the
 //               128B-swizzled layout the MMA reads
-//   warp 14     scales: each (row, group) pair of the stage: the fp32 scale for the drain; (s z)
+//   warp 22     scales: each (row, group) pair of the stage: the fp32 scale for the drain; (s z)
 //               split into fp16 hi + lo for the zero-point MMA (a separate warp, because these
 //               conversion chains would otherwise sit on the unpack warps' critical path)
-//   warps 6-13  drain: every group's 128 x 128 int32 partial tile leaves tensor memory
+//   warps 6-21  drain (four per lane quarter, 32 token columns each: the loop is a chain of
+//               latencies, so more warps per scheduler hide it better than longer warps): every
+//               group's 128 x 128 int32 partial tile leaves tensor memory
 //               (tcgen05.ld), is converted (integer add of a float bit pattern + float subtract: the
 //               cvt instruction runs at 16 lanes per clock per SM and would bound the kernel) and
 //               accumulated as acc += s * P in registers while the
@@ -52,8 +54,9 @@ constexpr int kScaleSlots = 2 * kStages + 4;  // groups whose scales may be live
 constexpr int kPkStages = 6;                  // ring of packed-code stages (8 KiB each)
 constexpr int kPkLead = 2;                    // stages the packed ring is produced ahead of the activations
 constexpr int kTabSlots = 3;                  // ring of per-chunk (scale, zero) tables (8 row blocks x 512 B)
-constexpr int kThreads = 15 * 32;
-constexpr int kUnpackWarp0 = 2, kDrainWarp0 = 6, kScaleWarp = 14;
+constexpr int kDrainWarps = 16;
+constexpr int kUnpackWarp0 = 2, kDrainWarp0 = 6, kScaleWarp = kDrainWarp0 + kDrainWarps;
+constexpr int kThreads = (kScaleWarp + 1) * 32;
 constexpr uint32_t kMaxPolls = 1u << 22;
 constexpr int kAcc = 3;                       // int32 group accumulators in tensor memory (128 columns each)
 constexpr uint32_t kTmemCols = 512;           // 3 x 128 int32 accumulators + 128 fp32 zero-point term
@@ -140,7 +143,7 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < kStages; ++i) { mbar_init(&ab_full[i], 6); mbar_init(&ab_empty[i], 1); }
-        for (int i = 0; i < kAcc; ++i) { mbar_init(&tm_full[i], 1); mbar_init(&tm_empty[i], 8); }
+        for (int i = 0; i < kAcc; ++i) { mbar_init(&tm_full[i], 1); mbar_init(&tm_empty[i], kDrainWarps); }
         for (int i = 0; i < 2; ++i) { mbar_init(&c_full[i], 2); mbar_init(&c_empty[i], 1); }
         mbar_init(corr_done, 1);
         for (int i = 0; i < kPkStages; ++i) { mbar_init(&pk_full[i], 1); mbar_init(&pk_empty[i], 4); }
@@ -162,6 +165,7 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
     const uint32_t tmem_base = *tmem_slot;
 
     // a failed wait marks the CTA as aborted; every role then leaves its loop
+    // (every lane polls: letting one lane poll and broadcasting its verdict was measured 2x slower)
     auto wait = [&](uint64_t* bar, uint32_t parity, uint32_t code) -> bool {
         if (mbar_wait_bounded(bar, parity, kMaxPolls)) return true;
         if (*abort_flag == 0) {
@@ -174,7 +178,7 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
     if (warp == 0) {
         // ------------------------------------------------------------------ producer (TMA)
         const int rb0 = n0 / kRowsPerBlock;
-        for (int i = 0; i < n_stages + kPkLead && !*abort_flag; ++i) {
+        for (int i = 0; i < n_stages + kPkLead; ++i) {
             if (i < n_stages) {
                 // packed codes of stage i (and, at the start of a 512-k chunk, its scale/zero tables)
                 const int pslot = i % kPkStages, j = i >> 2;
@@ -218,21 +222,26 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issue
+        // Per stage: one wait for the operands, one for each accumulator, then a single elected
+        // region issues every MMA and commit of the stage back to back (the issue path is a serial
+        // chain of ~50-cycle steps; done once per stage instead of once per group it stays shorter
+        // than the drain).
         int gcount = 0, ccount = 0;
         const uint32_t wq_addr = smem_u32(smem + Smem::wq), aq_addr = smem_u32(smem + Smem::aq);
         bool ok = true;
-        for (int st = 0; st < n_stages && ok && !*abort_flag; ++st) {
+        for (int st = 0; st < n_stages && ok; ++st) {
             const int slot = st % kStages, round = st / kStages;
-            if (!wait(&ab_full[slot], round & 1, 3)) break;
-            tc_fence_after_sync();
             const int ngr = (G - st * GPS) < GPS ? (G - st * GPS) : GPS;
-            for (int gi = 0; gi < ngr; ++gi) {
-                const int b = gcount % kAcc;
-                if (!wait(&tm_empty[b], ((gcount / kAcc) & 1) ^ 1, 4)) { ok = false; break; }
-                tc_fence_after_sync();
-                if (elect_one()) {
-                    const uint64_t da = desc_sw128(wq_addr + slot * kStageBytes);
-                    const uint64_t db = desc_sw128(aq_addr + slot * kStageBytes);
+            if (!wait(&ab_full[slot], round & 1, 3)) break;
+            for (int gi = 0; gi < ngr; ++gi)
+                if (!wait(&tm_empty[(gcount + gi) % kAcc], (((gcount + gi) / kAcc) & 1) ^ 1, 4)) { ok = false; break; }
+            if (!ok) break;
+            tc_fence_after_sync();
+            if (elect_one()) {
+                const uint64_t da = desc_sw128(wq_addr + slot * kStageBytes);
+                const uint64_t db = desc_sw128(aq_addr + slot * kStageBytes);
+                for (int gi = 0; gi < ngr; ++gi) {
+                    const int b = (gcount + gi) % kAcc;
 #pragma unroll
                     for (int kk = 0; kk < GROUP / 32; ++kk) {
                         const uint64_t adv = (uint64_t)((gi * GROUP + kk * 32) >> 4);
@@ -240,11 +249,10 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
                     }
                     mma_commit(&tm_full[b]);
                 }
-                __syncwarp();
-                ++gcount;
+                mma_commit(&ab_empty[slot]);
             }
-            if (!ok) break;
-            if (elect_one()) mma_commit(&ab_empty[slot]);
+            __syncwarp();
+            gcount += ngr;
             if (!PARTIALS && ((gcount & 3) == 0 || st == n_stages - 1)) {
                 const int cslot = ccount & 1;
                 if (!wait(&c_full[cslot], (ccount >> 1) & 1, 5)) break;
@@ -254,9 +262,9 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
                                desc_sw32(smem_u32(smem + Smem::cb + cslot * kCorrBytes)), kIdescF16, ccount > 0);
                     mma_commit(&c_empty[cslot]);
                 }
+                __syncwarp();
                 ++ccount;
             }
-            __syncwarp();
         }
         if (!PARTIALS && elect_one()) mma_commit(corr_done);
         __syncwarp();
@@ -264,7 +272,7 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
         // ------------------------------------------------------------------ unpack
         const int wu = warp - kUnpackWarp0;
         const int nrb = (p.n_row_blocks - n0 / kRowsPerBlock) < 8 ? (p.n_row_blocks - n0 / kRowsPerBlock) : 8;
-        for (int st = 0; st < n_stages && !*abort_flag; ++st) {
+        for (int st = 0; st < n_stages; ++st) {
             const int slot = st % kStages, round = st / kStages;
             const int pslot = st % kPkStages, j = st >> 2;
             const int ns_chunk = (p.n_slabs - 8 * j) < 8 ? (p.n_slabs - 8 * j) : 8;
@@ -282,21 +290,27 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(&pk_empty[pslot]);
+            // codes -> int8 (registers) before the stage's slot is waited for; then only the stores
+            constexpr uint32_t M4 = 0x0F0F0F0Fu;
+            uint4 lo8[4], hi8[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const uint4 w = cur[i];
+                lo8[i] = make_uint4(w.x & M4, (w.x >> 4) & M4, w.y & M4, (w.y >> 4) & M4);   // row R0
+                hi8[i] = make_uint4(w.z & M4, (w.z >> 4) & M4, w.w & M4, (w.w >> 4) & M4);   // row R0 + 8
+            }
             if (!wait(&ab_empty[slot], (round & 1) ^ 1, 6)) break;
-
-            // codes -> int8, 128B-swizzled K-major rows
+            // 128B-swizzled K-major rows
             uint8_t* wq = smem + Smem::wq + slot * kStageBytes;
             const int r = lane >> 2, c = lane & 3;
-            constexpr uint32_t M4 = 0x0F0F0F0Fu;
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 const int sidx = i * 4 + wu;
                 const int R0 = (sidx >> 1) * 16 + r;          // rows R0 and R0 + 8 of the tile
                 const int kc = (sidx & 1) * 4 + c;            // 16-byte chunk of the 128-byte row
                 const uint32_t off = (uint32_t)(R0 >> 3) * 1024u + (uint32_t)r * 128u + (uint32_t)((kc ^ r) << 4);
-                const uint4 w = cur[i];
-                *reinterpret_cast<uint4*>(wq + off) = make_uint4(w.x & M4, (w.x >> 4) & M4, w.y & M4, (w.y >> 4) & M4);
-                *reinterpret_cast<uint4*>(wq + off + 1024u) = make_uint4(w.z & M4, (w.z >> 4) & M4, w.w & M4, (w.w >> 4) & M4);
+                *reinterpret_cast<uint4*>(wq + off) = lo8[i];
+                *reinterpret_cast<uint4*>(wq + off + 1024u) = hi8[i];
             }
             fence_proxy_async_smem();
             __syncwarp();
@@ -306,7 +320,7 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
         // ------------------------------------------------------------------ scales and (s z) halves
         const int nrb = (p.n_row_blocks - n0 / kRowsPerBlock) < 8 ? (p.n_row_blocks - n0 / kRowsPerBlock) : 8;
         bool ok = true;
-        for (int st = 0; st < n_stages && ok && !*abort_flag; ++st) {
+        for (int st = 0; st < n_stages && ok; ++st) {
             const int slot = st % kStages, round = st / kStages;
             const int j = st >> 2, tslot = j % kTabSlots;
             const int ns_chunk = (p.n_slabs - 8 * j) < 8 ? (p.n_slabs - 8 * j) : 8;
@@ -328,7 +342,10 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&tab_empty[tslot]);
             }
-            if (!wait(&ab_empty[slot], (round & 1) ^ 1, 14)) break;
+            // The conversion chains and the zero-point tile (which has its own flow control) come
+            // first; only the cheap publication of the scales waits for the stage's slot, so that
+            // this warp is never what the MMA waits for.
+            float sreg[4][GPS];
 #pragma unroll
             for (int gi = 0; gi < GPS; ++gi) {
                 const int g = st * GPS + gi;
@@ -340,7 +357,7 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
                     const int row = lane + 32 * i;
                     const __half2 h2 = *reinterpret_cast<const __half2*>(&zc[i][gi]);
                     const float s = __low2float(h2), z = __high2float(h2);
-                    scale_ring[(g % kScaleSlots) * kTileN + row] = s;
+                    sreg[i][gi] = s;
                     if (!PARTIALS) {
                         const float szf = s * z;  // exact: 11-bit x 11-bit significands
                         const __half hi = __float2half_rn(szf);
@@ -362,45 +379,50 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
                 }
             }
             if (!ok) break;
+            if (!wait(&ab_empty[slot], (round & 1) ^ 1, 14)) break;
+#pragma unroll
+            for (int gi = 0; gi < GPS; ++gi) {
+                const int g = st * GPS + gi;
+                if (g >= G) break;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) scale_ring[(g % kScaleSlots) * kTileN + lane + 32 * i] = sreg[i][gi];
+            }
             __syncwarp();
             if (lane == 0) mbar_arrive(&ab_full[slot]);
         }
     } else {
         // ------------------------------------------------------------------ drain + epilogue
         const int q4 = warp & 3;                      // tensor-memory lane quarter this warp may read
-        const int half = (warp - kDrainWarp0) >> 2;   // which 64 token columns
+        const int part = (warp - kDrainWarp0) >> 2;   // which 32 token columns
         const int nl = q4 * 32 + lane, n = n0 + nl;
-        const uint32_t lane_base = tmem_base + ((uint32_t)(q4 * 32) << 16);
-        float acc[64];
+        const uint32_t lane_base = tmem_base + ((uint32_t)(q4 * 32) << 16) + part * 32;
+        float acc[32];
 #pragma unroll
-        for (int i = 0; i < 64; ++i) acc[i] = 0.f;
+        for (int i = 0; i < 32; ++i) acc[i] = 0.f;
         bool ok = true;
-        for (int g = 0; g < G && !*abort_flag; ++g) {
+        for (int g = 0; g < G; ++g) {
             const int b = g % kAcc;
             if (!wait(&tm_full[b], (g / kAcc) & 1, 8)) { ok = false; break; }
             tc_fence_after_sync();
+            uint32_t v[32];
+            tmem_ld_x32(lane_base + b * kTileT, v);
             const float sf = scale_ring[(g % kScaleSlots) * kTileN + nl];
+            tmem_ld_wait();
+            if (PARTIALS) {
+                if (n < p.N)
 #pragma unroll
-            for (int cc = 0; cc < 2; ++cc) {
-                uint32_t v[32];
-                tmem_ld_x32(lane_base + b * kTileT + half * 64 + cc * 32, v);
-                tmem_ld_wait();
-                if (PARTIALS) {
-                    if (n < p.N)
+                    for (int j = 0; j < 32; ++j) {
+                        const int m = m0 + part * 32 + j;
+                        if (m < p.M) p.P[((size_t)m * p.N + n) * G + g] = (int32_t)v[j];
+                    }
+            } else {
+                // int32 -> fp32 without the conversion instruction (16 lanes per clock per SM, it
+                // would bound the kernel): |P| < 2^22, so adding the bit pattern of 1.5 * 2^23
+                // (ulp 1) as an integer and subtracting the same constant as a float is exact
+                // (packed f32x2 arithmetic was measured slower here)
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) {
-                            const int m = m0 + half * 64 + cc * 32 + j;
-                            if (m < p.M) p.P[((size_t)m * p.N + n) * G + g] = (int32_t)v[j];
-                        }
-                } else {
-                    // int32 -> fp32 without the conversion instruction (16 lanes per clock per SM, it
-                    // would bound the kernel): |P| < 2^22, so adding the bit pattern of 1.5 * 2^23
-                    // (ulp 1) as an integer and subtracting the same constant as a float is exact
-                    // (packed f32x2 arithmetic was measured slower here: 950 vs 520 cycles per group)
-#pragma unroll
-                    for (int j = 0; j < 32; ++j)
-                        acc[cc * 32 + j] = fmaf(sf, __uint_as_float(v[j] + 0x4B400000u) - 12582912.0f, acc[cc * 32 + j]);
-                }
+                for (int j = 0; j < 32; ++j)
+                    acc[j] = fmaf(sf, __uint_as_float(v[j] + 0x4B400000u) - 12582912.0f, acc[j]);
             }
             tc_fence_before_sync();
             __syncwarp();
@@ -408,18 +430,15 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
         }
         if (!PARTIALS && ok && !*abort_flag && wait(corr_done, 0, 9)) {
             tc_fence_after_sync();
+            uint32_t v[32];
+            tmem_ld_x32(lane_base + kColCorr, v);
+            tmem_ld_wait();
 #pragma unroll
-            for (int cc = 0; cc < 2; ++cc) {
-                uint32_t v[32];
-                tmem_ld_x32(lane_base + kColCorr + half * 64 + cc * 32, v);
-                tmem_ld_wait();
-#pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    const int m = m0 + half * 64 + cc * 32 + j;
-                    if (m < p.M && n < p.N) {
-                        const float val = __ldg(p.a_scale + m) * (acc[cc * 32 + j] - __uint_as_float(v[j]));
-                        store_y(p.y, p.y_dtype, (size_t)m * p.N + n, val);
-                    }
+            for (int j = 0; j < 32; ++j) {
+                const int m = m0 + part * 32 + j;
+                if (m < p.M && n < p.N) {
+                    const float val = __ldg(p.a_scale + m) * (acc[j] - __uint_as_float(v[j]));
+                    store_y(p.y, p.y_dtype, (size_t)m * p.N + n, val);
                 }
             }
         }
