@@ -28,7 +28,7 @@ using namespace ptx;
 
 namespace {
 
-constexpr uint32_t kMaxPolls = 1u << 22;
+constexpr uint32_t kMaxPolls = 1u << 15;  // x 20 us per try: gives up after ~0.65 s
 
 template <int GROUP, int MP>
 struct Cfg {

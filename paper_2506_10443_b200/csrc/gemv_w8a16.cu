@@ -16,7 +16,7 @@ using namespace ptx;
 
 namespace {
 
-constexpr uint32_t kMaxPolls = 1u << 22;
+constexpr uint32_t kMaxPolls = 1u << 15;  // x 20 us per try: gives up after ~0.65 s
 constexpr int QB = 16 * kSlabBytes;                 // bytes of a full quantum
 constexpr int PART_FLOATS = kGemvMaxRBI * 8 * 16;   // [it][token][row]
 constexpr int XS_FLOATS = 8;                        // per warp: sum of x over its chunks, per token
