@@ -250,6 +250,78 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+def _time_steps(step, steps, warmup):
+    """Milliseconds per step of `step()` on the current stream (CUDA events, after warm-up)."""
+    import torch
+
+    for _ in range(warmup):
+        step()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / steps
+
+
+def secondary_measurements(stack, model, peaks):
+    """The other rows of the hot path on the same GPU, reported beside the headline: the W4A8
+    prefill of a 1024-token prompt over the same packed weights, and the LM-head GEMVs (int4 group
+    128 and int8 per channel, fp32 logits).  Each entry carries its own roofline fraction."""
+    import torch
+
+    from paper_2506_10443_b200 import binding as B
+    from paper_2506_10443_b200 import inputs
+    from paper_2506_10443_b200.workloads import LinearStack, w4_bytes
+
+    out = {}
+    hbm = float(peaks["hbm_gbs"])
+    int8_peak = float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])) * INT8_OVER_BF16
+
+    M = 1024
+    pre = LinearStack(model, 3, M, GROUP, outliers=True, weights_from=stack)
+    pre.run_w4a8()
+    assert B.read_status() == 0
+    g = torch.cuda.CUDAGraph()
+    cap = torch.cuda.Stream()
+    cap.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.graph(g, stream=cap):
+        pre.run_w4a8(cap)
+    ms = _time_steps(g.replay, 20, 3)
+    tops = pre.ops / (ms * 1e-3) / 1e12
+    out["prefill_w4a8_m1024"] = {
+        "metric": "prefill W4A8 TOPS", "value": tops, "unit": "TOPS", "ms_per_step": ms, "tokens_per_s": M / (ms * 1e-3),
+        "roofline": {"bound": "tensor", "kernel": "gemm_w4a8_kernel", "achieved": tops, "peak": int8_peak,
+                     "frac": tops / int8_peak, "frac_of_nominal_4500": tops / 4500.0}}
+    del g, pre
+
+    N, K, grp = inputs.LM_HEAD["N"], inputs.LM_HEAD["K"], inputs.LM_HEAD["group"]
+    W = inputs.weights(inputs.seed_for(5, 0, 0, 0), N, K)
+    x = torch.from_numpy(inputs.activations(inputs.seed_for(5, 0, 0, 1), 4, K)).cuda()
+    y = torch.empty((4, N), dtype=torch.float32, device="cuda")
+    p4 = torch.from_numpy(B.pack_w4(W, grp)).cuda()
+    for Mh in (1, 4):
+        ms = _time_steps(lambda: B.linear_w4a16_ex(x, p4, y, Mh, N, K, grp, B.F16, B.F32), 50, 5)
+        nbytes = w4_bytes(N, K, grp) + 2 * Mh * K + 4 * Mh * N
+        gbs = nbytes / (ms * 1e-3) / 1e9
+        out["lm_head_w4a16_g128_m%d" % Mh] = {
+            "metric": "decode W4 GEMV GB/s", "value": gbs, "unit": "GB/s", "us": 1e3 * ms,
+            "roofline": {"bound": "hbm", "kernel": "gemv_w4a16_kernel", "achieved": gbs, "peak": hbm, "frac": gbs / hbm}}
+    del p4
+    p8 = torch.from_numpy(B.pack_w8(W)).cuda()
+    del W
+    ms = _time_steps(lambda: B.linear_w8a16(x, p8, y, 1, N, K, B.F32), 50, 5)
+    nbytes = N * K + 4 * N + 2 * K + 4 * N
+    gbs = nbytes / (ms * 1e-3) / 1e9
+    out["lm_head_w8a16_m1"] = {
+        "metric": "decode W8 GEMV GB/s", "value": gbs, "unit": "GB/s", "us": 1e3 * ms,
+        "roofline": {"bound": "hbm", "kernel": "gemv_w8a16_kernel", "achieved": gbs, "peak": hbm, "frac": gbs / hbm}}
+    assert B.read_status() == 0
+    return out
+
+
 def run_ours(args):
     import torch
 
@@ -386,15 +458,20 @@ def run_ours(args):
             "clocks": sampler.summary(t0, t1),
             "roofline": roof,
         }
+        if world == 1 and kind == "decode" and not args.no_secondary:
+            line["secondary"] = secondary_measurements(stack, model, peaks)
         if world == 1 and not args.no_cpu_baseline:
             sample, what, threads = oracle_sample(wl, model, args.cpu_seconds)
             t = time.perf_counter()
-            for x, q, s, z, _ in sample:
-                oracle_linear(kind, x, q, s, z)
+            passes = 0
+            while passes == 0 or time.perf_counter() - t < args.cpu_seconds:   # about cpu_seconds of oracle work
+                for x, q, s, z, _ in sample:
+                    oracle_linear(kind, x, q, s, z)
+                passes += 1
             spent = time.perf_counter() - t
             line["cpu_baseline"] = {
-                "value": sum(p[4] for p in sample) / spent / scale_of(kind), "unit": unit, "cores": threads,
-                "kind": "oracle", "sample": "%s, %.1f s of oracle time" % (what, spent),
+                "value": passes * sum(p[4] for p in sample) / spent / scale_of(kind), "unit": unit, "cores": threads,
+                "kind": "oracle", "sample": "%s, %d pass(es), %.1f s of oracle time" % (what, passes, spent),
             }
         print(json.dumps(line), flush=True)
     if dist is not None:
@@ -410,6 +487,8 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
     ap.add_argument("--no-graph", action="store_true", help="issue the launches directly instead of replaying a CUDA graph")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-secondary", action="store_true",
+                    help="skip the extra measurements (prefill on the same weights, LM-head GEMVs) added to the line")
     ap.add_argument("--cpu-seconds", type=float, default=10.0, help="oracle time budget of the cpu_baseline leg")
     args = ap.parse_args()
     decode = WORKLOADS[args.workload]["kind"] == "decode"
