@@ -45,7 +45,8 @@ __device__ __forceinline__ void widen8<__nv_bfloat16>(const uint4& v, float (&f)
 template <typename T>
 __global__ void __launch_bounds__(kThreads) act_quant_kernel(const T* __restrict__ x, int K, int group,
                                                              int8_t* __restrict__ a_q, float* __restrict__ a_scale,
-                                                             int32_t* __restrict__ A, uint2* __restrict__ AC, int G4) {
+                                                             int32_t* __restrict__ A, uint2* __restrict__ AC, int G4,
+                                                             uint32_t code_xor) {
     __shared__ float warp_max[kThreads / 32];
     ptx::pdl_launch_dependents();
     ptx::pdl_wait();
@@ -95,6 +96,9 @@ __global__ void __launch_bounds__(kThreads) act_quant_kernel(const T* __restrict
                    ((uint32_t)(q[3] & 0xFF) << 24);
             pk.y = (uint32_t)(q[4] & 0xFF) | ((uint32_t)(q[5] & 0xFF) << 8) | ((uint32_t)(q[6] & 0xFF) << 16) |
                    ((uint32_t)(q[7] & 0xFF) << 24);
+            // code_xor = 0x80808080 stores a_q + 128 as unsigned bytes (the GEMM's operand form)
+            pk.x ^= code_xor;
+            pk.y ^= code_xor;
             out[v] = pk;
         }
         // group sums: a group is 8 (or 16) consecutive vectors, i.e. consecutive lanes of one warp
@@ -121,7 +125,8 @@ __global__ void __launch_bounds__(kThreads) act_quant_kernel(const T* __restrict
 }  // namespace
 
 cudaError_t act_quant_launch(const void* x, int x_dtype, int M, int K, int group, int8_t* a_q, float* a_scale,
-                             int32_t* A, void* AC, cudaStream_t stream) {
+                             int32_t* A, void* AC, bool offset128, cudaStream_t stream) {
+    const uint32_t code_xor = offset128 ? 0x80808080u : 0u;
     const int G4 = (K / group + 3) / 4 * 4;
     uint2* ac = reinterpret_cast<uint2*>(AC);
     cudaLaunchConfig_t cfg = {};
@@ -135,9 +140,9 @@ cudaError_t act_quant_launch(const void* x, int x_dtype, int M, int K, int group
     cfg.numAttrs = 1;
     if (x_dtype == MNNLLM_F16)
         return cudaLaunchKernelEx(&cfg, act_quant_kernel<__half>, (const __half*)x, K, group, a_q, a_scale, A, ac,
-                                  G4);
+                                  G4, code_xor);
     return cudaLaunchKernelEx(&cfg, act_quant_kernel<__nv_bfloat16>, (const __nv_bfloat16*)x, K, group, a_q, a_scale,
-                              A, ac, G4);
+                              A, ac, G4, code_xor);
 }
 
 }  // namespace mnnllm

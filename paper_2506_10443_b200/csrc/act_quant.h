@@ -10,7 +10,9 @@ namespace mnnllm {
 // x [M, K] (fp16 or bf16) -> a_q int8 [M, K], a_scale fp32 [M], A int32 [M, K / group] (may be null)
 // and, when AC is not null, the group sums as fp16 quadruples (64h, l, 64h, l), A = 64h + l,
 // [M, G4] x 8 bytes with G4 = K / group rounded up to a multiple of 4 (padding written as zeros).
+// With offset128 the codes are stored as unsigned bytes a_q + 128 (what the GEMM multiplies); the
+// sums A and AC are those of the signed codes either way.
 cudaError_t act_quant_launch(const void* x, int x_dtype, int M, int K, int group, int8_t* a_q, float* a_scale,
-                             int32_t* A, void* AC, cudaStream_t stream);
+                             int32_t* A, void* AC, bool offset128, cudaStream_t stream);
 
 }  // namespace mnnllm

@@ -64,7 +64,7 @@ int mnnllm_quantize_activations(const void* x, int x_dtype, int M, int K, int gr
     if (!a_q || !a_scale || !A) return MNNLLM_ERR_INVALID_ARG;
     if (((uintptr_t)a_q & 15) || ((uintptr_t)a_scale & 3) || ((uintptr_t)A & 3)) return MNNLLM_ERR_ALIGNMENT;
     if (!device_is_supported()) return MNNLLM_ERR_UNSUPPORTED;
-    if (act_quant_launch(x, x_dtype, M, K, group, a_q, a_scale, A, nullptr, (cudaStream_t)stream) != cudaSuccess) {
+    if (act_quant_launch(x, x_dtype, M, K, group, a_q, a_scale, A, nullptr, false, (cudaStream_t)stream) != cudaSuccess) {
         (void)cudaGetLastError();
         return MNNLLM_ERR_CUDA;
     }
@@ -94,7 +94,7 @@ int mnnllm_linear_w4a8(const void* x, const void* packed, void* y, int M, int N,
     int8_t* a_q = (int8_t*)(ws + w.a_q);
     float* a_scale = (float*)(ws + w.a_scale);
     void* ac = ws + w.ac;
-    if (act_quant_launch(x, x_dtype, M, K, group, a_q, a_scale, nullptr, ac, (cudaStream_t)stream) != cudaSuccess) {
+    if (act_quant_launch(x, x_dtype, M, K, group, a_q, a_scale, nullptr, ac, true, (cudaStream_t)stream) != cudaSuccess) {
         (void)cudaGetLastError();
         return MNNLLM_ERR_CUDA;
     }
@@ -120,7 +120,9 @@ int mnnllm_debug_w4a8_partials(const void* x, int x_dtype, const void* packed, i
     if (!device_is_supported()) return MNNLLM_ERR_UNSUPPORTED;
     uint32_t* status = status_word_ptr();
     if (!status) return MNNLLM_ERR_CUDA;
-    if (act_quant_launch(x, x_dtype, M, K, group, a_q, a_scale, A, nullptr, (cudaStream_t)stream) != cudaSuccess) {
+    // the GEMM multiplies the codes in their unsigned form (a_q + 128); the caller gets the signed
+    // ones, written by a second run of the quantiser once the GEMM has consumed the buffer
+    if (act_quant_launch(x, x_dtype, M, K, group, a_q, a_scale, A, nullptr, true, (cudaStream_t)stream) != cudaSuccess) {
         (void)cudaGetLastError();
         return MNNLLM_ERR_CUDA;
     }
@@ -131,6 +133,10 @@ int mnnllm_debug_w4a8_partials(const void* x, int x_dtype, const void* packed, i
     if (e != cudaSuccess) {
         (void)cudaGetLastError();
         return e == cudaErrorNotSupported ? MNNLLM_ERR_UNSUPPORTED : MNNLLM_ERR_CUDA;
+    }
+    if (act_quant_launch(x, x_dtype, M, K, group, a_q, a_scale, A, nullptr, false, (cudaStream_t)stream) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return MNNLLM_ERR_CUDA;
     }
     return MNNLLM_OK;
 }

@@ -3,6 +3,15 @@
 //     P[m,n,g] = sum_{k in g} a_q[m,k] * q[n,k]                       int32, exact
 //     y[m,n]   = a_scale[m] * ( sum_g s[n,g] * P[m,n,g]  -  sum_g (s z)[n,g] * A[m,g] )
 //
+// The MMA multiplies the activations in their unsigned form a_u = a_q + 128 (written so by the
+// quantiser), so that its result P_u = P + 128 * Q[n,g], Q = sum of the group's codes, is never
+// negative.  A non-negative int32 below 2^23 IS a (denormal) float, P_u * 2^-149, bit for bit: the
+// drain needs no int->float conversion at all.  It subtracts the denormal 128 Q (exact) and
+// multiplies by s * 2^100 in one FMA, two instructions per partial; the accumulators carry
+// 2^-49 * sum_g s P and the epilogue scales back.  (cvt.rn.f32.s32 runs at 16 lanes per clock per SM
+// and would bound the kernel at 1024 cycles per group; adding a float bit pattern as an integer
+// and subtracting it as a float is exact too but costs three instructions per partial.)
+//
 // One CTA computes a tile of 128 weight rows x 128 tokens.  The weights are the M side of the MMA,
 // so that a tensor-memory lane is one output channel n and its per-group scale is a per-thread
 // scalar in the drain.  Warp roles (23 warps):
@@ -15,17 +24,15 @@
 //   warp 1      allocates tensor memory, issues tcgen05.mma (kind::i8 into one of three int32
 //               accumulators per group; kind::f16 for the zero-point term) and the commits
 //   warps 2-5   unpack: packed int4 codes (shared-memory ring) -> int8 K-major tile in the
-//               128B-swizzled layout the MMA reads
+//               128B-swizzled layout the MMA reads; the sum Q of every (row, group)'s codes
 //   warp 22     scales: each (row, group) pair of the stage: the fp32 scale for the drain; (s z)
 //               split into fp16 hi + lo for the zero-point MMA (a separate warp, because these
 //               conversion chains would otherwise sit on the unpack warps' critical path)
 //   warps 6-21  drain (four per lane quarter, 32 token columns each: the loop is a chain of
 //               latencies, so more warps per scheduler hide it better than longer warps): every
 //               group's 128 x 128 int32 partial tile leaves tensor memory
-//               (tcgen05.ld), is converted (integer add of a float bit pattern + float subtract: the
-//               cvt instruction runs at 16 lanes per clock per SM and would bound the kernel) and
-//               accumulated as acc += s * P in registers while the
-//               MMA fills the other accumulators; epilogue applies the zero-point term and a_scale.
+//               (tcgen05.ld) and is accumulated as acc += (s 2^100) * (P_u - 128 Q) in registers
+//               while the MMA fills the other accumulators; epilogue applies the zero-point term and a_scale.
 // The zero-point term is a rank-G product, evaluated on the tensor cores without loss:
 //   (s z) = hi + lo (fp16 each; s and z are fp16, so the product has 22 significant bits),
 //   A     = 64 h + l (both exact in fp16), four fp16 products per group, fp32 accumulation in a
@@ -75,7 +82,8 @@ struct Smem {
     static constexpr int pk = cb + 2 * kCorrBytes;
     static constexpr int tab = pk + kPkStages * kPkBytes;
     static constexpr int scale = tab + kTabSlots * kTabBytes;
-    static constexpr int bars = scale + kScaleSlots * kTileN * 4;
+    static constexpr int qsum = scale + kScaleSlots * kTileN * 4;   // 128 * Q per (group slot, row), as integers
+    static constexpr int bars = qsum + kScaleSlots * kTileN * 4;
     static constexpr int n_bars = 2 * kStages + 2 * kAcc + 2 + 2 + 1 + 2 * kPkStages + 2 * kTabSlots;
     static constexpr int misc = bars + n_bars * 8;
     static constexpr int total = misc + 16;
@@ -103,7 +111,8 @@ __device__ __forceinline__ uint64_t desc_sw32(uint32_t smem_addr) {
 }
 // instruction descriptors: D format (bits 4-5), A/B formats (7-9, 10-12), both K-major, N >> 3 at
 // bit 17, M >> 4 at bit 24
-constexpr uint32_t kIdescI8 = (2u << 4) | (1u << 7) | (1u << 10) | ((kTileT >> 3) << 17) | ((kTileN >> 4) << 24);
+// (kind::i8 formats: 0 = unsigned, 1 = signed 8 bit; codes 0..15 and activations a_q + 128 are both unsigned)
+constexpr uint32_t kIdescI8 = (2u << 4) | (0u << 7) | (0u << 10) | ((kTileT >> 3) << 17) | ((kTileN >> 4) << 24);
 constexpr uint32_t kIdescF16 = (1u << 4) | (0u << 7) | (0u << 10) | ((kTileT >> 3) << 17) | ((kTileN >> 4) << 24);
 
 __device__ __forceinline__ void store_y(void* y, int dtype, size_t idx, float v) {
@@ -136,6 +145,7 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + Smem::misc);
     volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + Smem::misc + 4);
     float* scale_ring = reinterpret_cast<float*>(smem + Smem::scale);
+    uint32_t* qsum_ring = reinterpret_cast<uint32_t*>(smem + Smem::qsum);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n0 = blockIdx.x * kTileN, m0 = blockIdx.y * kTileT;
@@ -283,7 +293,7 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
                 const uint4* pk = reinterpret_cast<const uint4*>(smem + Smem::pk + pslot * kPkBytes);
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
-                    const int sidx = i * 4 + wu;
+                    const int sidx = wu * 4 + i;   // row blocks 2 wu and 2 wu + 1, both slabs of each
                     const bool valid = (sidx >> 1) < nrb && (st & 3) * 2 + (sidx & 1) < ns_chunk;
                     cur[i] = valid ? pk[sidx * 32 + lane] : make_uint4(0, 0, 0, 0);
                 }
@@ -293,11 +303,20 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
             // codes -> int8 (registers) before the stage's slot is waited for; then only the stores
             constexpr uint32_t M4 = 0x0F0F0F0Fu;
             uint4 lo8[4], hi8[4];
+            uint32_t q0[4], q1[4];   // sums of the codes of rows R0 and R0 + 8 over the slab (after the lane reduction)
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 const uint4 w = cur[i];
                 lo8[i] = make_uint4(w.x & M4, (w.x >> 4) & M4, w.y & M4, (w.y >> 4) & M4);   // row R0
                 hi8[i] = make_uint4(w.z & M4, (w.z >> 4) & M4, w.w & M4, (w.w >> 4) & M4);   // row R0 + 8
+                uint32_t a = __dp4a(lo8[i].x, 0x01010101u, 0u), b = __dp4a(hi8[i].x, 0x01010101u, 0u);
+                a = __dp4a(lo8[i].y, 0x01010101u, a); b = __dp4a(hi8[i].y, 0x01010101u, b);
+                a = __dp4a(lo8[i].z, 0x01010101u, a); b = __dp4a(hi8[i].z, 0x01010101u, b);
+                a = __dp4a(lo8[i].w, 0x01010101u, a); b = __dp4a(hi8[i].w, 0x01010101u, b);
+                // the four lanes 4r .. 4r+3 hold the four 16-k pieces of the same rows
+                a += __shfl_xor_sync(0xffffffffu, a, 1); b += __shfl_xor_sync(0xffffffffu, b, 1);
+                a += __shfl_xor_sync(0xffffffffu, a, 2); b += __shfl_xor_sync(0xffffffffu, b, 2);
+                q0[i] = a; q1[i] = b;
             }
             if (!wait(&ab_empty[slot], (round & 1) ^ 1, 6)) break;
             // 128B-swizzled K-major rows
@@ -305,12 +324,26 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
             const int r = lane >> 2, c = lane & 3;
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                const int sidx = i * 4 + wu;
+                const int sidx = wu * 4 + i;
                 const int R0 = (sidx >> 1) * 16 + r;          // rows R0 and R0 + 8 of the tile
                 const int kc = (sidx & 1) * 4 + c;            // 16-byte chunk of the 128-byte row
                 const uint32_t off = (uint32_t)(R0 >> 3) * 1024u + (uint32_t)r * 128u + (uint32_t)((kc ^ r) << 4);
                 *reinterpret_cast<uint4*>(wq + off) = lo8[i];
                 *reinterpret_cast<uint4*>(wq + off + 1024u) = hi8[i];
+            }
+            // 128 * Q per (row, group) for the drain: a slab is a group of 64, two slabs a group of 128
+            if (c == 0) {
+#pragma unroll
+                for (int i = 0; i < 4; i += (GROUP == 64 ? 1 : 2)) {
+                    const int g = GROUP == 64 ? st * 2 + (i & 1) : st;
+                    if (g < G) {
+                        const int R0 = (wu * 2 + (i >> 1)) * 16 + r;
+                        const uint32_t s0 = GROUP == 64 ? q0[i] : q0[i] + q0[i + 1];
+                        const uint32_t s1 = GROUP == 64 ? q1[i] : q1[i] + q1[i + 1];
+                        qsum_ring[(g % kScaleSlots) * kTileN + R0] = 128u * s0;
+                        qsum_ring[(g % kScaleSlots) * kTileN + R0 + 8] = 128u * s1;
+                    }
+                }
             }
             fence_proxy_async_smem();
             __syncwarp();
@@ -385,7 +418,8 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
                 const int g = st * GPS + gi;
                 if (g >= G) break;
 #pragma unroll
-                for (int i = 0; i < 4; ++i) scale_ring[(g % kScaleSlots) * kTileN + lane + 32 * i] = sreg[i][gi];
+                for (int i = 0; i < 4; ++i)   // s * 2^100 (the drain's operand is the denormal P * 2^-149)
+                    scale_ring[(g % kScaleSlots) * kTileN + lane + 32 * i] = __fmul_rn(sreg[i][gi], 0x1p100f);
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(&ab_full[slot]);
@@ -407,22 +441,21 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
             uint32_t v[32];
             tmem_ld_x32(lane_base + b * kTileT, v);
             const float sf = scale_ring[(g % kScaleSlots) * kTileN + nl];
+            const uint32_t qb_bits = qsum_ring[(g % kScaleSlots) * kTileN + nl];   // 128 Q, also the float 128 Q 2^-149
+            const float qb = __uint_as_float(qb_bits);
             tmem_ld_wait();
             if (PARTIALS) {
                 if (n < p.N)
 #pragma unroll
                     for (int j = 0; j < 32; ++j) {
                         const int m = m0 + part * 32 + j;
-                        if (m < p.M) p.P[((size_t)m * p.N + n) * G + g] = (int32_t)v[j];
+                        if (m < p.M) p.P[((size_t)m * p.N + n) * G + g] = (int32_t)(v[j] - qb_bits);
                     }
             } else {
-                // int32 -> fp32 without the conversion instruction (16 lanes per clock per SM, it
-                // would bound the kernel): |P| < 2^22, so adding the bit pattern of 1.5 * 2^23
-                // (ulp 1) as an integer and subtracting the same constant as a float is exact
-                // (packed f32x2 arithmetic was measured slower here)
+                // v is P_u >= 0 and below 2^23: its bits are the float P_u * 2^-149; the subtraction of
+                // the denormal 128 Q is exact, the product with s * 2^100 is rounded once in the FMA
 #pragma unroll
-                for (int j = 0; j < 32; ++j)
-                    acc[j] = fmaf(sf, __uint_as_float(v[j] + 0x4B400000u) - 12582912.0f, acc[j]);
+                for (int j = 0; j < 32; ++j) acc[j] = fmaf(sf, __uint_as_float(v[j]) - qb, acc[j]);
             }
             tc_fence_before_sync();
             __syncwarp();
@@ -437,7 +470,7 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
             for (int j = 0; j < 32; ++j) {
                 const int m = m0 + part * 32 + j;
                 if (m < p.M && n < p.N) {
-                    const float val = __ldg(p.a_scale + m) * (acc[j] - __uint_as_float(v[j]));
+                    const float val = __ldg(p.a_scale + m) * (acc[j] * 0x1p49f - __uint_as_float(v[j]));
                     store_y(p.y, p.y_dtype, (size_t)m * p.N + n, val);
                 }
             }

@@ -44,10 +44,27 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity, ui
 }
 // Bounded wait: returns false when the phase did not complete within `max_polls` tries of up to
 // 20 microseconds each.
+__device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
 __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, uint32_t max_polls) {
+#ifdef MNNLLM_SPIN_WAIT
+    for (uint32_t i = 0; i < max_polls * 64u; ++i)
+        if (mbar_test_wait(bar, parity)) return true;
+    return false;
+#else
     for (uint32_t i = 0; i < max_polls; ++i)
         if (mbar_try_wait(bar, parity)) return true;
     return false;
+#endif
 }
 
 // ---- bulk asynchronous copy (TMA, untiled): global -> shared, completion on an mbarrier --------
