@@ -142,6 +142,20 @@ size_t mnnllm_workspace_size_w4a8(int M, int N, int K, int group);
 int mnnllm_linear_w4a8(const void* x, const void* packed, void* y, int M, int N, int K, int group,
                        int x_dtype, int y_dtype, void* workspace, size_t workspace_bytes, void* stream);
 
+/* Several weight matrices that multiply the SAME activations (q, k, v of a layer; gate and up) in
+ * one call: the activations are quantised once and one GEMM launch covers all the matrices
+ * (Section 4.2; the fusion itself is this library's).  All problems share M, K, group and x; the
+ * workspace is that of a single problem (mnnllm_workspace_size_w4a8 does not depend on N). */
+#define MNNLLM_MAX_BATCH_W4A8 4
+typedef struct {
+    const void* packed; /* device, from mnnllm_pack_w4 for [N, K], the call's group */
+    void* y;            /* device [M, N] of y_dtype, overwritten */
+    int N;
+    int y_dtype;
+} mnnllm_w4a8_problem;
+int mnnllm_linear_w4a8_batch(const mnnllm_w4a8_problem* problems, int count, const void* x, int M, int K, int group,
+                             int x_dtype, void* workspace, size_t workspace_bytes, void* stream);
+
 /* Same computation as mnnllm_linear_w4a8 for callers that cannot allocate device memory.  (The paper
  * has no counterpart; this is a convenience of this library.)  Some users of this code run where
  * cudaMalloc is off limits: inside a plugin whose host application owns every allocation, in a

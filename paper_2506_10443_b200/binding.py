@@ -37,6 +37,10 @@ class MnnllmError(RuntimeError):
         super().__init__("%s: %s (status %d)" % (where, lib.mnnllm_status_string(status).decode(), status))
 
 
+class _ProblemW4A8(_c.Structure):
+    _fields_ = [("packed", _P), ("y", _P), ("N", _c.c_int), ("y_dtype", _c.c_int)]
+
+
 class _Problem(_c.Structure):
     _fields_ = [("x", _P), ("packed", _P), ("y", _P), ("N", _c.c_int), ("K", _c.c_int), ("group", _c.c_int),
                 ("y_dtype", _c.c_int)]
@@ -65,6 +69,8 @@ _sig("mnnllm_linear_w8a16", _c.c_int, [_P, _P, _P, _c.c_int, _c.c_int, _c.c_int,
 _sig("mnnllm_workspace_size_w4a8", _c.c_size_t, [_c.c_int, _c.c_int, _c.c_int, _c.c_int])
 _sig("mnnllm_linear_w4a8", _c.c_int,
      [_P, _P, _P, _c.c_int, _c.c_int, _c.c_int, _c.c_int, _c.c_int, _c.c_int, _P, _c.c_size_t, _P])
+_sig("mnnllm_linear_w4a8_batch", _c.c_int,
+     [_c.POINTER(_ProblemW4A8), _c.c_int, _P, _c.c_int, _c.c_int, _c.c_int, _c.c_int, _P, _c.c_size_t, _P])
 _sig("mnnllm_linear_w4a8_static", _c.c_int,
      [_P, _P, _P, _c.c_int, _c.c_int, _c.c_int, _c.c_int, _c.c_int, _c.c_int, _P])
 _sig("mnnllm_quantize_activations", _c.c_int, [_P, _c.c_int, _c.c_int, _c.c_int, _c.c_int, _P, _P, _P, _P])
@@ -76,7 +82,7 @@ _sig("mnnllm_device_supported", _c.c_int, [])
 EXPORTS = [
     "mnnllm_status_string", "mnnllm_packed_size_w4", "mnnllm_pack_w4", "mnnllm_unpack_w4", "mnnllm_packed_info",
     "mnnllm_packed_size_w8", "mnnllm_pack_w8", "mnnllm_unpack_w8", "mnnllm_linear_w4a16", "mnnllm_linear_w4a16_ex",
-    "mnnllm_linear_w4a16_batch", "mnnllm_linear_w8a16", "mnnllm_workspace_size_w4a8", "mnnllm_linear_w4a8", "mnnllm_linear_w4a8_static",
+    "mnnllm_linear_w4a16_batch", "mnnllm_linear_w8a16", "mnnllm_workspace_size_w4a8", "mnnllm_linear_w4a8", "mnnllm_linear_w4a8_batch", "mnnllm_linear_w4a8_static",
     "mnnllm_quantize_activations", "mnnllm_debug_w4a8_partials", "mnnllm_read_status", "mnnllm_device_supported",
 ]
 
@@ -209,6 +215,21 @@ def linear_w4a8(x, packed, y, M, N, K, group, workspace, workspace_bytes, x_dtyp
                 stream=None) -> None:
     _check(lib.mnnllm_linear_w4a8(_ptr(x), _ptr(packed), _ptr(y), M, N, K, group, x_dtype, y_dtype, _ptr(workspace),
                                   workspace_bytes, _stream(stream)), "linear_w4a8")
+
+
+def make_batch_w4a8(problems: Sequence[dict]):
+    """Marshals dicts (packed, y, N, y_dtype) into the C array of ``linear_w4a8_batch``."""
+    arr = (_ProblemW4A8 * len(problems))()
+    for a, p in zip(arr, problems):
+        a.packed, a.y, a.N, a.y_dtype = _ptr(p["packed"]), _ptr(p["y"]), p["N"], p.get("y_dtype", F16)
+    return arr
+
+
+def linear_w4a8_batch(problems, x, M, K, group, workspace, workspace_bytes, x_dtype=F16, stream=None) -> None:
+    """Weight matrices that share the activations ``x``: one quantiser pass, one GEMM launch."""
+    arr = problems if isinstance(problems, _c.Array) else make_batch_w4a8(problems)
+    _check(lib.mnnllm_linear_w4a8_batch(arr, len(arr), _ptr(x), M, K, group, x_dtype, _ptr(workspace), workspace_bytes,
+                                        _stream(stream)), "linear_w4a8_batch")
 
 
 STATIC_SCRATCH_BYTES = 8 << 20

@@ -76,13 +76,17 @@ size_t mnnllm_workspace_size_w4a8(int M, int N, int K, int group) {
     return workspace_layout(M, K, group).total;
 }
 
-int mnnllm_linear_w4a8(const void* x, const void* packed, void* y, int M, int N, int K, int group, int x_dtype,
-                       int y_dtype, void* workspace, size_t workspace_bytes, void* stream) {
+int mnnllm_linear_w4a8_batch(const mnnllm_w4a8_problem* problems, int count, const void* x, int M, int K, int group,
+                             int x_dtype, void* workspace, size_t workspace_bytes, void* stream) {
     const int st = check_xq(x, x_dtype, M, K, group);
     if (st != MNNLLM_OK) return st;
-    if (!packed || !y || N < 1) return MNNLLM_ERR_INVALID_ARG;
-    if (y_dtype != MNNLLM_F16 && y_dtype != MNNLLM_BF16 && y_dtype != MNNLLM_F32) return MNNLLM_ERR_UNSUPPORTED;
-    if (((uintptr_t)y & 15) || ((uintptr_t)packed & 127)) return MNNLLM_ERR_ALIGNMENT;
+    if (!problems || count < 1 || count > MNNLLM_MAX_BATCH_W4A8) return MNNLLM_ERR_INVALID_ARG;
+    for (int i = 0; i < count; ++i) {
+        const mnnllm_w4a8_problem& q = problems[i];
+        if (!q.packed || !q.y || q.N < 1) return MNNLLM_ERR_INVALID_ARG;
+        if (q.y_dtype != MNNLLM_F16 && q.y_dtype != MNNLLM_BF16 && q.y_dtype != MNNLLM_F32) return MNNLLM_ERR_UNSUPPORTED;
+        if (((uintptr_t)q.y & 15) || ((uintptr_t)q.packed & 127)) return MNNLLM_ERR_ALIGNMENT;
+    }
     const Workspace w = workspace_layout(M, K, group);
     if (!workspace || workspace_bytes < w.total) return MNNLLM_ERR_WORKSPACE;
     if ((uintptr_t)workspace & 255) return MNNLLM_ERR_ALIGNMENT;
@@ -94,19 +98,31 @@ int mnnllm_linear_w4a8(const void* x, const void* packed, void* y, int M, int N,
     int8_t* a_q = (int8_t*)(ws + w.a_q);
     float* a_scale = (float*)(ws + w.a_scale);
     void* ac = ws + w.ac;
+    // the activations are quantised once for all the matrices of the batch
     if (act_quant_launch(x, x_dtype, M, K, group, a_q, a_scale, nullptr, ac, true, (cudaStream_t)stream) != cudaSuccess) {
         (void)cudaGetLastError();
         return MNNLLM_ERR_CUDA;
     }
     GemmW4A8Args a;
-    a.packed = packed; a.a_q = a_q; a.a_scale = a_scale; a.AC = ac; a.y = y; a.P = nullptr;
-    a.M = M; a.N = N; a.K = K; a.group = group; a.y_dtype = y_dtype;
+    a.count = count;
+    for (int i = 0; i < count; ++i) {
+        a.packed[i] = problems[i].packed; a.y[i] = problems[i].y; a.N[i] = problems[i].N; a.y_dtype[i] = problems[i].y_dtype;
+    }
+    a.a_q = a_q; a.a_scale = a_scale; a.AC = ac; a.P = nullptr;
+    a.M = M; a.K = K; a.group = group;
     const cudaError_t e = gemm_w4a8_launch(a, status, (cudaStream_t)stream);
     if (e != cudaSuccess) {
         (void)cudaGetLastError();
         return e == cudaErrorNotSupported ? MNNLLM_ERR_UNSUPPORTED : MNNLLM_ERR_CUDA;
     }
     return MNNLLM_OK;
+}
+
+int mnnllm_linear_w4a8(const void* x, const void* packed, void* y, int M, int N, int K, int group, int x_dtype,
+                       int y_dtype, void* workspace, size_t workspace_bytes, void* stream) {
+    mnnllm_w4a8_problem q;
+    q.packed = packed; q.y = y; q.N = N; q.y_dtype = y_dtype;
+    return mnnllm_linear_w4a8_batch(&q, 1, x, M, K, group, x_dtype, workspace, workspace_bytes, stream);
 }
 
 int mnnllm_debug_w4a8_partials(const void* x, int x_dtype, const void* packed, int32_t* P, int8_t* a_q, float* a_scale,
@@ -127,8 +143,10 @@ int mnnllm_debug_w4a8_partials(const void* x, int x_dtype, const void* packed, i
         return MNNLLM_ERR_CUDA;
     }
     GemmW4A8Args a;
-    a.packed = packed; a.a_q = a_q; a.a_scale = a_scale; a.AC = nullptr; a.y = nullptr; a.P = P;
-    a.M = M; a.N = N; a.K = K; a.group = group; a.y_dtype = MNNLLM_F32;
+    a.count = 1;
+    a.packed[0] = packed; a.y[0] = nullptr; a.N[0] = N; a.y_dtype[0] = MNNLLM_F32;
+    a.a_q = a_q; a.a_scale = a_scale; a.AC = nullptr; a.P = P;
+    a.M = M; a.K = K; a.group = group;
     const cudaError_t e = gemm_w4a8_launch(a, status, (cudaStream_t)stream);
     if (e != cudaSuccess) {
         (void)cudaGetLastError();

@@ -91,15 +91,21 @@ struct Smem {
 };
 constexpr size_t kSmemBytes = Smem::total + 1024;  // slack to align the base to 1024 bytes
 
-struct Params {
-    const uint8_t* packed;
-    const float* a_scale;
+struct Problem {
     void* y;
+    int N, n_row_blocks, y_dtype;
+    int tile_begin;   // first n-tile (blockIdx.x) of this weight matrix
+};
+struct Params {
+    const float* a_scale;
     int32_t* P;
-    int M, N, K, G;
-    int n_row_blocks, n_slabs, n_stages;
-    int y_dtype;
-    unsigned long long row_block_bytes, chunk_bytes;
+    int M, K, G;
+    int n_slabs, n_stages, count;
+    unsigned long long chunk_bytes;
+    Problem prob[kGemmMaxBatch];
+};
+struct WeightMaps {   // the packed bodies as 2-D tensors: codes box and table box per weight matrix
+    CUtensorMap pk[kGemmMaxBatch], tab[kGemmMaxBatch];
 };
 
 // K-major operand tile whose rows are 128 bytes, 128B swizzle: 8-row groups are 1024 bytes apart.
@@ -125,8 +131,8 @@ __device__ __forceinline__ void store_y(void* y, int dtype, size_t idx, float v)
 template <int GROUP, bool PARTIALS>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ CUtensorMap tm_ac,
-                 const __grid_constant__ CUtensorMap tm_pk, const __grid_constant__ CUtensorMap tm_tab,
-                 const __grid_constant__ Params p, uint32_t* __restrict__ status) {
+                 const __grid_constant__ WeightMaps wmaps, const __grid_constant__ Params p,
+                 uint32_t* __restrict__ status) {
     constexpr int GPS = kStageK / GROUP;  // groups per stage (2 or 1)
     constexpr int SPB = 4 / GPS;          // stages per block of four groups (zero-point MMA cadence)
     extern __shared__ uint8_t smem_raw[];
@@ -149,7 +155,12 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
     uint32_t* qsum_ring = reinterpret_cast<uint32_t*>(smem + Smem::qsum);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int n0 = blockIdx.x * kTileN, m0 = blockIdx.y * kTileT;
+    int pi = 0;
+    while (pi + 1 < p.count && (int)blockIdx.x >= p.prob[pi + 1].tile_begin) ++pi;
+    const Problem& q = p.prob[pi];
+    const CUtensorMap& tm_pk = wmaps.pk[pi];
+    const CUtensorMap& tm_tab = wmaps.tab[pi];
+    const int n0 = ((int)blockIdx.x - q.tile_begin) * kTileN, m0 = blockIdx.y * kTileT;
     const int n_stages = p.n_stages, G = p.G;
 
     if (threadIdx.x == 0) {
@@ -282,7 +293,7 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
     } else if (warp < kDrainWarp0) {
         // ------------------------------------------------------------------ unpack
         const int wu = warp - kUnpackWarp0;
-        const int nrb = (p.n_row_blocks - n0 / kRowsPerBlock) < 8 ? (p.n_row_blocks - n0 / kRowsPerBlock) : 8;
+        const int nrb = (q.n_row_blocks - n0 / kRowsPerBlock) < 8 ? (q.n_row_blocks - n0 / kRowsPerBlock) : 8;
         for (int st = 0; st < n_stages; ++st) {
             const int slot = st % kStages, round = st / kStages;
             const int pslot = st % kPkStages, j = st >> 2;
@@ -352,7 +363,7 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
         }
     } else if (warp == kScaleWarp) {
         // ------------------------------------------------------------------ scales and (s z) halves
-        const int nrb = (p.n_row_blocks - n0 / kRowsPerBlock) < 8 ? (p.n_row_blocks - n0 / kRowsPerBlock) : 8;
+        const int nrb = (q.n_row_blocks - n0 / kRowsPerBlock) < 8 ? (q.n_row_blocks - n0 / kRowsPerBlock) : 8;
         bool ok = true;
         for (int st = 0; st < n_stages && ok; ++st) {
             const int slot = st % kStages, round = st / kStages;
@@ -445,11 +456,11 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
             const uint32_t qb_bits = qsum_ring[(g % kScaleSlots) * kTileN + nl];   // 128 Q, also the float 128 Q 2^-149
             tmem_ld_wait();
             if (PARTIALS) {
-                if (n < p.N)
+                if (n < q.N)
 #pragma unroll
                     for (int j = 0; j < 32; ++j) {
                         const int m = m0 + part * 32 + j;
-                        if (m < p.M) p.P[((size_t)m * p.N + n) * G + g] = (int32_t)(v[j] - qb_bits);
+                        if (m < p.M) p.P[((size_t)m * q.N + n) * G + g] = (int32_t)(v[j] - qb_bits);
                     }
             } else {
                 // v is P_u >= 0 and below 2^23: its bits are the float P_u * 2^-149; the subtraction of
@@ -476,9 +487,9 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
                 const int m = m0 + part * 32 + j;
-                if (m < p.M && n < p.N) {
+                if (m < p.M && n < q.N) {
                     const float val = __ldg(p.a_scale + m) * (acc[j] * 0x1p49f - __uint_as_float(v[j]));
-                    store_y(p.y, p.y_dtype, (size_t)m * p.N + n, val);
+                    store_y(q.y, q.y_dtype, (size_t)m * q.N + n, val);
                 }
             }
         }
@@ -511,8 +522,8 @@ EncodeTiledFn encode_fn() {
 }
 
 template <int GROUP, bool PARTIALS>
-cudaError_t launch(const CUtensorMap& tm_act, const CUtensorMap& tm_ac, const CUtensorMap& tm_pk,
-                   const CUtensorMap& tm_tab, const Params& p, dim3 grid, uint32_t* status, cudaStream_t stream) {
+cudaError_t launch(const CUtensorMap& tm_act, const CUtensorMap& tm_ac, const WeightMaps& wmaps, const Params& p,
+                   dim3 grid, uint32_t* status, cudaStream_t stream) {
     static bool configured = false;
     auto kern = gemm_w4a8_kernel<GROUP, PARTIALS>;
     if (!configured) {
@@ -520,7 +531,7 @@ cudaError_t launch(const CUtensorMap& tm_act, const CUtensorMap& tm_ac, const CU
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    kern<<<grid, kThreads, kSmemBytes, stream>>>(tm_act, tm_ac, tm_pk, tm_tab, p, status);
+    kern<<<grid, kThreads, kSmemBytes, stream>>>(tm_act, tm_ac, wmaps, p, status);
     return cudaGetLastError();
 }
 
@@ -529,23 +540,44 @@ cudaError_t launch(const CUtensorMap& tm_act, const CUtensorMap& tm_ac, const CU
 cudaError_t gemm_w4a8_launch(const GemmW4A8Args& a, uint32_t* status, cudaStream_t stream) {
     EncodeTiledFn enc = encode_fn();
     if (!enc) return cudaErrorNotSupported;
-    const W4Geometry geo = w4_geometry(a.N, a.K, a.group);
+    if (a.count < 1 || a.count > kGemmMaxBatch) return cudaErrorInvalidValue;
     const bool partials = a.P != nullptr;
+    const W4Geometry geo0 = w4_geometry(a.N[0], a.K, a.group);
 
-    CUtensorMap tm_act, tm_ac, tm_pk, tm_tab;
-    {   // the packed body as [row block][32-bit words]: codes box 8 x 1 KiB, table box 8 x 512 B
+    CUtensorMap tm_act, tm_ac;
+    WeightMaps wmaps;
+    Params p;
+    p.a_scale = a.a_scale;
+    p.P = a.P;
+    p.M = a.M; p.K = a.K; p.G = geo0.G;
+    p.n_slabs = geo0.n_slabs;
+    p.n_stages = (a.K + kStageK - 1) / kStageK;
+    p.count = a.count;
+    p.chunk_bytes = geo0.chunk_bytes;
+    int tiles = 0;
+    for (int i = 0; i < kGemmMaxBatch; ++i) {
+        const int src = i < a.count ? i : 0;   // unused slots repeat the first matrix
+        const W4Geometry geo = w4_geometry(a.N[src], a.K, a.group);
+        // the packed body as [row block][32-bit words]: codes box 8 x 1 KiB, table box 8 x 512 B
         const cuuint64_t dims[2] = {(cuuint64_t)(geo.row_block_bytes / 4), (cuuint64_t)geo.n_row_blocks};
         const cuuint64_t strides[1] = {(cuuint64_t)geo.row_block_bytes};
         const cuuint32_t box_pk[2] = {2 * kSlabBytes / 4, 8}, box_tab[2] = {512 / 4, 8};
         const cuuint32_t estr[2] = {1, 1};
-        void* body = (void*)((const uint8_t*)a.packed + kHeaderBytes);
-        if (enc(&tm_pk, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, body, dims, strides, box_pk, estr,
+        void* body = (void*)((const uint8_t*)a.packed[src] + kHeaderBytes);
+        if (enc(&wmaps.pk[i], CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, body, dims, strides, box_pk, estr,
                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS ||
-            enc(&tm_tab, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, body, dims, strides, box_tab, estr,
+            enc(&wmaps.tab[i], CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, body, dims, strides, box_tab, estr,
                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return cudaErrorInvalidValue;
+        Problem& q = p.prob[i];
+        q.y = a.y[src];
+        q.N = a.N[src];
+        q.n_row_blocks = geo.n_row_blocks;
+        q.y_dtype = a.y_dtype[src];
+        q.tile_begin = tiles;
+        if (i < a.count) tiles += (a.N[i] + kTileN - 1) / kTileN;
     }
     {
         const cuuint64_t dims[2] = {(cuuint64_t)a.K, (cuuint64_t)a.M};
@@ -558,7 +590,7 @@ cudaError_t gemm_w4a8_launch(const GemmW4A8Args& a, uint32_t* status, cudaStream
             return cudaErrorInvalidValue;
     }
     if (!partials) {
-        const int G4 = (geo.G + 3) / 4 * 4;
+        const int G4 = (geo0.G + 3) / 4 * 4;
         const cuuint64_t dims[2] = {(cuuint64_t)G4 * 4, (cuuint64_t)a.M};
         const cuuint64_t strides[1] = {(cuuint64_t)G4 * 8};
         const cuuint32_t box[2] = {16, (cuuint32_t)kTileT};
@@ -570,23 +602,12 @@ cudaError_t gemm_w4a8_launch(const GemmW4A8Args& a, uint32_t* status, cudaStream
     } else {
         tm_ac = tm_act;  // never read in the partials form
     }
-
-    Params p;
-    p.packed = (const uint8_t*)a.packed;
-    p.a_scale = a.a_scale;
-    p.y = a.y;
-    p.P = a.P;
-    p.M = a.M; p.N = a.N; p.K = a.K; p.G = geo.G;
-    p.n_row_blocks = geo.n_row_blocks; p.n_slabs = geo.n_slabs;
-    p.n_stages = (a.K + kStageK - 1) / kStageK;
-    p.y_dtype = a.y_dtype;
-    p.row_block_bytes = geo.row_block_bytes; p.chunk_bytes = geo.chunk_bytes;
-    const dim3 grid((unsigned)((a.N + kTileN - 1) / kTileN), (unsigned)((a.M + kTileT - 1) / kTileT));
+    const dim3 grid((unsigned)tiles, (unsigned)((a.M + kTileT - 1) / kTileT));
     if (a.group == 64)
-        return partials ? launch<64, true>(tm_act, tm_ac, tm_pk, tm_tab, p, grid, status, stream)
-                        : launch<64, false>(tm_act, tm_ac, tm_pk, tm_tab, p, grid, status, stream);
-    return partials ? launch<128, true>(tm_act, tm_ac, tm_pk, tm_tab, p, grid, status, stream)
-                    : launch<128, false>(tm_act, tm_ac, tm_pk, tm_tab, p, grid, status, stream);
+        return partials ? launch<64, true>(tm_act, tm_ac, wmaps, p, grid, status, stream)
+                        : launch<64, false>(tm_act, tm_ac, wmaps, p, grid, status, stream);
+    return partials ? launch<128, true>(tm_act, tm_ac, wmaps, p, grid, status, stream)
+                    : launch<128, false>(tm_act, tm_ac, wmaps, p, grid, status, stream);
 }
 
 }  // namespace mnnllm

@@ -7,15 +7,21 @@
 
 namespace mnnllm {
 
+constexpr int kGemmMaxBatch = 4;
+
+// `count` weight matrices that multiply the same quantised activations (q, k, v of a layer; gate and
+// up): one launch, the n-tiles of all of them in one grid.
 struct GemmW4A8Args {
-    const void* packed;    // device, written by mnnllm_pack_w4
-    const int8_t* a_q;     // device int8 [M, K]
+    const void* packed[kGemmMaxBatch];  // device, written by mnnllm_pack_w4 (same K and group)
+    void* y[kGemmMaxBatch];             // device [M, N[i]] of y_dtype[i] (unused in the partials form)
+    int N[kGemmMaxBatch];
+    int y_dtype[kGemmMaxBatch];
+    int count;
+    const int8_t* a_q;     // device [M, K]: the codes a_q + 128 as unsigned bytes
     const float* a_scale;  // device fp32 [M]
     const void* AC;        // device fp16 quadruples [M, G4] x 8 bytes (null in the partials form)
-    void* y;               // device [M, N] of y_dtype (null in the partials form)
-    int32_t* P;            // device int32 [M, N, G] (partials form only)
-    int M, N, K, group;
-    int y_dtype;
+    int32_t* P;            // device int32 [M, N[0], G] (partials form only, count == 1)
+    int M, K, group;
 };
 
 // Enqueues the GEMM on `stream`.  With args.P set the kernel stores every int32 group partial and

@@ -123,15 +123,26 @@ class LinearStack:
     # ---- prefill ----
     @property
     def launches_per_step_w4a8(self) -> int:
-        return 2 * 7 * self.n_layers   # activation quantiser + GEMM per linear
+        return 2 * 4 * self.n_layers   # per layer: q+k+v, o, gate+up, down; quantiser + GEMM each
+
+    def _prefill_launches(self):
+        if getattr(self, "_pre", None) is None:
+            out = []
+            for l, L in enumerate(self.layers):
+                for names in (("q", "k", "v"), ("o",), ("gate", "up"), ("down",)):
+                    lins = [next(t for t in self.linears if t.name == n) for n in names]
+                    arr = B.make_batch_w4a8([dict(packed=L.packed[t.name], y=self.y_view(l, t.name), N=t.N, y_dtype=B.F16)
+                                             for t in lins])
+                    out.append((arr, self.x_view(l, names[0]), lins[0].K))
+            self._pre = out
+        return self._pre
 
     def run_w4a8(self, stream=None) -> None:
-        """One prefill step: every linear of every layer as quantise-activations + W4A8 GEMM."""
+        """One prefill step: per layer the matrices that share their input go in one call (one
+        quantiser pass, one GEMM launch): q+k+v, o, gate+up, down."""
         if self._workspace is None:
             need = max(B.workspace_size_w4a8(self.M, t.N, t.K, self.group) for t in self.linears)
             self._workspace = torch.empty(need, dtype=torch.uint8, device=self.device)
         ws, nbytes = self._workspace, self._workspace.numel()
-        for l, L in enumerate(self.layers):
-            for lin in self.linears:
-                B.linear_w4a8(self.x_view(l, lin.name), L.packed[lin.name], self.y_view(l, lin.name), self.M, lin.N,
-                              lin.K, self.group, ws, nbytes, stream=stream)
+        for arr, x, K in self._prefill_launches():
+            B.linear_w4a8_batch(arr, x, self.M, K, self.group, ws, nbytes, stream=stream)

@@ -99,6 +99,31 @@ def test_w4a8_unusual_zero_points():
     assert (y[7] == 0).all()
 
 
+def test_w4a8_batch_qkv_one_launch():
+    # three matrices on the same activations: one quantiser pass, one GEMM grid; ragged N on purpose
+    M, K, group = 200, 1536, 64
+    shapes = [1536, 256, 200]
+    x = inputs.activations(41, M, K, outliers=True)
+    xd = dev(x)
+    probs, refs, ys, keep = [], [], [], []
+    for i, N in enumerate(shapes):
+        W, packed, (q, s, z) = quantized(42 + i, N, K, group)
+        pd = dev(packed)
+        y = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
+        keep.append(pd)
+        probs.append(dict(packed=pd, y=y, N=N, y_dtype=B.F32))
+        refs.append(oracle.linear_w4a8(x.astype(np.float32), q, s, z, group))
+        ys.append(y)
+    nbytes = B.workspace_size_w4a8(M, max(shapes), K, group)
+    ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    B.linear_w4a8_batch(probs, xd, M, K, group, ws, nbytes)
+    assert B.read_status() == 0
+    for y, ref in zip(ys, refs):
+        assert_close(y.cpu().numpy(), ref)
+    assert B.lib.mnnllm_linear_w4a8_batch(B.make_batch_w4a8(probs), 5, xd.data_ptr(), M, K, group, B.F16, ws.data_ptr(),
+                                          nbytes, None) == 1
+
+
 def test_w4a8_deterministic():
     M, N, K, group = 200, 640, 1536, 64
     W, packed, _ = quantized(31, N, K, group)
