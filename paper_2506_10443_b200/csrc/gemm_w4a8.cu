@@ -185,6 +185,11 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    // Programmatic dependent launch: this grid may start while the activation quantiser still runs.
+    // Everything up to here and the whole weight side (packed codes, tables, unpack, scales) does
+    // not depend on it; the threads that read its outputs (activation codes and group sums through
+    // TMA, a_scale in the epilogue) call griddepcontrol.wait first.
+    pdl_launch_dependents();
 
     // a failed wait marks the CTA as aborted; every role then leaves its loop
     // (every lane polls: letting one lane poll and broadcasting its verdict was measured 2x slower)
@@ -224,6 +229,7 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
                 }
             }
             const int st = i - kPkLead;
+            if (st == 0) pdl_wait();   // the quantised activations are complete from here on
             if (st >= 0) {
                 const int slot = st % kStages, round = st / kStages;
                 if (!wait(&ab_empty[slot], (round & 1) ^ 1, 1)) break;
@@ -476,6 +482,7 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
             __syncwarp();
             if (lane == 0) mbar_arrive(&tm_empty[b]);
         }
+        pdl_wait();   // a_scale (long since written; the call makes the ordering explicit)
         if (!PARTIALS && ok && !*abort_flag && wait(corr_done, 0, 9)) {
             tc_fence_after_sync();
             uint32_t v[32];
@@ -531,8 +538,17 @@ cudaError_t launch(const CUtensorMap& tm_act, const CUtensorMap& tm_ac, const We
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    kern<<<grid, kThreads, kSmemBytes, stream>>>(tm_act, tm_ac, wmaps, p, status);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = kSmemBytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, tm_act, tm_ac, wmaps, p, status);
 }
 
 }  // namespace
