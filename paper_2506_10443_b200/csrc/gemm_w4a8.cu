@@ -82,9 +82,8 @@ struct Smem {
     static constexpr int cb = ca + 2 * kCorrBytes;
     static constexpr int pk = cb + 2 * kCorrBytes;
     static constexpr int tab = pk + kPkStages * kPkBytes;
-    static constexpr int scale = tab + kTabSlots * kTabBytes;
-    static constexpr int qsum = scale + kScaleSlots * kTileN * 4;   // 128 * Q per (group slot, row), as integers
-    static constexpr int bars = qsum + kScaleSlots * kTileN * 4;
+    static constexpr int scale = tab + kTabSlots * kTabBytes;        // per (group slot, row): {s * 2^100, 128 * Q}
+    static constexpr int bars = scale + kScaleSlots * kTileN * 8;
     static constexpr int n_bars = 2 * kStages + 2 * kAcc + 2 + 2 + 1 + 2 * kPkStages + 2 * kTabSlots;
     static constexpr int misc = bars + n_bars * 8;
     static constexpr int total = misc + 16;
@@ -151,8 +150,7 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
     uint64_t* tab_empty = tab_full + kTabSlots;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + Smem::misc);
     volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + Smem::misc + 4);
-    float* scale_ring = reinterpret_cast<float*>(smem + Smem::scale);
-    uint32_t* qsum_ring = reinterpret_cast<uint32_t*>(smem + Smem::qsum);
+    uint2* sq_ring = reinterpret_cast<uint2*>(smem + Smem::scale);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     int pi = 0;
@@ -204,7 +202,9 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
 
     if (warp == 0) {
         // ------------------------------------------------------------------ producer (TMA)
+        // one elected thread runs the whole loop: every step is a wait and a copy by a single thread
         const int rb0 = n0 / kRowsPerBlock;
+        if (elect_one())
         for (int i = 0; i < n_stages + kPkLead; ++i) {
             if (i < n_stages) {
                 // packed codes of stage i (and, at the start of a 512-k chunk, its scale/zero tables)
@@ -216,85 +216,73 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
                 if ((i & 3) == 0) {
                     const int tslot = j % kTabSlots;
                     if (!wait(&tab_empty[tslot], ((j / kTabSlots) & 1) ^ 1, 12)) break;
-                    if (elect_one()) {
-                        mbar_arrive_expect_tx(&tab_full[tslot], kTabBytes);
-                        tma_load_2d(smem + Smem::tab + tslot * kTabBytes, &tm_tab,
-                                    (int)((chunk_off + (unsigned long long)ns_chunk * kSlabBytes) >> 2), rb0, &tab_full[tslot]);
-                    }
+                    mbar_arrive_expect_tx(&tab_full[tslot], kTabBytes);
+                    tma_load_2d(smem + Smem::tab + tslot * kTabBytes, &tm_tab,
+                                (int)((chunk_off + (unsigned long long)ns_chunk * kSlabBytes) >> 2), rb0, &tab_full[tslot]);
                 }
-                if (elect_one()) {
-                    mbar_arrive_expect_tx(&pk_full[pslot], kPkBytes);
-                    tma_load_2d(smem + Smem::pk + pslot * kPkBytes, &tm_pk,
-                                (int)((chunk_off + (unsigned long long)(i & 3) * 2 * kSlabBytes) >> 2), rb0, &pk_full[pslot]);
-                }
+                mbar_arrive_expect_tx(&pk_full[pslot], kPkBytes);
+                tma_load_2d(smem + Smem::pk + pslot * kPkBytes, &tm_pk,
+                            (int)((chunk_off + (unsigned long long)(i & 3) * 2 * kSlabBytes) >> 2), rb0, &pk_full[pslot]);
             }
             const int st = i - kPkLead;
             if (st == 0) pdl_wait();   // the quantised activations are complete from here on
             if (st >= 0) {
                 const int slot = st % kStages, round = st / kStages;
                 if (!wait(&ab_empty[slot], (round & 1) ^ 1, 1)) break;
-                if (elect_one()) {
-                    mbar_arrive_expect_tx(&ab_full[slot], kTileT * kStageK);
-                    tma_load_2d(smem + Smem::aq + slot * kStageBytes, &tm_act, st * kStageK, m0, &ab_full[slot]);
-                }
+                mbar_arrive_expect_tx(&ab_full[slot], kTileT * kStageK);
+                tma_load_2d(smem + Smem::aq + slot * kStageBytes, &tm_act, st * kStageK, m0, &ab_full[slot]);
                 if (!PARTIALS && st % SPB == 0) {
                     const int cblk = st / SPB, cslot = cblk & 1;
                     if (!wait(&c_empty[cslot], ((cblk >> 1) & 1) ^ 1, 2)) break;
-                    if (elect_one()) {
-                        mbar_arrive_expect_tx(&c_full[cslot], kTileT * 32);
-                        tma_load_2d(smem + Smem::cb + cslot * kCorrBytes, &tm_ac, cblk * 16, m0, &c_full[cslot]);
-                    }
+                    mbar_arrive_expect_tx(&c_full[cslot], kTileT * 32);
+                    tma_load_2d(smem + Smem::cb + cslot * kCorrBytes, &tm_ac, cblk * 16, m0, &c_full[cslot]);
                 }
             }
-            __syncwarp();
         }
+        __syncwarp();
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issue
-        // Per stage: one wait for the operands, one for each accumulator, then a single elected
-        // region issues every MMA and commit of the stage back to back (the issue path is a serial
-        // chain of ~50-cycle steps; done once per stage instead of once per group it stays shorter
-        // than the drain).
-        int gcount = 0, ccount = 0;
-        const uint32_t wq_addr = smem_u32(smem + Smem::wq), aq_addr = smem_u32(smem + Smem::aq);
-        bool ok = true;
-        for (int st = 0; st < n_stages && ok; ++st) {
-            const int slot = st % kStages, round = st / kStages;
-            const int ngr = (G - st * GPS) < GPS ? (G - st * GPS) : GPS;
-            if (!wait(&ab_full[slot], round & 1, 3)) break;
-            for (int gi = 0; gi < ngr; ++gi)
-                if (!wait(&tm_empty[(gcount + gi) % kAcc], (((gcount + gi) / kAcc) & 1) ^ 1, 4)) { ok = false; break; }
-            if (!ok) break;
-            tc_fence_after_sync();
-            if (elect_one()) {
+        // One elected thread runs the whole loop (waits, MMAs and commits are single-thread
+        // operations; the issue path is a serial chain of ~50-cycle steps, so nothing is spent on
+        // re-electing or re-converging the warp per stage).  A group's MMAs are issued as soon as
+        // its own accumulator has been drained.
+        if (elect_one()) {
+            int gcount = 0, ccount = 0, b = 0;
+            uint32_t epar = 1;   // parity of the tm_empty phase that frees accumulator b
+            const uint32_t wq_addr = smem_u32(smem + Smem::wq), aq_addr = smem_u32(smem + Smem::aq);
+            bool ok = true;
+            for (int st = 0; st < n_stages && ok; ++st) {
+                const int slot = st % kStages, round = st / kStages;
+                const int ngr = (G - st * GPS) < GPS ? (G - st * GPS) : GPS;
+                if (!wait(&ab_full[slot], round & 1, 3)) break;
                 const uint64_t da = desc_sw128(wq_addr + slot * kStageBytes);
                 const uint64_t db = desc_sw128(aq_addr + slot * kStageBytes);
                 for (int gi = 0; gi < ngr; ++gi) {
-                    const int b = (gcount + gi) % kAcc;
+                    if (!wait(&tm_empty[b], epar, 4)) { ok = false; break; }
+                    tc_fence_after_sync();
 #pragma unroll
                     for (int kk = 0; kk < GROUP / 32; ++kk) {
                         const uint64_t adv = (uint64_t)((gi * GROUP + kk * 32) >> 4);
                         mma_i8_ss(tmem_base + b * kTileT, da + adv, db + adv, kIdescI8, kk > 0);
                     }
                     mma_commit(&tm_full[b]);
+                    if (++b == kAcc) { b = 0; epar ^= 1u; }
                 }
+                if (!ok) break;
                 mma_commit(&ab_empty[slot]);
-            }
-            __syncwarp();
-            gcount += ngr;
-            if (!PARTIALS && ((gcount & 3) == 0 || st == n_stages - 1)) {
-                const int cslot = ccount & 1;
-                if (!wait(&c_full[cslot], (ccount >> 1) & 1, 5)) break;
-                tc_fence_after_sync();
-                if (elect_one()) {
+                gcount += ngr;
+                if (!PARTIALS && ((gcount & 3) == 0 || st == n_stages - 1)) {
+                    const int cslot = ccount & 1;
+                    if (!wait(&c_full[cslot], (ccount >> 1) & 1, 5)) break;
+                    tc_fence_after_sync();
                     mma_f16_ss(tmem_base + kColCorr, desc_sw32(smem_u32(smem + Smem::ca + cslot * kCorrBytes)),
                                desc_sw32(smem_u32(smem + Smem::cb + cslot * kCorrBytes)), kIdescF16, ccount > 0);
                     mma_commit(&c_empty[cslot]);
+                    ++ccount;
                 }
-                __syncwarp();
-                ++ccount;
             }
+            if (!PARTIALS) mma_commit(corr_done);
         }
-        if (!PARTIALS && elect_one()) mma_commit(corr_done);
         __syncwarp();
     } else if (warp < kDrainWarp0) {
         // ------------------------------------------------------------------ unpack
@@ -306,12 +294,16 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
             const int ns_chunk = (p.n_slabs - 8 * j) < 8 ? (p.n_slabs - 8 * j) : 8;
             if (!wait(&pk_full[pslot], (st / kPkStages) & 1, 11)) break;
             // this thread's four 16-byte entries of the stage (zero where the tile or K runs out)
+            // Lanes of odd rows take the two slabs of a row block in the other order: the 16-byte
+            // stores of rows 2p and 2p + 1 (one shared-memory wavefront) then fall into different
+            // halves of the 128-byte swizzle row instead of colliding two-way.
+            const int odd = (lane >> 2) & 1;
             uint4 cur[4];
             {
                 const uint4* pk = reinterpret_cast<const uint4*>(smem + Smem::pk + pslot * kPkBytes);
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
-                    const int sidx = wu * 4 + i;   // row blocks 2 wu and 2 wu + 1, both slabs of each
+                    const int sidx = wu * 4 + (i ^ odd);   // row blocks 2 wu and 2 wu + 1, both slabs of each
                     const bool valid = (sidx >> 1) < nrb && (st & 3) * 2 + (sidx & 1) < ns_chunk;
                     cur[i] = valid ? pk[sidx * 32 + lane] : make_uint4(0, 0, 0, 0);
                 }
@@ -342,7 +334,7 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
             const int r = lane >> 2, c = lane & 3;
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                const int sidx = wu * 4 + i;
+                const int sidx = wu * 4 + (i ^ odd);
                 const int R0 = (sidx >> 1) * 16 + r;          // rows R0 and R0 + 8 of the tile
                 const int kc = (sidx & 1) * 4 + c;            // 16-byte chunk of the 128-byte row
                 const uint32_t off = (uint32_t)(R0 >> 3) * 1024u + (uint32_t)r * 128u + (uint32_t)((kc ^ r) << 4);
@@ -353,13 +345,13 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
             if (c == 0) {
 #pragma unroll
                 for (int i = 0; i < 4; i += (GROUP == 64 ? 1 : 2)) {
-                    const int g = GROUP == 64 ? st * 2 + (i & 1) : st;
+                    const int g = GROUP == 64 ? st * 2 + ((i ^ odd) & 1) : st;
                     if (g < G) {
                         const int R0 = (wu * 2 + (i >> 1)) * 16 + r;
                         const uint32_t s0 = GROUP == 64 ? q0[i] : q0[i] + q0[i + 1];
                         const uint32_t s1 = GROUP == 64 ? q1[i] : q1[i] + q1[i + 1];
-                        qsum_ring[(g % kScaleSlots) * kTileN + R0] = 128u * s0;
-                        qsum_ring[(g % kScaleSlots) * kTileN + R0 + 8] = 128u * s1;
+                        sq_ring[(g % kScaleSlots) * kTileN + R0].y = 128u * s0;
+                        sq_ring[(g % kScaleSlots) * kTileN + R0 + 8].y = 128u * s1;
                     }
                 }
             }
@@ -437,7 +429,7 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
                 if (g >= G) break;
 #pragma unroll
                 for (int i = 0; i < 4; ++i)   // s * 2^100 (the drain's operand is the denormal P * 2^-149)
-                    scale_ring[(g % kScaleSlots) * kTileN + lane + 32 * i] = __fmul_rn(sreg[i][gi], 0x1p100f);
+                    sq_ring[(g % kScaleSlots) * kTileN + lane + 32 * i].x = __float_as_uint(__fmul_rn(sreg[i][gi], 0x1p100f));
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(&ab_full[slot]);
@@ -452,14 +444,24 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
 #pragma unroll
         for (int i = 0; i < 16; ++i) acc2[i] = 0ull;
         bool ok = true;
+        // The loop is a chain of latencies, so everything that can be started early is: ring
+        // positions are counters (no divisions), the group's scale and 128 Q come in one load, and
+        // the next group's barrier is probed (non-blocking) while this group's partials are in
+        // flight, so that the usual case enters the next iteration without waiting at all.
+        int b = 0, ss = 0;
+        uint32_t par = 0;
+        bool ready = false;
         for (int g = 0; g < G; ++g) {
-            const int b = g % kAcc;
-            if (!wait(&tm_full[b], (g / kAcc) & 1, 8)) { ok = false; break; }
+            if (!ready && !wait(&tm_full[b], par, 8)) { ok = false; break; }
             tc_fence_after_sync();
             uint32_t v[32];
             tmem_ld_x32(lane_base + b * kTileT, v);
-            const float sf = scale_ring[(g % kScaleSlots) * kTileN + nl];
-            const uint32_t qb_bits = qsum_ring[(g % kScaleSlots) * kTileN + nl];   // 128 Q, also the float 128 Q 2^-149
+            const uint2 sq = sq_ring[ss * kTileN + nl];
+            const float sf = __uint_as_float(sq.x);
+            const uint32_t qb_bits = sq.y;   // 128 Q, also the float 128 Q 2^-149
+            const int bn = (b + 1 == kAcc) ? 0 : b + 1;
+            const uint32_t parn = par ^ (bn == 0 ? 1u : 0u);
+            ready = __all_sync(0xffffffffu, mbar_test_wait(&tm_full[bn], parn));
             tmem_ld_wait();
             if (PARTIALS) {
                 if (n < q.N)
@@ -481,6 +483,9 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(&tm_empty[b]);
+            b = bn;
+            par = parn;
+            ss = (ss + 1 == kScaleSlots) ? 0 : ss + 1;
         }
         pdl_wait();   // a_scale (long since written; the call makes the ordering explicit)
         if (!PARTIALS && ok && !*abort_flag && wait(corr_done, 0, 9)) {
