@@ -84,7 +84,7 @@ struct Smem {
     static constexpr int tab = pk + kPkStages * kPkBytes;
     static constexpr int scale = tab + kTabSlots * kTabBytes;        // per (group slot, row): {s * 2^100, 128 * Q}
     static constexpr int bars = scale + kScaleSlots * kTileN * 8;
-    static constexpr int n_bars = 2 * kStages + 2 * kAcc + 2 + 2 + 1 + 2 * kPkStages + 2 * kTabSlots;
+    static constexpr int n_bars = 2 * kStages + 2 * kAcc + 2 + 2 + 2 + 2 * kPkStages + 2 * kTabSlots;
     static constexpr int misc = bars + n_bars * 8;
     static constexpr int total = misc + 16;
 };
@@ -93,13 +93,14 @@ constexpr size_t kSmemBytes = Smem::total + 1024;  // slack to align the base to
 struct Problem {
     void* y;
     int N, n_row_blocks, y_dtype;
-    int tile_begin;   // first n-tile (blockIdx.x) of this weight matrix
+    int tile_begin;   // first weight-row tile of this matrix among the launch's row tiles
 };
 struct Params {
     const float* a_scale;
     int32_t* P;
     int M, K, G;
     int n_slabs, n_stages, count;
+    int tiles_m, total_tiles;   // token tiles; all (weight tile, token tile) pairs of the launch
     unsigned long long chunk_bytes;
     Problem prob[kGemmMaxBatch];
 };
@@ -128,7 +129,7 @@ __device__ __forceinline__ void store_y(void* y, int dtype, size_t idx, float v)
 }
 
 template <int GROUP, bool PARTIALS>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreads, 1)   // 80 registers: 84 would not spill, but 23 warps x 84 do not fit the register file's allocation units
 gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ CUtensorMap tm_ac,
                  const __grid_constant__ WeightMaps wmaps, const __grid_constant__ Params p,
                  uint32_t* __restrict__ status) {
@@ -144,7 +145,8 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
     uint64_t* c_full = tm_empty + kAcc;
     uint64_t* c_empty = c_full + 2;
     uint64_t* corr_done = c_empty + 2;
-    uint64_t* pk_full = corr_done + 1;
+    uint64_t* corr_free = corr_done + 1;
+    uint64_t* pk_full = corr_free + 1;
     uint64_t* pk_empty = pk_full + kPkStages;
     uint64_t* tab_full = pk_empty + kPkStages;
     uint64_t* tab_empty = tab_full + kTabSlots;
@@ -153,26 +155,41 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
     uint2* sq_ring = reinterpret_cast<uint2*>(smem + Smem::scale);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    int pi = 0;
-    while (pi + 1 < p.count && (int)blockIdx.x >= p.prob[pi + 1].tile_begin) ++pi;
-    const Problem& q = p.prob[pi];
-    const CUtensorMap& tm_pk = wmaps.pk[pi];
-    const CUtensorMap& tm_tab = wmaps.tab[pi];
-    const int n0 = ((int)blockIdx.x - q.tile_begin) * kTileN, m0 = blockIdx.y * kTileT;
     const int n_stages = p.n_stages, G = p.G;
+    const int n_cblk = (G + 3) >> 2;   // blocks of four groups (one zero-point MMA each) per tile
+    const int total_tiles = p.total_tiles;
+
+    // The CTA is persistent: it works through the tiles blockIdx.x, blockIdx.x + gridDim.x, ...
+    // Every ring and barrier keeps running across tiles (slots and parities come from running
+    // counts), so the producer, unpack, scale and MMA roles start on the next tile while the
+    // drain warps are still in the epilogue of the current one.  The token tile index runs
+    // fastest: CTAs that work at the same time share their weight tile.
+    struct Tile { int pi, n0, m0; };
+    auto tile_of = [&](int t) {
+        Tile c;
+        const int tn = t / p.tiles_m;
+        c.m0 = (t - tn * p.tiles_m) * kTileT;
+        c.pi = 0;
+        while (c.pi + 1 < p.count && tn >= p.prob[c.pi + 1].tile_begin) ++c.pi;
+        c.n0 = (tn - p.prob[c.pi].tile_begin) * kTileN;
+        return c;
+    };
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < kStages; ++i) { mbar_init(&ab_full[i], 6); mbar_init(&ab_empty[i], 1); }
         for (int i = 0; i < kAcc; ++i) { mbar_init(&tm_full[i], 1); mbar_init(&tm_empty[i], kDrainWarps); }
         for (int i = 0; i < 2; ++i) { mbar_init(&c_full[i], 2); mbar_init(&c_empty[i], 1); }
         mbar_init(corr_done, 1);
+        mbar_init(corr_free, kDrainWarps);
         for (int i = 0; i < kPkStages; ++i) { mbar_init(&pk_full[i], 1); mbar_init(&pk_empty[i], 4); }
         for (int i = 0; i < kTabSlots; ++i) { mbar_init(&tab_full[i], 1); mbar_init(&tab_empty[i], 1); }
         *abort_flag = 0;
         fence_mbar_init();
         prefetch_tensormap(&tm_act);
-        prefetch_tensormap(&tm_pk);
-        prefetch_tensormap(&tm_tab);
+        for (int i = 0; i < p.count; ++i) {
+            prefetch_tensormap(&wmaps.pk[i]);
+            prefetch_tensormap(&wmaps.tab[i]);
+        }
         if (!PARTIALS) prefetch_tensormap(&tm_ac);
     }
     if (warp == 1) {
@@ -189,10 +206,10 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
     // TMA, a_scale in the epilogue) call griddepcontrol.wait first.
     pdl_launch_dependents();
 
-    // a failed wait marks the CTA as aborted; every role then leaves its loop
-    // (every lane polls: letting one lane poll and broadcasting its verdict was measured 2x slower)
+    // a failed wait marks the CTA as aborted; every role then leaves its loops
+    // (every lane polls: letting one lane poll and broadcasting its verdict was measured slower)
     auto wait = [&](uint64_t* bar, uint32_t parity, uint32_t code) -> bool {
-        if (mbar_wait_bounded(bar, parity, kMaxPolls)) return true;
+        if (mbar_wait_bounded_compact(bar, parity, kMaxPolls)) return true;
         if (*abort_flag == 0) {
             *abort_flag = 1;
             atomicOr(status, 0x200u | code);
@@ -202,40 +219,60 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
 
     if (warp == 0) {
         // ------------------------------------------------------------------ producer (TMA)
-        // one elected thread runs the whole loop: every step is a wait and a copy by a single thread
-        const int rb0 = n0 / kRowsPerBlock;
-        if (elect_one())
-        for (int i = 0; i < n_stages + kPkLead; ++i) {
-            if (i < n_stages) {
-                // packed codes of stage i (and, at the start of a 512-k chunk, its scale/zero tables)
-                const int pslot = i % kPkStages, j = i >> 2;
-                if (!wait(&pk_empty[pslot], ((i / kPkStages) & 1) ^ 1, 10)) break;
-                const int ns_chunk = (p.n_slabs - 8 * j) < 8 ? (p.n_slabs - 8 * j) : 8;
-                const unsigned long long chunk_off = (unsigned long long)j * p.chunk_bytes;
-                // boxes are counted in full even where they run past the tensor (zero fill)
-                if ((i & 3) == 0) {
-                    const int tslot = j % kTabSlots;
-                    if (!wait(&tab_empty[tslot], ((j / kTabSlots) & 1) ^ 1, 12)) break;
-                    mbar_arrive_expect_tx(&tab_full[tslot], kTabBytes);
-                    tma_load_2d(smem + Smem::tab + tslot * kTabBytes, &tm_tab,
-                                (int)((chunk_off + (unsigned long long)ns_chunk * kSlabBytes) >> 2), rb0, &tab_full[tslot]);
+        // One elected thread runs the whole loop: every step is a wait and a copy by one thread.
+        // Two cursors walk the same (tile, stage) sequence: the packed codes (with each 512-k
+        // chunk's scale/zero tables) run kPkLead stages ahead of the activations.
+        if (elect_one()) {
+            int t_pk = blockIdx.x, i_pk = 0, t_ac = blockIdx.x, st = 0, lead = 0;
+            uint32_t ip = 0, jc = 0, gs = 0, cb = 0;   // running counts: packed stages, chunks, stages, zero-point blocks
+            Tile cp = tile_of(t_pk), ca = cp;
+            bool first = true;
+            while (t_ac < total_tiles) {
+                if (t_pk < total_tiles) {
+                    const int pslot = ip % kPkStages, j = i_pk >> 2, rb0 = cp.n0 / kRowsPerBlock;
+                    if (!wait(&pk_empty[pslot], ((ip / kPkStages) & 1) ^ 1, 10)) break;
+                    const int ns_chunk = (p.n_slabs - 8 * j) < 8 ? (p.n_slabs - 8 * j) : 8;
+                    const unsigned long long chunk_off = (unsigned long long)j * p.chunk_bytes;
+                    // boxes are counted in full even where they run past the tensor (zero fill)
+                    if ((i_pk & 3) == 0) {
+                        const int tslot = jc % kTabSlots;
+                        if (!wait(&tab_empty[tslot], ((jc / kTabSlots) & 1) ^ 1, 12)) break;
+                        mbar_arrive_expect_tx(&tab_full[tslot], kTabBytes);
+                        tma_load_2d(smem + Smem::tab + tslot * kTabBytes, &wmaps.tab[cp.pi],
+                                    (int)((chunk_off + (unsigned long long)ns_chunk * kSlabBytes) >> 2), rb0, &tab_full[tslot]);
+                        ++jc;
+                    }
+                    mbar_arrive_expect_tx(&pk_full[pslot], kPkBytes);
+                    tma_load_2d(smem + Smem::pk + pslot * kPkBytes, &wmaps.pk[cp.pi],
+                                (int)((chunk_off + (unsigned long long)(i_pk & 3) * 2 * kSlabBytes) >> 2), rb0, &pk_full[pslot]);
+                    ++ip;
+                    ++lead;
+                    if (++i_pk == n_stages) {
+                        i_pk = 0;
+                        t_pk += gridDim.x;
+                        if (t_pk < total_tiles) cp = tile_of(t_pk);
+                    }
                 }
-                mbar_arrive_expect_tx(&pk_full[pslot], kPkBytes);
-                tma_load_2d(smem + Smem::pk + pslot * kPkBytes, &tm_pk,
-                            (int)((chunk_off + (unsigned long long)(i & 3) * 2 * kSlabBytes) >> 2), rb0, &pk_full[pslot]);
-            }
-            const int st = i - kPkLead;
-            if (st == 0) pdl_wait();   // the quantised activations are complete from here on
-            if (st >= 0) {
-                const int slot = st % kStages, round = st / kStages;
-                if (!wait(&ab_empty[slot], (round & 1) ^ 1, 1)) break;
-                mbar_arrive_expect_tx(&ab_full[slot], kTileT * kStageK);
-                tma_load_2d(smem + Smem::aq + slot * kStageBytes, &tm_act, st * kStageK, m0, &ab_full[slot]);
-                if (!PARTIALS && st % SPB == 0) {
-                    const int cblk = st / SPB, cslot = cblk & 1;
-                    if (!wait(&c_empty[cslot], ((cblk >> 1) & 1) ^ 1, 2)) break;
-                    mbar_arrive_expect_tx(&c_full[cslot], kTileT * 32);
-                    tma_load_2d(smem + Smem::cb + cslot * kCorrBytes, &tm_ac, cblk * 16, m0, &c_full[cslot]);
+                if (lead > kPkLead || t_pk >= total_tiles) {
+                    if (first) { pdl_wait(); first = false; }   // the quantised activations are complete from here on
+                    const int slot = gs % kStages;
+                    if (!wait(&ab_empty[slot], ((gs / kStages) & 1) ^ 1, 1)) break;
+                    mbar_arrive_expect_tx(&ab_full[slot], kTileT * kStageK);
+                    tma_load_2d(smem + Smem::aq + slot * kStageBytes, &tm_act, st * kStageK, ca.m0, &ab_full[slot]);
+                    if (!PARTIALS && st % SPB == 0) {
+                        const int cslot = cb & 1;
+                        if (!wait(&c_empty[cslot], ((cb >> 1) & 1) ^ 1, 2)) break;
+                        mbar_arrive_expect_tx(&c_full[cslot], kTileT * 32);
+                        tma_load_2d(smem + Smem::cb + cslot * kCorrBytes, &tm_ac, (st / SPB) * 16, ca.m0, &c_full[cslot]);
+                        ++cb;
+                    }
+                    ++gs;
+                    --lead;
+                    if (++st == n_stages) {
+                        st = 0;
+                        t_ac += gridDim.x;
+                        if (t_ac < total_tiles) ca = tile_of(t_ac);
+                    }
                 }
             }
         }
@@ -247,252 +284,297 @@ gemm_w4a8_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_consta
         // re-electing or re-converging the warp per stage).  A group's MMAs are issued as soon as
         // its own accumulator has been drained.
         if (elect_one()) {
-            int gcount = 0, ccount = 0, b = 0;
-            uint32_t epar = 1;   // parity of the tm_empty phase that frees accumulator b
+            int b = 0, it = 0;
+            uint32_t epar = 1;        // parity of the tm_empty phase that frees accumulator b
+            uint32_t gs = 0, cb = 0;  // running counts of stages and zero-point blocks
             const uint32_t wq_addr = smem_u32(smem + Smem::wq), aq_addr = smem_u32(smem + Smem::aq);
             bool ok = true;
-            for (int st = 0; st < n_stages && ok; ++st) {
-                const int slot = st % kStages, round = st / kStages;
-                const int ngr = (G - st * GPS) < GPS ? (G - st * GPS) : GPS;
-                if (!wait(&ab_full[slot], round & 1, 3)) break;
-                const uint64_t da = desc_sw128(wq_addr + slot * kStageBytes);
-                const uint64_t db = desc_sw128(aq_addr + slot * kStageBytes);
-                for (int gi = 0; gi < ngr; ++gi) {
-                    if (!wait(&tm_empty[b], epar, 4)) { ok = false; break; }
-                    tc_fence_after_sync();
+            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++it) {
+                int gcount = 0;
+                bool cfirst = true;
+                for (int st = 0; st < n_stages && ok; ++st, ++gs) {
+                    const int slot = gs % kStages;
+                    const int ngr = (G - st * GPS) < GPS ? (G - st * GPS) : GPS;
+                    if (!wait(&ab_full[slot], (gs / kStages) & 1, 3)) { ok = false; break; }
+                    const uint64_t da = desc_sw128(wq_addr + slot * kStageBytes);
+                    const uint64_t db = desc_sw128(aq_addr + slot * kStageBytes);
+                    for (int gi = 0; gi < ngr; ++gi) {
+                        if (!wait(&tm_empty[b], epar, 4)) { ok = false; break; }
+                        tc_fence_after_sync();
 #pragma unroll
-                    for (int kk = 0; kk < GROUP / 32; ++kk) {
-                        const uint64_t adv = (uint64_t)((gi * GROUP + kk * 32) >> 4);
-                        mma_i8_ss(tmem_base + b * kTileT, da + adv, db + adv, kIdescI8, kk > 0);
+                        for (int kk = 0; kk < GROUP / 32; ++kk) {
+                            const uint64_t adv = (uint64_t)((gi * GROUP + kk * 32) >> 4);
+                            mma_i8_ss(tmem_base + b * kTileT, da + adv, db + adv, kIdescI8, kk > 0);
+                        }
+                        mma_commit(&tm_full[b]);
+                        if (++b == kAcc) { b = 0; epar ^= 1u; }
                     }
-                    mma_commit(&tm_full[b]);
-                    if (++b == kAcc) { b = 0; epar ^= 1u; }
+                    if (!ok) break;
+                    mma_commit(&ab_empty[slot]);
+                    gcount += ngr;
+                    if (!PARTIALS && ((gcount & 3) == 0 || st == n_stages - 1)) {
+                        const int cslot = cb & 1;
+                        if (!wait(&c_full[cslot], (cb >> 1) & 1, 5)) { ok = false; break; }
+                        // the previous tile's zero-point term must have left tensor memory
+                        if (cfirst && it > 0 && !wait(corr_free, (it - 1) & 1, 15)) { ok = false; break; }
+                        tc_fence_after_sync();
+                        mma_f16_ss(tmem_base + kColCorr, desc_sw32(smem_u32(smem + Smem::ca + cslot * kCorrBytes)),
+                                   desc_sw32(smem_u32(smem + Smem::cb + cslot * kCorrBytes)), kIdescF16, !cfirst);
+                        mma_commit(&c_empty[cslot]);
+                        cfirst = false;
+                        ++cb;
+                    }
                 }
-                if (!ok) break;
-                mma_commit(&ab_empty[slot]);
-                gcount += ngr;
-                if (!PARTIALS && ((gcount & 3) == 0 || st == n_stages - 1)) {
-                    const int cslot = ccount & 1;
-                    if (!wait(&c_full[cslot], (ccount >> 1) & 1, 5)) break;
-                    tc_fence_after_sync();
-                    mma_f16_ss(tmem_base + kColCorr, desc_sw32(smem_u32(smem + Smem::ca + cslot * kCorrBytes)),
-                               desc_sw32(smem_u32(smem + Smem::cb + cslot * kCorrBytes)), kIdescF16, ccount > 0);
-                    mma_commit(&c_empty[cslot]);
-                    ++ccount;
-                }
+                if (!PARTIALS && ok) mma_commit(corr_done);
             }
-            if (!PARTIALS) mma_commit(corr_done);
         }
         __syncwarp();
     } else if (warp < kDrainWarp0) {
         // ------------------------------------------------------------------ unpack
         const int wu = warp - kUnpackWarp0;
-        const int nrb = (q.n_row_blocks - n0 / kRowsPerBlock) < 8 ? (q.n_row_blocks - n0 / kRowsPerBlock) : 8;
-        for (int st = 0; st < n_stages; ++st) {
-            const int slot = st % kStages, round = st / kStages;
-            const int pslot = st % kPkStages, j = st >> 2;
-            const int ns_chunk = (p.n_slabs - 8 * j) < 8 ? (p.n_slabs - 8 * j) : 8;
-            if (!wait(&pk_full[pslot], (st / kPkStages) & 1, 11)) break;
-            // this thread's four 16-byte entries of the stage (zero where the tile or K runs out)
-            // Lanes of odd rows take the two slabs of a row block in the other order: the 16-byte
-            // stores of rows 2p and 2p + 1 (one shared-memory wavefront) then fall into different
-            // halves of the 128-byte swizzle row instead of colliding two-way.
-            const int odd = (lane >> 2) & 1;
-            uint4 cur[4];
-            {
-                const uint4* pk = reinterpret_cast<const uint4*>(smem + Smem::pk + pslot * kPkBytes);
+        const int r = lane >> 2, c = lane & 3;
+        // Lanes of odd rows take the two slabs of a row block in the other order: the 16-byte
+        // stores of rows 2p and 2p + 1 (one shared-memory wavefront) then fall into different
+        // halves of the 128-byte swizzle row instead of colliding two-way.
+        const int odd = r & 1;
+        uint32_t ip = 0, gs = 0, gg = 0;   // running counts: packed stages, stages, groups (at the tile's start)
+        bool ok = true;
+        for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, gg += G) {
+            const Tile tc = tile_of(t);
+            const Problem& q = p.prob[tc.pi];
+            const int nrb = (q.n_row_blocks - tc.n0 / kRowsPerBlock) < 8 ? (q.n_row_blocks - tc.n0 / kRowsPerBlock) : 8;
+            for (int st = 0; st < n_stages; ++st, ++ip, ++gs) {
+                const int slot = gs % kStages, pslot = ip % kPkStages, j = st >> 2;
+                const int ns_chunk = (p.n_slabs - 8 * j) < 8 ? (p.n_slabs - 8 * j) : 8;
+                if (!wait(&pk_full[pslot], (ip / kPkStages) & 1, 11)) { ok = false; break; }
+                // this thread's four 16-byte entries of the stage (zero where the tile or K runs out)
+                uint4 cur[4];
+                {
+                    const uint4* pk = reinterpret_cast<const uint4*>(smem + Smem::pk + pslot * kPkBytes);
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int sidx = wu * 4 + (i ^ odd);   // row blocks 2 wu and 2 wu + 1, both slabs of each
-                    const bool valid = (sidx >> 1) < nrb && (st & 3) * 2 + (sidx & 1) < ns_chunk;
-                    cur[i] = valid ? pk[sidx * 32 + lane] : make_uint4(0, 0, 0, 0);
-                }
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&pk_empty[pslot]);
-            // codes -> int8 (registers) before the stage's slot is waited for; then only the stores
-            constexpr uint32_t M4 = 0x0F0F0F0Fu;
-            uint4 lo8[4], hi8[4];
-            uint32_t q0[4], q1[4];   // sums of the codes of rows R0 and R0 + 8 over the slab (after the lane reduction)
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const uint4 w = cur[i];
-                lo8[i] = make_uint4(w.x & M4, (w.x >> 4) & M4, w.y & M4, (w.y >> 4) & M4);   // row R0
-                hi8[i] = make_uint4(w.z & M4, (w.z >> 4) & M4, w.w & M4, (w.w >> 4) & M4);   // row R0 + 8
-                uint32_t a = __dp4a(lo8[i].x, 0x01010101u, 0u), b = __dp4a(hi8[i].x, 0x01010101u, 0u);
-                a = __dp4a(lo8[i].y, 0x01010101u, a); b = __dp4a(hi8[i].y, 0x01010101u, b);
-                a = __dp4a(lo8[i].z, 0x01010101u, a); b = __dp4a(hi8[i].z, 0x01010101u, b);
-                a = __dp4a(lo8[i].w, 0x01010101u, a); b = __dp4a(hi8[i].w, 0x01010101u, b);
-                // the four lanes 4r .. 4r+3 hold the four 16-k pieces of the same rows
-                a += __shfl_xor_sync(0xffffffffu, a, 1); b += __shfl_xor_sync(0xffffffffu, b, 1);
-                a += __shfl_xor_sync(0xffffffffu, a, 2); b += __shfl_xor_sync(0xffffffffu, b, 2);
-                q0[i] = a; q1[i] = b;
-            }
-            if (!wait(&ab_empty[slot], (round & 1) ^ 1, 6)) break;
-            // 128B-swizzled K-major rows
-            uint8_t* wq = smem + Smem::wq + slot * kStageBytes;
-            const int r = lane >> 2, c = lane & 3;
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int sidx = wu * 4 + (i ^ odd);
-                const int R0 = (sidx >> 1) * 16 + r;          // rows R0 and R0 + 8 of the tile
-                const int kc = (sidx & 1) * 4 + c;            // 16-byte chunk of the 128-byte row
-                const uint32_t off = (uint32_t)(R0 >> 3) * 1024u + (uint32_t)r * 128u + (uint32_t)((kc ^ r) << 4);
-                *reinterpret_cast<uint4*>(wq + off) = lo8[i];
-                *reinterpret_cast<uint4*>(wq + off + 1024u) = hi8[i];
-            }
-            // 128 * Q per (row, group) for the drain: a slab is a group of 64, two slabs a group of 128
-            if (c == 0) {
-#pragma unroll
-                for (int i = 0; i < 4; i += (GROUP == 64 ? 1 : 2)) {
-                    const int g = GROUP == 64 ? st * 2 + ((i ^ odd) & 1) : st;
-                    if (g < G) {
-                        const int R0 = (wu * 2 + (i >> 1)) * 16 + r;
-                        const uint32_t s0 = GROUP == 64 ? q0[i] : q0[i] + q0[i + 1];
-                        const uint32_t s1 = GROUP == 64 ? q1[i] : q1[i] + q1[i + 1];
-                        sq_ring[(g % kScaleSlots) * kTileN + R0].y = 128u * s0;
-                        sq_ring[(g % kScaleSlots) * kTileN + R0 + 8].y = 128u * s1;
+                    for (int i = 0; i < 4; ++i) {
+                        const int sidx = wu * 4 + (i ^ odd);   // row blocks 2 wu and 2 wu + 1, both slabs of each
+                        const bool valid = (sidx >> 1) < nrb && (st & 3) * 2 + (sidx & 1) < ns_chunk;
+                        cur[i] = valid ? pk[sidx * 32 + lane] : make_uint4(0, 0, 0, 0);
                     }
                 }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&pk_empty[pslot]);
+                // codes -> int8 (registers) before the stage's slot is waited for; then only the stores
+                // (doing the conversion after the wait instead was measured 8 % slower end to end)
+                constexpr uint32_t M4 = 0x0F0F0F0Fu;
+                uint4 lo8[4], hi8[4];
+                uint32_t q0[4], q1[4];   // sums of the codes of rows R0 and R0 + 8 over the slab (after the lane reduction)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const uint4 w = cur[i];
+                    lo8[i] = make_uint4(w.x & M4, (w.x >> 4) & M4, w.y & M4, (w.y >> 4) & M4);   // row R0
+                    hi8[i] = make_uint4(w.z & M4, (w.z >> 4) & M4, w.w & M4, (w.w >> 4) & M4);   // row R0 + 8
+                    uint32_t a = __dp4a(lo8[i].x, 0x01010101u, 0u), b = __dp4a(hi8[i].x, 0x01010101u, 0u);
+                    a = __dp4a(lo8[i].y, 0x01010101u, a); b = __dp4a(hi8[i].y, 0x01010101u, b);
+                    a = __dp4a(lo8[i].z, 0x01010101u, a); b = __dp4a(hi8[i].z, 0x01010101u, b);
+                    a = __dp4a(lo8[i].w, 0x01010101u, a); b = __dp4a(hi8[i].w, 0x01010101u, b);
+                    // the four lanes 4r .. 4r+3 hold the four 16-k pieces of the same rows
+                    a += __shfl_xor_sync(0xffffffffu, a, 1); b += __shfl_xor_sync(0xffffffffu, b, 1);
+                    a += __shfl_xor_sync(0xffffffffu, a, 2); b += __shfl_xor_sync(0xffffffffu, b, 2);
+                    q0[i] = a; q1[i] = b;
+                }
+                if (!wait(&ab_empty[slot], ((gs / kStages) & 1) ^ 1, 6)) { ok = false; break; }
+                // 128B-swizzled K-major rows
+                uint8_t* wq = smem + Smem::wq + slot * kStageBytes;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int sidx = wu * 4 + (i ^ odd);
+                    const int R0 = (sidx >> 1) * 16 + r;          // rows R0 and R0 + 8 of the tile
+                    const int kc = (sidx & 1) * 4 + c;            // 16-byte chunk of the 128-byte row
+                    const uint32_t off = (uint32_t)(R0 >> 3) * 1024u + (uint32_t)r * 128u + (uint32_t)((kc ^ r) << 4);
+                    *reinterpret_cast<uint4*>(wq + off) = lo8[i];
+                    *reinterpret_cast<uint4*>(wq + off + 1024u) = hi8[i];
+                }
+                // 128 * Q per (row, group) for the drain: a slab is a group of 64, two slabs a group of 128
+                if (c == 0) {
+                    const uint32_t gslot0 = (gg + (uint32_t)st * GPS) % kScaleSlots;
+#pragma unroll
+                    for (int i = 0; i < 4; i += (GROUP == 64 ? 1 : 2)) {
+                        const int gl = GROUP == 64 ? ((i ^ odd) & 1) : 0;   // group of the stage
+                        if (st * GPS + gl < G) {
+                            const uint32_t gslot = (gslot0 + gl == kScaleSlots) ? 0u : gslot0 + gl;
+                            const int R0 = (wu * 2 + (i >> 1)) * 16 + r;
+                            const uint32_t s0 = GROUP == 64 ? q0[i] : q0[i] + q0[i + 1];
+                            const uint32_t s1 = GROUP == 64 ? q1[i] : q1[i] + q1[i + 1];
+                            sq_ring[gslot * kTileN + R0].y = 128u * s0;
+                            sq_ring[gslot * kTileN + R0 + 8].y = 128u * s1;
+                        }
+                    }
+                }
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&ab_full[slot]);
             }
-            fence_proxy_async_smem();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&ab_full[slot]);
         }
     } else if (warp == kScaleWarp) {
         // ------------------------------------------------------------------ scales and (s z) halves
-        const int nrb = (q.n_row_blocks - n0 / kRowsPerBlock) < 8 ? (q.n_row_blocks - n0 / kRowsPerBlock) : 8;
+        uint32_t gs = 0, jc = 0, gg = 0, cbase = 0;   // running counts: stages, chunks, groups and zero-point blocks (at the tile's start)
         bool ok = true;
-        for (int st = 0; st < n_stages && ok; ++st) {
-            const int slot = st % kStages, round = st / kStages;
-            const int j = st >> 2, tslot = j % kTabSlots;
-            const int ns_chunk = (p.n_slabs - 8 * j) < 8 ? (p.n_slabs - 8 * j) : 8;
-            const int ng = ns_chunk * kSlabK4 / GROUP;
-            if ((st & 3) == 0 && !wait(&tab_full[tslot], (j / kTabSlots) & 1, 13)) break;
-            // this lane's rows: lane, lane + 32, lane + 64, lane + 96
-            uint32_t zc[4][GPS];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int row = lane + 32 * i;
-                const uint32_t* tab = reinterpret_cast<const uint32_t*>(smem + Smem::tab + tslot * kTabBytes + (row >> 4) * 512);
-#pragma unroll
-                for (int gi = 0; gi < GPS; ++gi) {
-                    const int gc = (st & 3) * GPS + gi;
-                    zc[i][gi] = ((row >> 4) < nrb && gc < ng) ? tab[(row & 15) * ng + gc] : 0u;
+        for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, gg += G, cbase += n_cblk) {
+            const Tile tc = tile_of(t);
+            const Problem& q = p.prob[tc.pi];
+            const int nrb = (q.n_row_blocks - tc.n0 / kRowsPerBlock) < 8 ? (q.n_row_blocks - tc.n0 / kRowsPerBlock) : 8;
+            uint32_t tslot = 0;
+            for (int st = 0; st < n_stages && ok; ++st, ++gs) {
+                const int slot = gs % kStages;
+                const int j = st >> 2;
+                const int ns_chunk = (p.n_slabs - 8 * j) < 8 ? (p.n_slabs - 8 * j) : 8;
+                const int ng = ns_chunk * kSlabK4 / GROUP;
+                if ((st & 3) == 0) {
+                    tslot = jc % kTabSlots;
+                    if (!wait(&tab_full[tslot], (jc / kTabSlots) & 1, 13)) { ok = false; break; }
+                    ++jc;
                 }
-            }
-            if ((st & 3) == 3 || st == n_stages - 1) {  // the chunk's table has been read in full
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&tab_empty[tslot]);
-            }
-            // The conversion chains and the zero-point tile (which has its own flow control) come
-            // first; only the cheap publication of the scales waits for the stage's slot, so that
-            // this warp is never what the MMA waits for.
-            float sreg[4][GPS];
-#pragma unroll
-            for (int gi = 0; gi < GPS; ++gi) {
-                const int g = st * GPS + gi;
-                if (g >= G) break;
-                const int pos = g & 3, cblk = g >> 2, cslot = cblk & 1;
-                if (!PARTIALS && pos == 0 && !wait(&c_empty[cslot], ((cblk >> 1) & 1) ^ 1, 7)) { ok = false; break; }
+                // this lane's rows: lane, lane + 32, lane + 64, lane + 96
+                uint32_t zc[4][GPS];
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     const int row = lane + 32 * i;
-                    const __half2 h2 = *reinterpret_cast<const __half2*>(&zc[i][gi]);
-                    const float s = __low2float(h2), z = __high2float(h2);
-                    sreg[i][gi] = s;
-                    if (!PARTIALS) {
-                        const float szf = s * z;  // exact: 11-bit x 11-bit significands
-                        const __half hi = __float2half_rn(szf);
-                        const __half lo = __float2half_rn(szf - __half2float(hi));
-                        const uint32_t hh = (uint32_t)__half_as_ushort(hi) * 0x00010001u;
-                        const uint32_t ll = (uint32_t)__half_as_ushort(lo) * 0x00010001u;
-                        uint8_t* tile = smem + Smem::ca + cslot * kCorrBytes;
-                        const int rowoff = (row >> 3) * 256 + (row & 7) * 32, sw = (row & 7) >> 2;
-                        *reinterpret_cast<uint2*>(tile + rowoff + (((pos >> 1) ^ sw) << 4) + (pos & 1) * 8) = make_uint2(hh, ll);
-                        if (g == G - 1)
-                            for (int q = pos + 1; q < 4; ++q)
-                                *reinterpret_cast<uint2*>(tile + rowoff + (((q >> 1) ^ sw) << 4) + (q & 1) * 8) = make_uint2(0u, 0u);
+                    const uint32_t* tab = reinterpret_cast<const uint32_t*>(smem + Smem::tab + tslot * kTabBytes + (row >> 4) * 512);
+#pragma unroll
+                    for (int gi = 0; gi < GPS; ++gi) {
+                        const int gc = (st & 3) * GPS + gi;
+                        zc[i][gi] = ((row >> 4) < nrb && gc < ng) ? tab[(row & 15) * ng + gc] : 0u;
                     }
                 }
-                if (!PARTIALS && (pos == 3 || g == G - 1)) {
-                    fence_proxy_async_smem();
+                if ((st & 3) == 3 || st == n_stages - 1) {  // the chunk's table has been read in full
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(&c_full[cslot]);
+                    if (lane == 0) mbar_arrive(&tab_empty[tslot]);
                 }
-            }
-            if (!ok) break;
-            if (!wait(&ab_empty[slot], (round & 1) ^ 1, 14)) break;
+                // The conversion chains and the zero-point tile (which has its own flow control) come
+                // first; only the cheap publication of the scales waits for the stage's slot, so that
+                // this warp is never what the MMA waits for.
+                float sreg[4][GPS];
 #pragma unroll
-            for (int gi = 0; gi < GPS; ++gi) {
-                const int g = st * GPS + gi;
-                if (g >= G) break;
+                for (int gi = 0; gi < GPS; ++gi) {
+                    const int g = st * GPS + gi;
+                    if (g >= G) break;
+                    const int pos = g & 3;
+                    const uint32_t cb = cbase + (uint32_t)(g >> 2);
+                    const int cslot = cb & 1;
+                    if (!PARTIALS && pos == 0 && !wait(&c_empty[cslot], ((cb >> 1) & 1) ^ 1, 7)) { ok = false; break; }
 #pragma unroll
-                for (int i = 0; i < 4; ++i)   // s * 2^100 (the drain's operand is the denormal P * 2^-149)
-                    sq_ring[(g % kScaleSlots) * kTileN + lane + 32 * i].x = __float_as_uint(__fmul_rn(sreg[i][gi], 0x1p100f));
+                    for (int i = 0; i < 4; ++i) {
+                        const int row = lane + 32 * i;
+                        const __half2 h2 = *reinterpret_cast<const __half2*>(&zc[i][gi]);
+                        const float s = __low2float(h2), z = __high2float(h2);
+                        sreg[i][gi] = s;
+                        if (!PARTIALS) {
+                            const float szf = s * z;  // exact: 11-bit x 11-bit significands
+                            const __half hi = __float2half_rn(szf);
+                            const __half lo = __float2half_rn(szf - __half2float(hi));
+                            const uint32_t hh = (uint32_t)__half_as_ushort(hi) * 0x00010001u;
+                            const uint32_t ll = (uint32_t)__half_as_ushort(lo) * 0x00010001u;
+                            uint8_t* tile = smem + Smem::ca + cslot * kCorrBytes;
+                            const int rowoff = (row >> 3) * 256 + (row & 7) * 32, sw = (row & 7) >> 2;
+                            *reinterpret_cast<uint2*>(tile + rowoff + (((pos >> 1) ^ sw) << 4) + (pos & 1) * 8) = make_uint2(hh, ll);
+                            if (g == G - 1)
+                                for (int e = pos + 1; e < 4; ++e)
+                                    *reinterpret_cast<uint2*>(tile + rowoff + (((e >> 1) ^ sw) << 4) + (e & 1) * 8) = make_uint2(0u, 0u);
+                        }
+                    }
+                    if (!PARTIALS && (pos == 3 || g == G - 1)) {
+                        fence_proxy_async_smem();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&c_full[cslot]);
+                    }
+                }
+                if (!ok) break;
+                if (!wait(&ab_empty[slot], ((gs / kStages) & 1) ^ 1, 14)) { ok = false; break; }
+                const uint32_t gslot0 = (gg + (uint32_t)st * GPS) % kScaleSlots;
+#pragma unroll
+                for (int gi = 0; gi < GPS; ++gi) {
+                    if (st * GPS + gi >= G) break;
+                    const uint32_t gslot = (gslot0 + gi == kScaleSlots) ? 0u : gslot0 + gi;
+#pragma unroll
+                    for (int i = 0; i < 4; ++i)   // s * 2^100 (the drain's operand is the denormal P * 2^-149)
+                        sq_ring[gslot * kTileN + lane + 32 * i].x = __float_as_uint(__fmul_rn(sreg[i][gi], 0x1p100f));
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&ab_full[slot]);
             }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&ab_full[slot]);
         }
     } else {
         // ------------------------------------------------------------------ drain + epilogue
         const int q4 = warp & 3;                      // tensor-memory lane quarter this warp may read
         const int part = (warp - kDrainWarp0) >> 2;   // which 32 token columns
-        const int nl = q4 * 32 + lane, n = n0 + nl;
+        const int nl = q4 * 32 + lane;
         const uint32_t lane_base = tmem_base + ((uint32_t)(q4 * 32) << 16) + part * 32;
-        uint64_t acc2[16];   // 32 fp32 accumulators as packed pairs (columns 2j, 2j + 1)
-#pragma unroll
-        for (int i = 0; i < 16; ++i) acc2[i] = 0ull;
-        bool ok = true;
         // The loop is a chain of latencies, so everything that can be started early is: ring
         // positions are counters (no divisions), the group's scale and 128 Q come in one load, and
         // the next group's barrier is probed (non-blocking) while this group's partials are in
         // flight, so that the usual case enters the next iteration without waiting at all.
-        int b = 0, ss = 0;
-        uint32_t par = 0;
+        // One counter of groups modulo 12 gives the scale slot (ss), the accumulator (ss % 3) and the
+        // parity of its barrier ((ss / 3) & 1): 12 is a multiple of both rings' periods (3 and 6).
+        uint32_t ss = 0;
         bool ready = false;
-        for (int g = 0; g < G; ++g) {
-            if (!ready && !wait(&tm_full[b], par, 8)) { ok = false; break; }
-            tc_fence_after_sync();
-            uint32_t v[32];
-            tmem_ld_x32(lane_base + b * kTileT, v);
-            const uint2 sq = sq_ring[ss * kTileN + nl];
-            const float sf = __uint_as_float(sq.x);
-            const uint32_t qb_bits = sq.y;   // 128 Q, also the float 128 Q 2^-149
-            const int bn = (b + 1 == kAcc) ? 0 : b + 1;
-            const uint32_t parn = par ^ (bn == 0 ? 1u : 0u);
-            ready = __all_sync(0xffffffffu, mbar_test_wait(&tm_full[bn], parn));
-            tmem_ld_wait();
-            if (PARTIALS) {
-                if (n < q.N)
+        const uint2* sq_lane = sq_ring + nl;
+        for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) {
+            uint64_t acc2[16];   // 32 fp32 accumulators as packed pairs (columns 2j, 2j + 1)
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        const int m = m0 + part * 32 + j;
-                        if (m < p.M) p.P[((size_t)m * q.N + n) * G + g] = (int32_t)(v[j] - qb_bits);
-                    }
-            } else {
-                // v is P_u >= 0 and below 2^23: its bits are the float P_u * 2^-149; the subtraction of
-                // the denormal 128 Q is exact, the product with s * 2^100 is rounded once in the FMA
-                // (packed f32x2 arithmetic: 444 instead of 605 cycles per group in an isolated model)
-                const uint64_t sf2 = f32x2_pack(__float_as_uint(sf), __float_as_uint(sf));
-                const uint64_t qb2 = f32x2_pack(qb_bits, qb_bits);
+            for (int i = 0; i < 16; ++i) acc2[i] = 0ull;
+            bool ok = true;
+            for (int g = 0; g < G; ++g) {
+                const uint32_t b = (0x924924u >> (2 * ss)) & 3u;   // ss % 3
+                const uint32_t par = (0xE38u >> ss) & 1u;          // (ss / 3) & 1
+                if (!ready && !wait(&tm_full[b], par, 8)) { ok = false; break; }
+                tc_fence_after_sync();
+                uint32_t v[32];
+                tmem_ld_x32(lane_base + b * kTileT, v);
+                const uint2 sq = sq_lane[ss * kTileN];
+                const float sf = __uint_as_float(sq.x);
+                const uint32_t qb_bits = sq.y;   // 128 Q, also the float 128 Q 2^-149
+                const uint32_t sn = (ss + 1 == kScaleSlots) ? 0u : ss + 1;
+                ready = __all_sync(0xffffffffu, mbar_test_wait(&tm_full[(0x924924u >> (2 * sn)) & 3u], (0xE38u >> sn) & 1u));
+                tmem_ld_wait();
+                if (PARTIALS) {
+                    const Tile tc = tile_of(t);
+                    const Problem& q = p.prob[tc.pi];
+                    const int n = tc.n0 + nl, m0 = tc.m0;
+                    if (n < q.N)
 #pragma unroll
-                for (int j = 0; j < 16; ++j)
-                    acc2[j] = f32x2_fma(sf2, f32x2_sub(f32x2_pack(v[2 * j], v[2 * j + 1]), qb2), acc2[j]);
+                        for (int j = 0; j < 32; ++j) {
+                            const int m = m0 + part * 32 + j;
+                            if (m < p.M) p.P[((size_t)m * q.N + n) * G + g] = (int32_t)(v[j] - qb_bits);
+                        }
+                } else {
+                    // v is P_u >= 0 and below 2^23: its bits are the float P_u * 2^-149; the subtraction of
+                    // the denormal 128 Q is exact, the product with s * 2^100 is rounded once in the FMA
+                    // (packed f32x2 arithmetic: 444 instead of 605 cycles per group in an isolated model)
+                    const uint64_t sf2 = f32x2_pack(__float_as_uint(sf), __float_as_uint(sf));
+                    const uint64_t qb2 = f32x2_pack(qb_bits, qb_bits);
+#pragma unroll
+                    for (int j = 0; j < 16; ++j)
+                        acc2[j] = f32x2_fma(sf2, f32x2_sub(f32x2_pack(v[2 * j], v[2 * j + 1]), qb2), acc2[j]);
+                }
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&tm_empty[b]);
+                ss = sn;
             }
-            tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&tm_empty[b]);
-            b = bn;
-            par = parn;
-            ss = (ss + 1 == kScaleSlots) ? 0 : ss + 1;
-        }
-        pdl_wait();   // a_scale (long since written; the call makes the ordering explicit)
-        if (!PARTIALS && ok && !*abort_flag && wait(corr_done, 0, 9)) {
+            if (!ok) break;
+            if (PARTIALS) continue;
+            // the tile's coordinates are only needed from here on (not kept live through the loop)
+            const Tile tc = tile_of(t);
+            const Problem& q = p.prob[tc.pi];
+            const int n = tc.n0 + nl, m0 = tc.m0;
+            const int it = (t - (int)blockIdx.x) / (int)gridDim.x;
+            if (it == 0) pdl_wait();   // a_scale (long since written; the call makes the ordering explicit)
+            if (!wait(corr_done, it & 1, 9)) break;
             tc_fence_after_sync();
             uint32_t v[32];
             tmem_ld_x32(lane_base + kColCorr, v);
             tmem_ld_wait();
+            // the zero-point term is in registers: the next tile may overwrite its accumulator
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(corr_free);
             float acc[32];
 #pragma unroll
             for (int j = 0; j < 16; ++j) f32x2_unpack(acc2[j], acc[2 * j], acc[2 * j + 1]);
@@ -531,6 +613,19 @@ EncodeTiledFn encode_fn() {
             fn = (EncodeTiledFn)ptr;
     }
     return fn;
+}
+
+// SMs of the current device (one persistent CTA each), asked once per device.
+int sm_count() {
+    static int cached[64];
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+    if (!cached[dev]) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+        cached[dev] = n;
+    }
+    return cached[dev];
 }
 
 template <int GROUP, bool PARTIALS>
@@ -623,7 +718,11 @@ cudaError_t gemm_w4a8_launch(const GemmW4A8Args& a, uint32_t* status, cudaStream
     } else {
         tm_ac = tm_act;  // never read in the partials form
     }
-    const dim3 grid((unsigned)tiles, (unsigned)((a.M + kTileT - 1) / kTileT));
+    p.tiles_m = (a.M + kTileT - 1) / kTileT;
+    p.total_tiles = tiles * p.tiles_m;
+    const int n_sm = sm_count();
+    if (n_sm <= 0) return cudaErrorInvalidDevice;
+    const dim3 grid((unsigned)(p.total_tiles < n_sm ? p.total_tiles : n_sm));   // one persistent CTA per SM
     if (a.group == 64)
         return partials ? launch<64, true>(tm_act, tm_ac, wmaps, p, grid, status, stream)
                         : launch<64, false>(tm_act, tm_ac, wmaps, p, grid, status, stream);
