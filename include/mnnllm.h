@@ -134,18 +134,26 @@ int mnnllm_linear_w8a16(const void* x, const void* packed, void* y, int M, int N
  *
  *   x          device [M, K] of x_dtype (MNNLLM_F16 or MNNLLM_BF16)
  *   y          device [M, N] of y_dtype, overwritten
- *   workspace  device scratch of at least mnnllm_workspace_size_w4a8(M, N, K, group) bytes,
- *              256-byte aligned; holds a_q, a_scale, A between the two kernels.  Contents are
- *              undefined afterwards; two calls that may overlap on the GPU need separate workspaces.
+ *   workspace  device scratch, 256-byte aligned; holds a_q, a_scale, A between the two kernels.
+ *              mnnllm_workspace_size_w4a8(M, N, K, group) is the size to allocate.  It includes
+ *              about 20 MB in which a problem with fewer 128 x 128 output tiles than the GPU has
+ *              SMs is split along K (the parts of a tile are summed there in fp32, in a fixed
+ *              order: results do not depend on timing).  A workspace of at least
+ *              mnnllm_workspace_min_w4a8(M, N, K, group) bytes is accepted too: such problems
+ *              then keep some SMs idle; the results are the same up to the fp32 summation order.
+ *              Smaller: MNNLLM_ERR_WORKSPACE.  Contents are undefined afterwards; two calls that
+ *              may overlap on the GPU need separate workspaces.  Both sizes are 0 for arguments
+ *              the call would reject.
  * ---------------------------------------------------------------------------------------------- */
 size_t mnnllm_workspace_size_w4a8(int M, int N, int K, int group);
+size_t mnnllm_workspace_min_w4a8(int M, int N, int K, int group);
 int mnnllm_linear_w4a8(const void* x, const void* packed, void* y, int M, int N, int K, int group,
                        int x_dtype, int y_dtype, void* workspace, size_t workspace_bytes, void* stream);
 
 /* Several weight matrices that multiply the SAME activations (q, k, v of a layer; gate and up) in
  * one call: the activations are quantised once and one GEMM launch covers all the matrices
  * (Section 4.2; the fusion itself is this library's).  All problems share M, K, group and x; the
- * workspace is that of a single problem (mnnllm_workspace_size_w4a8 does not depend on N). */
+ * workspace is that of a single problem (the workspace sizes do not depend on N). */
 #define MNNLLM_MAX_BATCH_W4A8 4
 typedef struct {
     const void* packed; /* device, from mnnllm_pack_w4 for [N, K], the call's group */
@@ -170,7 +178,8 @@ int mnnllm_linear_w4a8_batch(const mnnllm_w4a8_problem* problems, int count, con
  *   - Limit: the activations' int8 copy (M*K bytes), their scales (4*M) and the fp16 group sums
  *     (8 * M * ceil(K/group/4)*4), each rounded up to 256 bytes, must fit the array; a larger
  *     problem returns MNNLLM_ERR_WORKSPACE and nothing is launched.  8 MiB covers, for example,
- *     M = 1024 tokens at K = 3584 or M = 512 at K = 8960.
+ *     M = 1024 tokens at K = 3584 or M = 512 at K = 8960.  The array has no room for the scratch
+ *     in which mnnllm_linear_w4a8 splits small problems along K: this entry point never does.
  *   - The first call on each device looks up the array's device address (one runtime query, the
  *     device must be current); make that first call before starting any stream capture.
  *   - All calls on a device share the one array and it keeps whatever the last call left there.

@@ -67,6 +67,7 @@ _sig("mnnllm_linear_w4a16_ex", _c.c_int,
 _sig("mnnllm_linear_w4a16_batch", _c.c_int, [_c.POINTER(_Problem), _c.c_int, _c.c_int, _P])
 _sig("mnnllm_linear_w8a16", _c.c_int, [_P, _P, _P, _c.c_int, _c.c_int, _c.c_int, _c.c_int, _P])
 _sig("mnnllm_workspace_size_w4a8", _c.c_size_t, [_c.c_int, _c.c_int, _c.c_int, _c.c_int])
+_sig("mnnllm_workspace_min_w4a8", _c.c_size_t, [_c.c_int, _c.c_int, _c.c_int, _c.c_int])
 _sig("mnnllm_linear_w4a8", _c.c_int,
      [_P, _P, _P, _c.c_int, _c.c_int, _c.c_int, _c.c_int, _c.c_int, _c.c_int, _P, _c.c_size_t, _P])
 _sig("mnnllm_linear_w4a8_batch", _c.c_int,
@@ -82,7 +83,7 @@ _sig("mnnllm_device_supported", _c.c_int, [])
 EXPORTS = [
     "mnnllm_status_string", "mnnllm_packed_size_w4", "mnnllm_pack_w4", "mnnllm_unpack_w4", "mnnllm_packed_info",
     "mnnllm_packed_size_w8", "mnnllm_pack_w8", "mnnllm_unpack_w8", "mnnllm_linear_w4a16", "mnnllm_linear_w4a16_ex",
-    "mnnllm_linear_w4a16_batch", "mnnllm_linear_w8a16", "mnnllm_workspace_size_w4a8", "mnnllm_linear_w4a8", "mnnllm_linear_w4a8_batch", "mnnllm_linear_w4a8_static",
+    "mnnllm_linear_w4a16_batch", "mnnllm_linear_w8a16", "mnnllm_workspace_size_w4a8", "mnnllm_workspace_min_w4a8", "mnnllm_linear_w4a8", "mnnllm_linear_w4a8_batch", "mnnllm_linear_w4a8_static",
     "mnnllm_quantize_activations", "mnnllm_debug_w4a8_partials", "mnnllm_read_status", "mnnllm_device_supported",
 ]
 
@@ -209,6 +210,10 @@ def linear_w8a16(x, packed, y, M, N, K, y_dtype=F16, stream=None) -> None:
 
 def workspace_size_w4a8(M: int, N: int, K: int, group: int) -> int:
     return int(lib.mnnllm_workspace_size_w4a8(M, N, K, group))
+
+
+def workspace_min_w4a8(M: int, N: int, K: int, group: int) -> int:
+    return int(lib.mnnllm_workspace_min_w4a8(M, N, K, group))
 
 
 def linear_w4a8(x, packed, y, M, N, K, group, workspace, workspace_bytes, x_dtype=F16, y_dtype=F16,

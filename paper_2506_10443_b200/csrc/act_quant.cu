@@ -46,11 +46,12 @@ template <typename T>
 __global__ void __launch_bounds__(kThreads) act_quant_kernel(const T* __restrict__ x, int K, int group,
                                                              int8_t* __restrict__ a_q, float* __restrict__ a_scale,
                                                              int32_t* __restrict__ A, uint2* __restrict__ AC, int G4,
-                                                             uint32_t code_xor) {
+                                                             uint32_t code_xor, uint32_t* __restrict__ clear, int n_clear) {
     __shared__ float warp_max[kThreads / 32];
     ptx::pdl_launch_dependents();
     ptx::pdl_wait();
     const int m = blockIdx.x;
+    for (int i = m * kThreads + threadIdx.x; i < n_clear; i += gridDim.x * kThreads) clear[i] = 0u;
     const uint4* row = reinterpret_cast<const uint4*>(x + (size_t)m * K);
     const int nvec = K / 8;
 
@@ -125,7 +126,8 @@ __global__ void __launch_bounds__(kThreads) act_quant_kernel(const T* __restrict
 }  // namespace
 
 cudaError_t act_quant_launch(const void* x, int x_dtype, int M, int K, int group, int8_t* a_q, float* a_scale,
-                             int32_t* A, void* AC, bool offset128, cudaStream_t stream) {
+                             int32_t* A, void* AC, bool offset128, uint32_t* clear, int n_clear, cudaStream_t stream) {
+    if (!clear) n_clear = 0;
     const uint32_t code_xor = offset128 ? 0x80808080u : 0u;
     const int G4 = (K / group + 3) / 4 * 4;
     uint2* ac = reinterpret_cast<uint2*>(AC);
@@ -140,9 +142,9 @@ cudaError_t act_quant_launch(const void* x, int x_dtype, int M, int K, int group
     cfg.numAttrs = 1;
     if (x_dtype == MNNLLM_F16)
         return cudaLaunchKernelEx(&cfg, act_quant_kernel<__half>, (const __half*)x, K, group, a_q, a_scale, A, ac,
-                                  G4, code_xor);
+                                  G4, code_xor, clear, n_clear);
     return cudaLaunchKernelEx(&cfg, act_quant_kernel<__nv_bfloat16>, (const __nv_bfloat16*)x, K, group, a_q, a_scale,
-                              A, ac, G4, code_xor);
+                              A, ac, G4, code_xor, clear, n_clear);
 }
 
 }  // namespace mnnllm

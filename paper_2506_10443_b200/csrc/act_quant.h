@@ -11,8 +11,9 @@ namespace mnnllm {
 // and, when AC is not null, the group sums as fp16 quadruples (64h, l, 64h, l), A = 64h + l,
 // [M, G4] x 8 bytes with G4 = K / group rounded up to a multiple of 4 (padding written as zeros).
 // With offset128 the codes are stored as unsigned bytes a_q + 128 (what the GEMM multiplies); the
-// sums A and AC are those of the signed codes either way.
+// sums A and AC are those of the signed codes either way.  `clear` (may be null) is an array of
+// n_clear words that the kernel sets to zero: the counters of the GEMM that follows.
 cudaError_t act_quant_launch(const void* x, int x_dtype, int M, int K, int group, int8_t* a_q, float* a_scale,
-                             int32_t* A, void* AC, bool offset128, cudaStream_t stream);
+                             int32_t* A, void* AC, bool offset128, uint32_t* clear, int n_clear, cudaStream_t stream);
 
 }  // namespace mnnllm

@@ -20,8 +20,10 @@ int check_xq(const void* x, int x_dtype, int M, int K, int group) {
 size_t round256(size_t v) { return (v + 255) & ~(size_t)255; }
 
 // workspace: a_q int8 [M, K] | a_scale fp32 [M] | fp16 group-sum quadruples [M, G4] x 8 bytes
+//            | optional: counters | fp32 parts of tiles that several CTAs share
 struct Workspace {
-    size_t a_q, a_scale, ac, total;
+    size_t a_q, a_scale, ac, total;   // total: what every call needs
+    size_t counters, scratch, total_split;   // total_split: with the scratch that lets the GEMM balance its work
 };
 Workspace workspace_layout(int M, int K, int group) {
     Workspace w;
@@ -30,6 +32,9 @@ Workspace workspace_layout(int M, int K, int group) {
     w.a_scale = round256((size_t)M * K);
     w.ac = w.a_scale + round256((size_t)M * 4);
     w.total = w.ac + round256((size_t)M * G4 * 8);
+    w.counters = w.total;
+    w.scratch = w.counters + round256((size_t)kGemmCounters * 4);
+    w.total_split = w.scratch + kGemmScratchBytes;
     return w;
 }
 
@@ -64,7 +69,8 @@ int mnnllm_quantize_activations(const void* x, int x_dtype, int M, int K, int gr
     if (!a_q || !a_scale || !A) return MNNLLM_ERR_INVALID_ARG;
     if (((uintptr_t)a_q & 15) || ((uintptr_t)a_scale & 3) || ((uintptr_t)A & 3)) return MNNLLM_ERR_ALIGNMENT;
     if (!device_is_supported()) return MNNLLM_ERR_UNSUPPORTED;
-    if (act_quant_launch(x, x_dtype, M, K, group, a_q, a_scale, A, nullptr, false, (cudaStream_t)stream) != cudaSuccess) {
+    if (act_quant_launch(x, x_dtype, M, K, group, a_q, a_scale, A, nullptr, false, nullptr, 0, (cudaStream_t)stream) !=
+        cudaSuccess) {
         (void)cudaGetLastError();
         return MNNLLM_ERR_CUDA;
     }
@@ -72,6 +78,11 @@ int mnnllm_quantize_activations(const void* x, int x_dtype, int M, int K, int gr
 }
 
 size_t mnnllm_workspace_size_w4a8(int M, int N, int K, int group) {
+    if (M < 1 || N < 1 || K < 1 || (group != 64 && group != 128) || K % group != 0) return 0;
+    return workspace_layout(M, K, group).total_split;
+}
+
+size_t mnnllm_workspace_min_w4a8(int M, int N, int K, int group) {
     if (M < 1 || N < 1 || K < 1 || (group != 64 && group != 128) || K % group != 0) return 0;
     return workspace_layout(M, K, group).total;
 }
@@ -90,6 +101,7 @@ int mnnllm_linear_w4a8_batch(const mnnllm_w4a8_problem* problems, int count, con
     const Workspace w = workspace_layout(M, K, group);
     if (!workspace || workspace_bytes < w.total) return MNNLLM_ERR_WORKSPACE;
     if ((uintptr_t)workspace & 255) return MNNLLM_ERR_ALIGNMENT;
+    const bool split = workspace_bytes >= w.total_split;
     if (!device_is_supported()) return MNNLLM_ERR_UNSUPPORTED;
     uint32_t* status = status_word_ptr();
     if (!status) return MNNLLM_ERR_CUDA;
@@ -98,8 +110,11 @@ int mnnllm_linear_w4a8_batch(const mnnllm_w4a8_problem* problems, int count, con
     int8_t* a_q = (int8_t*)(ws + w.a_q);
     float* a_scale = (float*)(ws + w.a_scale);
     void* ac = ws + w.ac;
-    // the activations are quantised once for all the matrices of the batch
-    if (act_quant_launch(x, x_dtype, M, K, group, a_q, a_scale, nullptr, ac, true, (cudaStream_t)stream) != cudaSuccess) {
+    uint32_t* counters = split ? (uint32_t*)(ws + w.counters) : nullptr;
+    // the activations are quantised once for all the matrices of the batch (the same kernel clears
+    // the counters of the GEMM)
+    if (act_quant_launch(x, x_dtype, M, K, group, a_q, a_scale, nullptr, ac, true, counters, kGemmCounters,
+                         (cudaStream_t)stream) != cudaSuccess) {
         (void)cudaGetLastError();
         return MNNLLM_ERR_CUDA;
     }
@@ -109,6 +124,8 @@ int mnnllm_linear_w4a8_batch(const mnnllm_w4a8_problem* problems, int count, con
         a.packed[i] = problems[i].packed; a.y[i] = problems[i].y; a.N[i] = problems[i].N; a.y_dtype[i] = problems[i].y_dtype;
     }
     a.a_q = a_q; a.a_scale = a_scale; a.AC = ac; a.P = nullptr;
+    a.scratch = split ? (float*)(ws + w.scratch) : nullptr;
+    a.counters = counters;
     a.M = M; a.K = K; a.group = group;
     const cudaError_t e = gemm_w4a8_launch(a, status, (cudaStream_t)stream);
     if (e != cudaSuccess) {
@@ -138,7 +155,8 @@ int mnnllm_debug_w4a8_partials(const void* x, int x_dtype, const void* packed, i
     if (!status) return MNNLLM_ERR_CUDA;
     // the GEMM multiplies the codes in their unsigned form (a_q + 128); the caller gets the signed
     // ones, written by a second run of the quantiser once the GEMM has consumed the buffer
-    if (act_quant_launch(x, x_dtype, M, K, group, a_q, a_scale, A, nullptr, true, (cudaStream_t)stream) != cudaSuccess) {
+    if (act_quant_launch(x, x_dtype, M, K, group, a_q, a_scale, A, nullptr, true, nullptr, 0, (cudaStream_t)stream) !=
+        cudaSuccess) {
         (void)cudaGetLastError();
         return MNNLLM_ERR_CUDA;
     }
@@ -146,13 +164,15 @@ int mnnllm_debug_w4a8_partials(const void* x, int x_dtype, const void* packed, i
     a.count = 1;
     a.packed[0] = packed; a.y[0] = nullptr; a.N[0] = N; a.y_dtype[0] = MNNLLM_F32;
     a.a_q = a_q; a.a_scale = a_scale; a.AC = nullptr; a.P = P;
+    a.scratch = nullptr; a.counters = nullptr;
     a.M = M; a.K = K; a.group = group;
     const cudaError_t e = gemm_w4a8_launch(a, status, (cudaStream_t)stream);
     if (e != cudaSuccess) {
         (void)cudaGetLastError();
         return e == cudaErrorNotSupported ? MNNLLM_ERR_UNSUPPORTED : MNNLLM_ERR_CUDA;
     }
-    if (act_quant_launch(x, x_dtype, M, K, group, a_q, a_scale, A, nullptr, false, (cudaStream_t)stream) != cudaSuccess) {
+    if (act_quant_launch(x, x_dtype, M, K, group, a_q, a_scale, A, nullptr, false, nullptr, 0, (cudaStream_t)stream) !=
+        cudaSuccess) {
         (void)cudaGetLastError();
         return MNNLLM_ERR_CUDA;
     }

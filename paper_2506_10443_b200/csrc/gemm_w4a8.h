@@ -8,6 +8,12 @@
 namespace mnnllm {
 
 constexpr int kGemmMaxBatch = 4;
+// A launch with fewer tiles than SMs cuts every tile's K range into parts that run as separate
+// work items; they meet through scratch memory: one 128 x 128 fp32 slot per part and sixteen
+// counters per tile (the quantiser that precedes the GEMM clears the counters).
+constexpr int kGemmScratchSlots = 320;
+constexpr size_t kGemmScratchBytes = (size_t)kGemmScratchSlots * 128 * 128 * 4;
+constexpr int kGemmCounters = 160 * 16;
 
 // `count` weight matrices that multiply the same quantised activations (q, k, v of a layer; gate and
 // up): one launch, the n-tiles of all of them in one grid.
@@ -21,6 +27,8 @@ struct GemmW4A8Args {
     const float* a_scale;  // device fp32 [M]
     const void* AC;        // device fp16 quadruples [M, G4] x 8 bytes (null in the partials form)
     int32_t* P;            // device int32 [M, N[0], G] (partials form only, count == 1)
+    float* scratch;        // device, kGemmScratchBytes (null: tiles are never split along K)
+    uint32_t* counters;    // device, kGemmCounters words, zero when the kernel starts (null with scratch)
     int M, K, group;
 };
 

@@ -65,9 +65,10 @@ def test_gpu_entry_points_fail_loudly_without_a_device():
     assert B.lib.mnnllm_linear_w4a16(0x1008, 0x1000, 0x1000, 1, 16, 64, 64, None) == 3
     assert B.lib.mnnllm_linear_w4a16(0x1000, 0x1000, 0x1000, 1, 16, 64, 100, None) == 2
     assert not B.device_supported()
-    need = B.workspace_size_w4a8(4, 16, 64, 64)
+    need = B.workspace_min_w4a8(4, 16, 64, 64)
     assert need >= 4 * 64 + 4 * 4 + 4 * 4 * 8 and need % 256 == 0
-    assert B.workspace_size_w4a8(4, 16, 64, 48) == 0
+    assert B.workspace_size_w4a8(4, 16, 64, 64) > need          # room for splitting tiles along K
+    assert B.workspace_size_w4a8(4, 16, 64, 48) == 0 and B.workspace_min_w4a8(4, 16, 64, 48) == 0
     f = B.lib.mnnllm_linear_w4a8
     assert f(0x1000, 0x1000, 0x1000, 4, 16, 64, 64, B.F16, B.F16, 0x1000, need, None) == 2   # no device
     assert f(0x1000, 0x1000, 0x1000, 4, 16, 64, 64, B.F16, B.F16, 0x1000, need - 1, None) == 6

@@ -124,6 +124,37 @@ def test_w4a8_batch_qkv_one_launch():
                                           nbytes, None) == 1
 
 
+@pytest.mark.parametrize("M,N,K,group", [
+    (64, 1536, 8960, 64),     # down projection at a short prompt: 12 tiles, 17.5 chunks of K
+    (200, 272, 3584, 128),    # ragged M and N, group 128
+    (128, 128, 1024, 64),     # one tile, two chunks
+])
+def test_w4a8_tiles_split_along_k(M, N, K, group):
+    # With the full workspace a problem with fewer tiles than SMs is cut along K and the parts are
+    # summed in scratch memory; with the minimal workspace it is not.  Both must match the oracle,
+    # agree closely with each other, and the split form must not depend on timing.
+    W, packed, (q, s, z) = quantized(3 * M + N + K, N, K, group)
+    x = inputs.activations(M + 5 * N + K, M, K, outliers=True)
+    ref = oracle.linear_w4a8(x.astype(np.float32), q, s, z, group)
+    xd, pd = dev(x), dev(packed)
+
+    def run(nbytes):
+        ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+        y = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
+        B.linear_w4a8(xd, pd, y, M, N, K, group, ws, nbytes, y_dtype=B.F32)
+        assert B.read_status() == 0
+        return y.cpu().numpy()
+
+    full, small = B.workspace_size_w4a8(M, N, K, group), B.workspace_min_w4a8(M, N, K, group)
+    assert full > small
+    y_split, y_whole = run(full), run(small)
+    assert_close(y_split, ref)
+    assert_close(y_whole, ref)
+    assert_close(y_split, y_whole.astype(np.float64), 1e-5)
+    for _ in range(3):
+        assert (run(full).view(np.uint32) == y_split.view(np.uint32)).all()
+
+
 def test_w4a8_deterministic():
     M, N, K, group = 200, 640, 1536, 64
     W, packed, _ = quantized(31, N, K, group)
@@ -136,7 +167,7 @@ def test_w4a8_deterministic():
 def test_w4a8_argument_errors_on_gpu():
     t = torch.empty(1 << 16, dtype=torch.uint8, device="cuda")
     p = t.data_ptr()
-    need = B.workspace_size_w4a8(4, 16, 64, 64)
+    need = B.workspace_min_w4a8(4, 16, 64, 64)
     assert need > 0 and B.workspace_size_w4a8(4, 16, 96, 64) == 0
     f = B.lib.mnnllm_linear_w4a8
     assert f(p, p, p, 4, 16, 64, 64, B.F16, B.F16, p, need - 1, None) == 6       # workspace too small

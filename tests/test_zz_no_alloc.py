@@ -21,7 +21,7 @@ def test_static_entry_rejects_oversized_problems_before_touching_the_gpu():
     # 4096 tokens x 8960 k need 36 MB of int8 activations: beyond the 8 MiB built-in scratch
     p = 0x1000
     f = B.lib.mnnllm_linear_w4a8_static
-    assert B.workspace_size_w4a8(4096, 64, 8960, 64) > B.STATIC_SCRATCH_BYTES
+    assert B.workspace_min_w4a8(4096, 64, 8960, 64) > B.STATIC_SCRATCH_BYTES
     assert f(p, p, p, 4096, 64, 8960, 64, B.F16, B.F16, None) == 6
     assert f(None, p, p, 4, 64, 64, 64, B.F16, B.F16, None) == 1
     assert f(p, p, p, 4, 64, 64, 48, B.F16, B.F16, None) == 2
@@ -36,7 +36,7 @@ def test_static_entry_matches_the_workspace_entry_on_two_calls_in_a_row():
         W = inputs.weights(900 + i, N, K)
         pd = dev(B.pack_w4(W, group))
         xd = dev(inputs.activations(910 + i, M, K, outliers=True))
-        nbytes = B.workspace_size_w4a8(M, N, K, group)
+        nbytes = B.workspace_min_w4a8(M, N, K, group)   # like the built-in scratch: no room to split tiles along K
         assert nbytes <= B.STATIC_SCRATCH_BYTES
         ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
         y_ref = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
