@@ -128,6 +128,17 @@ __global__ void __launch_bounds__(kThreads) act_quant_kernel(const T* __restrict
 cudaError_t act_quant_launch(const void* x, int x_dtype, int M, int K, int group, int8_t* a_q, float* a_scale,
                              int32_t* A, void* AC, bool offset128, uint32_t* clear, int n_clear, cudaStream_t stream) {
     if (!clear) n_clear = 0;
+    static bool carveout_set = false;
+    if (!carveout_set) {
+        // the GEMM that follows needs the largest shared-memory carve-out: ask for the same here, so
+        // that the SMs are not re-partitioned between the two kernels of a call
+        cudaFuncSetAttribute(act_quant_kernel<__half>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                             (int)cudaSharedmemCarveoutMaxShared);
+        cudaFuncSetAttribute(act_quant_kernel<__nv_bfloat16>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                             (int)cudaSharedmemCarveoutMaxShared);
+        (void)cudaGetLastError();
+        carveout_set = true;
+    }
     const uint32_t code_xor = offset128 ? 0x80808080u : 0u;
     const int G4 = (K / group + 3) / 4 * 4;
     uint2* ac = reinterpret_cast<uint2*>(AC);

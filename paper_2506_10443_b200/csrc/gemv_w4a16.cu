@@ -386,6 +386,15 @@ size_t smem_bytes(int W, int SR, int S) {
 template <int GROUP, int MP>
 cudaError_t ensure_smem(size_t smem) {
     static size_t configured = 0;  // per instantiation
+    static bool carveout_set = false;
+    if (!carveout_set) {
+        // every launch of the library asks for the same (largest) shared-memory carve-out, so that
+        // an SM does not have to re-partition its L1 between consecutive dependent launches
+        cudaError_t e = cudaFuncSetAttribute(gemv_w4a16_kernel<GROUP, MP>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                             (int)cudaSharedmemCarveoutMaxShared);
+        if (e != cudaSuccess) return e;
+        carveout_set = true;
+    }
     if (smem > configured) {
         cudaError_t e = cudaFuncSetAttribute(gemv_w4a16_kernel<GROUP, MP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)smem);

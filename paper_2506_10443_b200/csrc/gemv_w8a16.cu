@@ -222,6 +222,13 @@ gemv_w8a16_kernel(const __grid_constant__ GemvLaunch L, uint32_t* __restrict__ s
 
 static cudaError_t ensure_smem_w8(size_t smem) {
     static size_t configured = 0;
+    static bool carveout_set = false;
+    if (!carveout_set) {   // the same carve-out as every other kernel of the library
+        cudaError_t e = cudaFuncSetAttribute(gemv_w8a16_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                             (int)cudaSharedmemCarveoutMaxShared);
+        if (e != cudaSuccess) return e;
+        carveout_set = true;
+    }
     if (smem > configured) {
         cudaError_t e = cudaFuncSetAttribute(gemv_w8a16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
