@@ -268,8 +268,12 @@ cudaError_t gemm_w4a8_launch(const GemmW4A8Args& a, uint32_t* status, cudaStream
     if (n_sm <= 0) return cudaErrorInvalidDevice;
     // With fewer tiles than SMs the K range of every tile is cut into `split` parts (whole 512-k
     // chunks) that run as separate work items and meet through scratch memory.  The split is the
-    // one with the shortest critical path: waves of work items x (groups per item + a fixed cost
-    // per item, in units of one group's time).
+    // one with the shortest critical path, in units of one group's time (~0.5 us):
+    //     whole tiles:  groups per tile
+    //     split:        waves of work items x (groups per item + 11) + 0.6 x split
+    // where 11 stands for what a part costs beyond a whole tile's epilogue (scratch round trip,
+    // fences, counter) and 0.6 for each part that the last arrival adds up (fitted to graph-replay
+    // timings of 64 to 1024 tokens, K from 512 to 8960).
     const int n_chunks = (p.n_stages + 3) / 4;
     p.split = 1;
     p.split_stages = 4 * n_chunks;
@@ -277,12 +281,12 @@ cudaError_t gemm_w4a8_launch(const GemmW4A8Args& a, uint32_t* status, cudaStream
     p.counters = a.counters;
     if (!partials && a.scratch && a.counters && p.total_tiles < n_sm && p.total_tiles * kDrainWarps <= kGemmCounters) {
         const int groups_per_chunk = 512 / a.group;
-        long long best = (long long)n_chunks * groups_per_chunk + 3;
+        long long best = 10ll * n_chunks * groups_per_chunk;   // tenths of a group
         for (int s = 2; s <= n_chunks && (long long)p.total_tiles * s <= kGemmScratchSlots; ++s) {
             const int cps = (n_chunks + s - 1) / s;
             if ((s - 1) * cps >= n_chunks) continue;   // a range would be empty
             const long long waves = ((long long)p.total_tiles * s + n_sm - 1) / n_sm;
-            const long long cost = waves * ((long long)cps * groups_per_chunk + 8);
+            const long long cost = waves * (10ll * cps * groups_per_chunk + 110) + 6 * s;
             if (cost < best) {
                 best = cost;
                 p.split = s;
