@@ -13,17 +13,20 @@
 // and would bound the kernel at 1024 cycles per group; adding a float bit pattern as an integer
 // and subtracting it as a float is exact too but costs three instructions per partial.)
 //
-// One CTA computes a tile of 128 weight rows x 128 tokens.  The weights are the M side of the MMA,
-// so that a tensor-memory lane is one output channel n and its per-group scale is a per-thread
-// scalar in the drain.  Warp roles (23 warps):
-//   warp 0      producer: TMA loads of the packed int4 codes (the packed buffer seen as a 2-D tensor
-//               [row block][bytes]: one box of 8 row blocks x 1 KiB per stage; issuing one small bulk
-//               copy per row block instead costs ~75 cycles each and starves the pipeline) and of
-//               each 512-k chunk's (scale, zero) tables into shared-memory rings; TMA loads of the
-//               int8 activation tile (128 tokens x 128 k, 128B swizzle) and of the fp16 group-sum
-//               quadruples that feed the zero-point MMA
-//   warp 1      allocates tensor memory, issues tcgen05.mma (kind::i8 into one of three int32
-//               accumulators per group; kind::f16 for the zero-point term) and the commits
+// A tile is 128 weight rows x 128 tokens.  The weights are the M side of the MMA, so that a
+// tensor-memory lane is one output channel n and its per-group scale is a per-thread scalar in the
+// drain.  The kernel is persistent: one CTA per SM walks the work items (tiles; or, when a launch
+// has fewer tiles than SMs, K ranges of tiles that meet through scratch memory: the kernel source
+// in gemm_w4a8_kernel.inc is expanded once for each form).  Rings and barriers run across work
+// items.  Warp roles (23 warps):
+//   warp 0      producer, one elected thread: TMA loads of the packed int4 codes (the packed buffer
+//               seen as a 2-D tensor [row block][words]: one box of 8 row blocks x 1 KiB per stage;
+//               issuing one small bulk copy per row block instead costs ~75 cycles each and
+//               starves the pipeline) and of each 512-k chunk's (scale, zero) tables into
+//               shared-memory rings; TMA loads of the int8 activation tile (128 tokens x 128 k,
+//               128B swizzle) and of the fp16 group-sum quadruples that feed the zero-point MMA
+//   warp 1      allocates tensor memory; one elected thread issues tcgen05.mma (kind::i8 into one of
+//               three int32 accumulators per group; kind::f16 for the zero-point term) and the commits
 //   warps 2-5   unpack: packed int4 codes (shared-memory ring) -> int8 K-major tile in the
 //               128B-swizzled layout the MMA reads; the sum Q of every (row, group)'s codes
 //   warp 22     scales: each (row, group) pair of the stage: the fp32 scale for the drain; (s z)
