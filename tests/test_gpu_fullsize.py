@@ -77,6 +77,7 @@ def test_lm_head_w8_per_channel_fp32_logits():
 
 @pytest.mark.parametrize("model,config,M,names", [
     (inputs.QWEN2_1P5B, 3, 1024, ("q", "k", "gate", "down")),
+    (inputs.QWEN2_1P5B, 3, 256, ("q", "o", "down")),   # o and down: tiles cut along K
     (inputs.QWEN2_1P5B, 3, 64, ("v", "down")),
     (inputs.QWEN2_7B, 4, 512, ("o", "up", "down")),
 ])
