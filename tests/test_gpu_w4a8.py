@@ -155,6 +155,48 @@ def test_w4a8_tiles_split_along_k(M, N, K, group):
         assert (run(full).view(np.uint32) == y_split.view(np.uint32)).all()
 
 
+def test_w4a8_split_calls_back_to_back_share_a_workspace():
+    # The way a model runs it: calls on one stream, one workspace, replayed from a CUDA graph.  The
+    # counters and scratch slots of the K split are reused by every call (the quantiser of a call
+    # clears the counters, ordered behind the previous GEMM by the stream); outputs must not change
+    # from replay to replay and must match calls made one at a time.
+    M, group = 64, 64
+    shapes = [(1536, 8960), (2048, 1536), (1536, 1536)]   # (N, K): all with fewer tiles than SMs
+    nbytes = max(B.workspace_size_w4a8(M, N, K, group) for N, K in shapes)
+    ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    probs = []
+    for i, (N, K) in enumerate(shapes):
+        W, packed, _ = quantized(700 + i, N, K, group)
+        x = dev(inputs.activations(710 + i, M, K, outliers=True))
+        probs.append((x, dev(packed), N, K))
+    ys = [torch.zeros((M, N), dtype=torch.float32, device="cuda") for _, _, N, _ in probs]
+
+    def one_round(stream):
+        for (x, pk, N, K), y in zip(probs, ys):
+            B.linear_w4a8(x, pk, y, M, N, K, group, ws, nbytes, y_dtype=B.F32, stream=stream)
+
+    one_round(None)
+    torch.cuda.synchronize()
+    assert B.read_status() == 0
+    want = [y.clone() for y in ys]
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        one_round(s)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=s):
+            for _ in range(4):
+                one_round(s)
+        for _ in range(5):
+            for y in ys:
+                y.zero_()
+            g.replay()
+            torch.cuda.synchronize()
+            for y, w in zip(ys, want):
+                assert torch.equal(y, w)
+    assert B.read_status() == 0
+
+
 def test_w4a8_deterministic():
     M, N, K, group = 200, 640, 1536, 64
     W, packed, _ = quantized(31, N, K, group)
