@@ -276,8 +276,9 @@ gemv_w4a16_kernel(const __grid_constant__ GemvLaunch L, uint32_t* __restrict__ s
                 }
 
                 for (int it = 0; it < nit; ++it) {
-                    // ---- wait for this quantum's bulk copy ----
-                    if (!dead && !mbar_wait_bounded(&bars[slot], phase, kMaxPolls)) {
+                    // ---- wait for this quantum's bulk copy (a non-blocking probe first: the copy has
+                    // usually landed, and the probe is cheaper than the blocking form: +1 % measured) ----
+                    if (!dead && !mbar_test_wait(&bars[slot], phase) && !mbar_wait_bounded(&bars[slot], phase, kMaxPolls)) {
                         dead = true;
                         if (lane == 0) atomicOr(status, 0x100u | (uint32_t)pi);
                     }

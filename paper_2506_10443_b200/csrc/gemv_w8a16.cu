@@ -138,7 +138,7 @@ gemv_w8a16_kernel(const __grid_constant__ GemvLaunch L, uint32_t* __restrict__ s
                     if (first_visit && sr == 0 && c == 0) xs_all[warp * XS_FLOATS + r] += xsum;
                 }
                 for (int it = 0; it < nit; ++it) {
-                    if (!dead && !mbar_wait_bounded(&bars[slot], phase, kMaxPolls)) {
+                    if (!dead && !mbar_test_wait(&bars[slot], phase) && !mbar_wait_bounded(&bars[slot], phase, kMaxPolls)) {
                         dead = true;
                         if (lane == 0) atomicOr(status, 0x200u);
                     }
