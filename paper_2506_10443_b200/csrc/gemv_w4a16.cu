@@ -37,7 +37,6 @@ struct Cfg {
     static constexpr int GPS = 8 / MP;                   // group slots per accumulator tile
     static constexpr int NSETS = (GC + GPS - 1) / GPS;   // accumulator tiles per quantum
     static constexpr int QB = 8 * kSlabBytes + 16 * GC * 4;  // bytes of a full quantum
-    static constexpr int CORR_FLOATS = MP * GC * 2;
     static constexpr int PART_FLOATS = kGemvMaxRBI * MP * 16;
 };
 
@@ -114,8 +113,7 @@ gemv_w4a16_kernel(const __grid_constant__ GemvLaunch L, uint32_t* __restrict__ s
     // shared memory carve-up
     uint8_t* ring = smem + (size_t)warp * S * C::QB;
     float* fbase = reinterpret_cast<float*>(smem + (size_t)W * S * C::QB);
-    float* corr = fbase + warp * C::CORR_FLOATS;
-    float* part_all = fbase + W * C::CORR_FLOATS;            // [W][2][RBI][MP][16]
+    float* part_all = fbase;                                 // [W][2][RBI][MP][16]
     float* red = part_all + W * 2 * C::PART_FLOATS;          // [2][SR][RBI][MP][16]
     uint64_t* bars = reinterpret_cast<uint64_t*>(red + 2 * SR * C::PART_FLOATS) + warp * kGemvMaxStages;
 
@@ -231,7 +229,9 @@ gemv_w4a16_kernel(const __grid_constant__ GemvLaunch L, uint32_t* __restrict__ s
                         B[sl][3][0] = __byte_perm(u1.x, u1.y, 0x7632);
                         B[sl][3][1] = __byte_perm(u1.z, u1.w, 0x7632);
                     }
-                    __syncwarp();  // the previous chunk's correction terms are no longer read
+                    // group sums of the activations: lane (r, c) adds up its 16-k pieces of group
+                    // gsB + GPS * i of token tokB, the four lanes of a quad complete the sum
+                    float v1[C::NSETS], v2[C::NSETS];
 #pragma unroll
                     for (int i = 0; i < C::NSETS; ++i) {
                         const int gi = gsB + C::GPS * i;
@@ -257,21 +257,17 @@ gemv_w4a16_kernel(const __grid_constant__ GemvLaunch L, uint32_t* __restrict__ s
                         hi += __shfl_xor_sync(0xffffffffu, hi, 1);
                         lo += __shfl_xor_sync(0xffffffffu, lo, 2);
                         hi += __shfl_xor_sync(0xffffffffu, hi, 2);
-                        if (c == 0 && gi < C::GC) {
-                            corr[(tokB * C::GC + gi) * 2 + 0] = 1024.f * lo + 64.f * hi;
-                            corr[(tokB * C::GC + gi) * 2 + 1] = lo + hi;
-                        }
+                        v1[i] = 1024.f * lo + 64.f * hi;
+                        v2[i] = lo + hi;
                     }
-                    __syncwarp();
+                    // the correction terms of accumulator column 2c + e = (token, group slot) sit in
+                    // the quad whose row index r equals that column
 #pragma unroll
                     for (int s = 0; s < C::NSETS; ++s)
 #pragma unroll
                         for (int e = 0; e < 2; ++e) {
-                            const int col = 2 * c + e;
-                            const int gi = s * C::GPS + col / MP;
-                            const bool ok = gi < C::GC;
-                            C1[s][e] = ok ? corr[((col % MP) * C::GC + gi) * 2 + 0] : 0.f;
-                            C2[s][e] = ok ? corr[((col % MP) * C::GC + gi) * 2 + 1] : 0.f;
+                            C1[s][e] = __shfl_sync(0xffffffffu, v1[s], 4 * (2 * c + e));
+                            C2[s][e] = __shfl_sync(0xffffffffu, v2[s], 4 * (2 * c + e));
                         }
                 }
 
@@ -379,7 +375,7 @@ gemv_w4a16_kernel(const __grid_constant__ GemvLaunch L, uint32_t* __restrict__ s
 template <int GROUP, int MP>
 size_t smem_bytes(int W, int SR, int S) {
     using C = Cfg<GROUP, MP>;
-    return (size_t)W * S * C::QB + (size_t)W * C::CORR_FLOATS * 4 + (size_t)W * 2 * C::PART_FLOATS * 4 +
+    return (size_t)W * S * C::QB + (size_t)W * 2 * C::PART_FLOATS * 4 +
            (size_t)2 * SR * C::PART_FLOATS * 4 + (size_t)W * kGemvMaxStages * 8;
 }
 
