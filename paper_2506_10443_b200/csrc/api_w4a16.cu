@@ -72,7 +72,9 @@ int cached_occupancy(int bits, int group, int MP, int W, int SR, int S) {
 Plan make_plan(int nb_total, int nc_max, int group, int MP, int bits = 4) {
     Plan p;
     p.CS = 1;
-    while (p.CS < 8 && nb_total * p.CS < 120 && p.CS * 2 <= nc_max && nc_max >= 4) p.CS *= 2;
+    while (p.CS < 8 && p.CS * 2 <= nc_max && nc_max >= 4 &&
+           (nb_total * p.CS < 120 || (nb_total * p.CS < 400 && p.CS * kGemvMaxWarps < nc_max)))
+        p.CS *= 2;
     p.WC = (nc_max + p.CS - 1) / p.CS;
     if (p.WC > kGemvMaxWarps) p.WC = kGemvMaxWarps;
     p.SR = kGemvMaxWarps / p.WC;
