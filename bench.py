@@ -33,7 +33,7 @@ INT8_OVER_BF16 = 2.0                 # nominal dense tensor-rate ratio (4.5 POPS
 # ncu capture (profiles/), keyed by workload; None when no capture matches the current kernel.
 NCU_TRAFFIC_BYTES_PER_LAUNCH = {
     # mean of one layer's four launches (q+k+v, o, gate+up, down), profiles/gemv_w4a16_decode_qwen2_1p5b.txt
-    "decode_qwen2_1p5b_w4a16_g64": 6629952,
+    "decode_qwen2_1p5b_w4a16_g64": 6629760,
 }
 
 
