@@ -158,9 +158,9 @@ def metric_of(kind):
 
 def units_of_linear(kind, N, K, M):
     """Algorithmic work of one linear in the metric's unit x 1e9 (bytes) or x 1e12 (int8 ops)."""
-    from paper_2506_10443_b200.workloads import linear_bytes
+    from paper_2506_10443_b200 import inputs   # byte counts only: the oracle arm must not load the CUDA library
 
-    return linear_bytes(N, K, GROUP, M) if kind == "decode" else 2 * M * N * K
+    return inputs.linear_bytes(N, K, GROUP, M) if kind == "decode" else 2 * M * N * K
 
 
 def scale_of(kind):

@@ -120,6 +120,53 @@ typedef struct {
 } mnnllm_w4a16_problem;
 int mnnllm_linear_w4a16_batch(const mnnllm_w4a16_problem* problems, int count, int M, void* stream);
 
+/* ------------------------------------------------------------------------------------------------
+ * A whole decoder stack of W4A16 linears in ONE launch (decode, M <= 8 tokens).
+ *
+ * Decode time is the time to read the weights (Section 2; Section 4.2: decode is memory-bound), but
+ * one linear of a small model is well under a microsecond of memory time and each depends on its
+ * predecessor, so a launch per linear spends most of its time at launch boundaries.  This entry
+ * point runs a list of up to MNNLLM_STACK_MAX_PROBLEMS linears (each computing exactly what
+ * mnnllm_linear_w4a16_ex computes) as one persistent grid that keeps streaming weights while a
+ * dependent problem waits for its input.  (The operation is the paper's; the single launch, the
+ * plan and the dependency list are this library's.)
+ *
+ *   problems   host array.  Problem p reads x only after the problems listed in deps[0..n_deps-1]
+ *              (indices < p) have stored all their outputs; a problem without deps may start at once.
+ *              Problems run in index order on every SM, so list them in execution order.
+ *   plan       built once on the host by mnnllm_stack_plan_w4a16 (mnnllm_stack_plan_size bytes),
+ *              then copied by the caller to device memory (16-byte aligned), like packed weights.
+ *              n_sms = 0 takes the SM count of the current device (needs a GPU); a positive value
+ *              plans for that many SMs without touching a device.  The plan holds the device
+ *              pointers of the problems: rebuild it when a buffer moves.
+ *   workspace  device, 256-byte aligned, mnnllm_stack_workspace_size(plan) bytes, ALL ZERO before
+ *              its first use (mnnllm_stack_workspace_init enqueues that memset).  The launch keeps
+ *              its completion counters there; it never needs clearing again, but after a launch that
+ *              reported MNNLLM_ERR_TIMEOUT it must be zeroed before it is reused.  Two launches
+ *              that may overlap on the GPU need separate workspaces.
+ *   The launch is cooperative (every CTA resident at once): it fails with MNNLLM_ERR_CUDA if the GPU
+ *   cannot hold the grid, e.g. under a partitioning that hides SMs.  x is fp16; accumulation fp32.
+ * ---------------------------------------------------------------------------------------------- */
+#define MNNLLM_STACK_MAX_PROBLEMS 256
+#define MNNLLM_STACK_MAX_DEPS 4
+typedef struct {
+    const void* x;      /* device fp16 [M, K] */
+    const void* packed; /* device, from mnnllm_pack_w4 for [N, K] and the plan's group */
+    void* y;            /* device [M, N] of y_dtype, overwritten */
+    int N, K;
+    int y_dtype;
+    int n_deps;
+    int deps[MNNLLM_STACK_MAX_DEPS];
+} mnnllm_stack_problem;
+size_t mnnllm_stack_plan_size(int count);
+int mnnllm_stack_plan_w4a16(const mnnllm_stack_problem* problems, int count, int M, int group, int n_sms,
+                            void* plan_out);
+size_t mnnllm_stack_workspace_size(const void* plan_host);
+int mnnllm_stack_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
+/* plan_host: the plan in host memory (only its header is read); plan_dev: the same bytes on the device. */
+int mnnllm_linear_w4a16_stack(const void* plan_host, const void* plan_dev, void* workspace, size_t workspace_bytes,
+                              void* stream);
+
 /* W8A16 with per-channel int8 weights packed by mnnllm_pack_w8. */
 int mnnllm_linear_w8a16(const void* x, const void* packed, void* y, int M, int N, int K, int y_dtype,
                         void* stream);

@@ -46,6 +46,11 @@ class _Problem(_c.Structure):
                 ("y_dtype", _c.c_int)]
 
 
+class _StackProblem(_c.Structure):
+    _fields_ = [("x", _P), ("packed", _P), ("y", _P), ("N", _c.c_int), ("K", _c.c_int), ("y_dtype", _c.c_int),
+                ("n_deps", _c.c_int), ("deps", _c.c_int * 4)]
+
+
 def _sig(name, restype, argtypes):
     f = getattr(lib, name)
     f.restype = restype
@@ -65,6 +70,11 @@ _sig("mnnllm_linear_w4a16", _c.c_int, [_P, _P, _P, _c.c_int, _c.c_int, _c.c_int,
 _sig("mnnllm_linear_w4a16_ex", _c.c_int,
      [_P, _P, _P, _c.c_int, _c.c_int, _c.c_int, _c.c_int, _c.c_int, _c.c_int, _P])
 _sig("mnnllm_linear_w4a16_batch", _c.c_int, [_c.POINTER(_Problem), _c.c_int, _c.c_int, _P])
+_sig("mnnllm_stack_plan_size", _c.c_size_t, [_c.c_int])
+_sig("mnnllm_stack_plan_w4a16", _c.c_int, [_c.POINTER(_StackProblem), _c.c_int, _c.c_int, _c.c_int, _c.c_int, _P])
+_sig("mnnllm_stack_workspace_size", _c.c_size_t, [_P])
+_sig("mnnllm_stack_workspace_init", _c.c_int, [_P, _c.c_size_t, _P])
+_sig("mnnllm_linear_w4a16_stack", _c.c_int, [_P, _P, _P, _c.c_size_t, _P])
 _sig("mnnllm_linear_w8a16", _c.c_int, [_P, _P, _P, _c.c_int, _c.c_int, _c.c_int, _c.c_int, _P])
 _sig("mnnllm_workspace_size_w4a8", _c.c_size_t, [_c.c_int, _c.c_int, _c.c_int, _c.c_int])
 _sig("mnnllm_workspace_min_w4a8", _c.c_size_t, [_c.c_int, _c.c_int, _c.c_int, _c.c_int])
@@ -83,7 +93,8 @@ _sig("mnnllm_device_supported", _c.c_int, [])
 EXPORTS = [
     "mnnllm_status_string", "mnnllm_packed_size_w4", "mnnllm_pack_w4", "mnnllm_unpack_w4", "mnnllm_packed_info",
     "mnnllm_packed_size_w8", "mnnllm_pack_w8", "mnnllm_unpack_w8", "mnnllm_linear_w4a16", "mnnllm_linear_w4a16_ex",
-    "mnnllm_linear_w4a16_batch", "mnnllm_linear_w8a16", "mnnllm_workspace_size_w4a8", "mnnllm_workspace_min_w4a8", "mnnllm_linear_w4a8", "mnnllm_linear_w4a8_batch", "mnnllm_linear_w4a8_static",
+    "mnnllm_linear_w4a16_batch", "mnnllm_stack_plan_size", "mnnllm_stack_plan_w4a16", "mnnllm_stack_workspace_size",
+    "mnnllm_stack_workspace_init", "mnnllm_linear_w4a16_stack", "mnnllm_linear_w8a16", "mnnllm_workspace_size_w4a8", "mnnllm_workspace_min_w4a8", "mnnllm_linear_w4a8", "mnnllm_linear_w4a8_batch", "mnnllm_linear_w4a8_static",
     "mnnllm_quantize_activations", "mnnllm_debug_w4a8_partials", "mnnllm_read_status", "mnnllm_device_supported",
 ]
 
@@ -202,6 +213,39 @@ def make_batch(problems: Sequence[dict]):
 def linear_w4a16_batch(problems, M: int, stream=None) -> None:
     arr = problems if isinstance(problems, _c.Array) else make_batch(problems)
     _check(lib.mnnllm_linear_w4a16_batch(arr, len(arr), M, _stream(stream)), "linear_w4a16_batch")
+
+
+def stack_plan_w4a16(problems: Sequence[dict], M: int, group: int, n_sms: int = 0) -> np.ndarray:
+    """Host plan of ``linear_w4a16_stack`` for a list of dicts (x, packed, y, N, K, y_dtype, deps).
+    ``n_sms = 0`` plans for the current device.  Returns the plan as a uint8 host array; the caller
+    copies it to the device."""
+    arr = (_StackProblem * len(problems))()
+    for a, p in zip(arr, problems):
+        a.x, a.packed, a.y = _ptr(p["x"]), _ptr(p["packed"]), _ptr(p["y"])
+        a.N, a.K, a.y_dtype = p["N"], p["K"], p.get("y_dtype", F16)
+        deps = list(p.get("deps", ()))
+        a.n_deps = len(deps)
+        for i, d in enumerate(deps[:4]):
+            a.deps[i] = d
+    size = int(lib.mnnllm_stack_plan_size(len(arr)))
+    if size == 0:
+        raise MnnllmError(1, "stack_plan_size(%d)" % len(arr))
+    out = aligned_empty(size)
+    _check(lib.mnnllm_stack_plan_w4a16(arr, len(arr), M, group, n_sms, _ptr(out)), "stack_plan_w4a16")
+    return out
+
+
+def stack_workspace_size(plan_host: np.ndarray) -> int:
+    return int(lib.mnnllm_stack_workspace_size(_ptr(plan_host)))
+
+
+def stack_workspace_init(workspace, workspace_bytes: int, stream=None) -> None:
+    _check(lib.mnnllm_stack_workspace_init(_ptr(workspace), workspace_bytes, _stream(stream)), "stack_workspace_init")
+
+
+def linear_w4a16_stack(plan_host: np.ndarray, plan_dev, workspace, workspace_bytes: int, stream=None) -> None:
+    _check(lib.mnnllm_linear_w4a16_stack(_ptr(plan_host), _ptr(plan_dev), _ptr(workspace), workspace_bytes,
+                                         _stream(stream)), "linear_w4a16_stack")
 
 
 def linear_w8a16(x, packed, y, M, N, K, y_dtype=F16, stream=None) -> None:

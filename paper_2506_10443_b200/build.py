@@ -20,6 +20,8 @@ SOURCES = [
     "api_w4a16.cu",
     "gemv_w4a16.cu",
     "gemv_w8a16.cu",
+    "stack_w4a16.cu",
+    "api_stack.cu",
     "act_quant.cu",
     "gemm_w4a8.cu",
     "api_w4a8.cu",

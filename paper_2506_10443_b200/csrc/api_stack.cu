@@ -1,0 +1,162 @@
+// C-ABI entry points of the whole-stack W4A16 decode launch: the host-side plan (how every
+// problem's quanta are dealt to the CTAs) and the launch itself.
+#include <cuda_fp16.h>
+
+#include <cstring>
+
+#include "common.h"
+#include "stack.h"
+
+namespace mnnllm {
+namespace {
+
+constexpr size_t kSmemBudget = 227 * 1024;
+
+int sm_count_of_current_device() {
+    static int cached[64];
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+    if (!cached[dev]) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+        cached[dev] = n;
+    }
+    return cached[dev];
+}
+
+int mp_of(int M) { return M <= 1 ? 1 : (M <= 2 ? 2 : (M <= 4 ? 4 : 8)); }
+
+// most quanta a CTA receives when U runs of `gran` quanta are dealt evenly to n CTAs
+long long max_share(long long U, int gran, int n) {
+    if (U < n) return gran;
+    return ((U + n - 1) / n) * gran;
+}
+
+}  // namespace
+}  // namespace mnnllm
+
+using namespace mnnllm;
+
+extern "C" {
+
+size_t mnnllm_stack_plan_size(int count) {
+    if (count < 1 || count > MNNLLM_STACK_MAX_PROBLEMS) return 0;
+    return sizeof(StackHeader) + (size_t)count * sizeof(StackProblem);
+}
+
+int mnnllm_stack_plan_w4a16(const mnnllm_stack_problem* problems, int count, int M, int group, int n_sms,
+                            void* plan_out) {
+    if (!problems || !plan_out || count < 1 || count > MNNLLM_STACK_MAX_PROBLEMS || M < 1) return MNNLLM_ERR_INVALID_ARG;
+    if (M > 8 || (group != 64 && group != 128)) return MNNLLM_ERR_UNSUPPORTED;
+    if (n_sms == 0) {
+        if (!device_is_supported()) return MNNLLM_ERR_UNSUPPORTED;
+        n_sms = sm_count_of_current_device();
+    }
+    if (n_sms < 1) return MNNLLM_ERR_INVALID_ARG;
+    const int MP = mp_of(M);
+    const int W = kStackConsumerWarps;
+
+    StackHeader H;
+    std::memset(&H, 0, sizeof(H));
+    StackProblem* out = reinterpret_cast<StackProblem*>((uint8_t*)plan_out + sizeof(StackHeader));
+    long long max_quanta = 1;
+    int rot = 0;
+    for (int p = 0; p < count; ++p) {
+        const mnnllm_stack_problem& q = problems[p];
+        if (!q.x || !q.packed || !q.y || q.N < 1 || q.K < 1) return MNNLLM_ERR_INVALID_ARG;
+        if (q.K % group != 0) return MNNLLM_ERR_UNSUPPORTED;
+        if (q.y_dtype != MNNLLM_F16 && q.y_dtype != MNNLLM_BF16 && q.y_dtype != MNNLLM_F32) return MNNLLM_ERR_UNSUPPORTED;
+        if (((uintptr_t)q.x & 15) || ((uintptr_t)q.y & 15) || ((uintptr_t)q.packed & 127)) return MNNLLM_ERR_ALIGNMENT;
+        if (q.n_deps < 0 || q.n_deps > MNNLLM_STACK_MAX_DEPS) return MNNLLM_ERR_INVALID_ARG;
+        for (int d = 0; d < q.n_deps; ++d)
+            if (q.deps[d] < 0 || q.deps[d] >= p) return MNNLLM_ERR_INVALID_ARG;   // only earlier problems
+
+        const W4Geometry g = w4_geometry(q.N, q.K, group);
+        StackProblem D;
+        std::memset(&D, 0, sizeof(D));
+        D.packed = (const uint8_t*)q.packed;
+        D.x = q.x;
+        D.y = q.y;
+        D.row_block_bytes = g.row_block_bytes;
+        D.N = q.N; D.K = q.K;
+        D.NB = g.n_row_blocks; D.NC = g.n_chunks; D.NS = g.n_slabs;
+        D.weff = D.NC <= W ? (W / D.NC) * D.NC : W;
+        // Whole 16-row blocks per CTA (no exchange between CTAs) or runs of single quanta (even
+        // shares, blocks shared between neighbours): whichever needs fewer rounds of the CTA's
+        // warps, an exchange counting as half a round.
+        const long long Q = (long long)D.NB * D.NC;
+        const long long whole = max_share(D.NB, D.NC, n_sms), single = max_share(Q, 1, n_sms);
+        const double cost_whole = (double)((whole + D.weff - 1) / D.weff);
+        const double cost_single = (double)((single + D.weff - 1) / D.weff) + 0.5;
+        D.gran = (D.NC > 1 && cost_single < cost_whole) ? 1 : D.NC;
+        const long long U = Q / D.gran;
+        const long long share = D.gran == 1 ? single : whole;
+        max_quanta = share > max_quanta ? share : max_quanta;
+        // consecutive small problems start on different SMs
+        D.rot = rot;
+        rot = (int)((rot + (U < n_sms ? U : 0)) % n_sms);
+        D.y_dtype = q.y_dtype;
+        D.n_deps = q.n_deps;
+        for (int d = 0; d < q.n_deps; ++d) D.deps[d] = q.deps[d];
+        out[p] = D;
+    }
+    // the ring takes what the partial sums leave of the CTA's shared memory
+    int slots = 0;
+    for (int s = 1; s <= 96; ++s)
+        if (stack_w4a16_smem(group, MP, s, (int)max_quanta) <= kSmemBudget) slots = s;
+    if (slots < 2) return MNNLLM_ERR_UNSUPPORTED;   // a problem too large for M <= 8 at this shape
+    H.magic = kStackMagic; H.version = 1;
+    H.count = count; H.M = M; H.group = group; H.MP = MP;
+    H.n_ctas = n_sms;
+    H.ring_slots = slots;
+    H.max_quanta = (int32_t)max_quanta;
+    H.smem_bytes = (uint32_t)stack_w4a16_smem(group, MP, slots, (int)max_quanta);
+    std::memcpy(plan_out, &H, sizeof(H));
+    return MNNLLM_OK;
+}
+
+size_t mnnllm_stack_workspace_size(const void* plan_host) {
+    if (!plan_host) return 0;
+    StackHeader H;
+    std::memcpy(&H, plan_host, sizeof(H));
+    if (H.magic != kStackMagic) return 0;
+    return stack_ws_bytes(H.count, H.n_ctas, H.MP);
+}
+
+int mnnllm_stack_workspace_init(void* workspace, size_t workspace_bytes, void* stream) {
+    if (!workspace || workspace_bytes == 0) return MNNLLM_ERR_INVALID_ARG;
+    if (cudaMemsetAsync(workspace, 0, workspace_bytes, (cudaStream_t)stream) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return MNNLLM_ERR_CUDA;
+    }
+    return MNNLLM_OK;
+}
+
+int mnnllm_linear_w4a16_stack(const void* plan_host, const void* plan_dev, void* workspace, size_t workspace_bytes,
+                              void* stream) {
+    if (!plan_host || !plan_dev) return MNNLLM_ERR_INVALID_ARG;
+    StackHeader H;
+    std::memcpy(&H, plan_host, sizeof(H));
+    if (H.magic != kStackMagic || H.version != 1 || H.count < 1) return MNNLLM_ERR_INVALID_ARG;
+    if ((uintptr_t)plan_dev & 15) return MNNLLM_ERR_ALIGNMENT;
+    if (!workspace || workspace_bytes < stack_ws_bytes(H.count, H.n_ctas, H.MP)) return MNNLLM_ERR_WORKSPACE;
+    if ((uintptr_t)workspace & 255) return MNNLLM_ERR_ALIGNMENT;
+    if (!device_is_supported()) return MNNLLM_ERR_UNSUPPORTED;
+    if (H.n_ctas > sm_count_of_current_device()) return MNNLLM_ERR_UNSUPPORTED;   // all CTAs must be resident
+    uint32_t* status = status_word_ptr();
+    if (!status) return MNNLLM_ERR_CUDA;
+    StackWorkspace ws;
+    uint8_t* base = (uint8_t*)workspace;
+    ws.epoch = (uint32_t*)base;
+    ws.done = (uint32_t*)(base + 4);
+    ws.flags = (uint32_t*)(base + stack_ws_flags_offset());
+    ws.parts = (unsigned long long*)(base + stack_ws_parts_offset(H.count));
+    const void* problems_dev = (const uint8_t*)plan_dev + sizeof(StackHeader);
+    if (stack_w4a16_launch(H, problems_dev, ws, status, (cudaStream_t)stream) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return MNNLLM_ERR_CUDA;
+    }
+    return MNNLLM_OK;
+}
+
+}  // extern "C"

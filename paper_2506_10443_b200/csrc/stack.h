@@ -1,0 +1,75 @@
+// Whole-stack W4A16 decode in ONE persistent launch: plan blob, workspace layout and the host/device
+// interface of the kernel (internal to the library).
+//
+// A "plan" is built on the host from the caller's problem list, copied to the device by the caller
+// (like packed weights) and read by every CTA.  The workspace holds the cross-CTA state:
+//   word 0        epoch: number of launches that have completed on this workspace
+//   word 1        CTAs of the running launch that have finished
+//   flags[p]      row blocks of problem p stored so far, summed over all launches: problem p of
+//                 launch number e (0-based) is complete when flags[p] == (e + 1) * NB_p (mod 2^32)
+//   parts         per (problem, CTA): 16 rows x MP tokens of 8-byte words {fp32 partial sum, tag}
+//                 through which the CTAs that share a 16-row block exchange their partial sums; a
+//                 word is valid for launch e when its tag equals e + 1
+// Nothing is ever cleared: the workspace has to be all zero before its first launch only.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/mnnllm.h"
+#include "layout.h"
+
+namespace mnnllm {
+
+constexpr uint32_t kStackMagic = 0x4B54534Du;  // "MSTK"
+constexpr int kStackMaxDeps = 4;
+constexpr int kStackConsumerWarps = 14;   // + 1 producer warp: 480 threads, 136 registers each
+constexpr int kStackThreads = (kStackConsumerWarps + 1) * 32;
+
+struct StackProblem {            // 96 bytes, 16-byte aligned
+    const uint8_t* packed;       // packed buffer (header included)
+    const void* x;               // fp16 [M, K]
+    void* y;                     // [M, N] of y_dtype
+    unsigned long long row_block_bytes;
+    int N, K;
+    int NB, NC, NS;              // 16-row blocks, 512-k chunks, 64-k slabs per row
+    int gran;                    // CTAs receive runs of quanta that are multiples of gran (1 or NC)
+    int rot;                     // CTA `cta` plays the role of virtual CTA (cta - rot) mod n_ctas
+    int weff;                    // consumer warps used (a multiple of NC where NC <= the warp count)
+    int y_dtype;
+    int n_deps;
+    int deps[kStackMaxDeps];     // earlier problems that must be complete before x is read
+    int pad[2];
+};
+static_assert(sizeof(StackProblem) == 96, "descriptor is 96 bytes");
+
+struct StackHeader {             // 64 bytes
+    uint32_t magic, version;
+    int32_t count, M, group, MP;
+    int32_t n_ctas;              // grid size the plan was made for
+    int32_t ring_slots;          // quanta slots of the shared-memory ring
+    int32_t max_quanta;          // most quanta one CTA holds of any one problem
+    uint32_t smem_bytes;
+    uint32_t reserved[6];
+};
+static_assert(sizeof(StackHeader) == 64, "header is 64 bytes");
+
+struct StackWorkspace {          // device pointers into the caller's workspace
+    uint32_t* epoch;
+    uint32_t* done;
+    uint32_t* flags;             // [count]
+    unsigned long long* parts;   // [count][n_ctas][MP][16]
+};
+
+// byte offsets inside the workspace
+inline size_t stack_ws_flags_offset() { return 256; }
+inline size_t stack_ws_parts_offset(int count) { return 256 + (((size_t)count * 4 + 255) & ~(size_t)255); }
+inline size_t stack_ws_bytes(int count, int n_ctas, int MP) {
+    return stack_ws_parts_offset(count) + (size_t)count * n_ctas * MP * 16 * 8;
+}
+
+cudaError_t stack_w4a16_launch(const StackHeader& H, const void* plan_dev, const StackWorkspace& ws, uint32_t* status,
+                               cudaStream_t stream);
+// shared memory of one CTA for a ring of `slots` quanta and partial sums of `max_quanta` quanta
+size_t stack_w4a16_smem(int group, int MP, int slots, int max_quanta);
+
+}  // namespace mnnllm

@@ -1,0 +1,438 @@
+// The linears of a whole decoder stack (W4A16, M <= 8 tokens) in ONE persistent launch.
+//
+// Decode time is the time to stream the weights (Section 2, Section 4.2), but a decoder layer's
+// linears are a few megabytes each - well under a microsecond of HBM time - and every one depends
+// on its predecessor.  Launched one by one, each pays a launch boundary of several microseconds.
+// Here one cooperative grid (one CTA per SM) walks a list of problems in order:
+//   * a producer warp streams the CTA's share of EVERY problem's packed weights, in order, through
+//     one deep ring of shared-memory slots (bulk copies completing on mbarriers).  Weights depend on
+//     nothing, so the ring runs ahead across problem boundaries: HBM keeps streaming while the
+//     consumers sit in a dependency bubble;
+//   * 14 consumer warps take the quanta (16 rows x 512 k) of the current problem round-robin,
+//     multiply them with the warp-level MMA formulation of the single-launch GEMV and leave one
+//     partial sum per quantum in shared memory; the CTA then adds them up in a fixed order;
+//   * a 16-row block whose k-chunks are spread over several CTAs is finished by the CTA that holds
+//     its first chunk: the others hand over their partial sums as 8-byte {value, tag} words that
+//     the finisher polls directly (no fence, no flag: the word is the message);
+//   * a problem that depends on earlier ones polls their completion counters (bounded) before it
+//     reads its activations; completion = a release-ordered add after the outputs are stored.
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
+#include "gemv_w4a16_core.cuh"
+#include "ptx.cuh"
+#include "stack.h"
+
+namespace mnnllm {
+
+using namespace ptx;
+using namespace w4a16;
+
+namespace {
+
+constexpr uint32_t kMaxBarPolls = 1u << 15;    // mbarrier tries of up to 20 us each: ~0.65 s
+constexpr uint32_t kMaxFlagPolls = 1u << 20;   // global-memory polls of roughly 0.5-1 us each
+
+__device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t* p) {
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ unsigned long long ld_relaxed_u64(const unsigned long long* p) {
+    unsigned long long v;
+    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_relaxed_u64(unsigned long long* p, unsigned long long v) {
+    asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+__device__ __forceinline__ void red_release_add(uint32_t* p, uint32_t v) {
+    asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+
+// Quanta [q0, q1) of a problem that fall to CTA `cta`, in row-block-major order (q = rb * NC + j):
+// an even share of the problem's runs of `gran` quanta.
+// With fewer runs than CTAs the first U virtual CTAs take one run each, so that consecutive small
+// problems (rotated against each other by the plan) land on different SMs.
+__device__ __forceinline__ void cta_range(int NB, int NC, int gran, int cv, int n_ctas, int& q0, int& q1) {
+    const long long U = (long long)NB * NC / gran;
+    if (U < n_ctas) {
+        q0 = cv < U ? cv * gran : 0x3fffffff;   // empty, and beyond every row block
+        q1 = cv < U ? q0 + gran : 0x3fffffff;
+    } else {
+        q0 = (int)(U * cv / n_ctas) * gran;
+        q1 = (int)(U * (cv + 1) / n_ctas) * gran;
+    }
+}
+__device__ __forceinline__ int virtual_cta(int cta, int rot, int n_ctas) {
+    const int v = cta - rot;
+    return v < 0 ? v + n_ctas : v;
+}
+
+template <int GROUP, int MP>
+__global__ void __launch_bounds__(kStackThreads, 1)
+stack_w4a16_kernel(const __grid_constant__ StackHeader H, const StackProblem* __restrict__ plan,
+                   const __grid_constant__ StackWorkspace ws, uint32_t* __restrict__ status) {
+    using C = Cfg<GROUP, MP>;
+    extern __shared__ __align__(128) uint8_t smem[];
+    constexpr int W = kStackConsumerWarps;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int cta = blockIdx.x, n_ctas = gridDim.x;
+    const int S = H.ring_slots;
+
+    uint8_t* ring = smem;
+    float* part = reinterpret_cast<float*>(smem + (size_t)S * C::QB);            // [max_quanta][MP][16]
+    uint64_t* full = reinterpret_cast<uint64_t*>(part + (size_t)H.max_quanta * MP * 16);
+    uint64_t* empty = full + S;
+    volatile uint32_t* dead = reinterpret_cast<volatile uint32_t*>(empty + S);   // a bounded wait gave up
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+        *dead = 0;
+        fence_mbar_init();
+    }
+    fence_proxy_async_smem();
+    __syncthreads();
+
+    const uint32_t tag = *reinterpret_cast<volatile const uint32_t*>(ws.epoch) + 1u;  // this launch's number, from 1
+
+    if (warp == W) {
+        // =================== producer: every problem's weights, in order, never waits for x ===================
+        if (lane == 0) {
+            const uint64_t stream_policy = policy_evict_first();
+            int slot = 0, issued = 0;
+            uint32_t use_parity = 0;   // parity of (uses of this slot so far)
+            bool wrapped = false;
+            for (int p = 0; p < H.count; ++p) {
+                const StackProblem& D = plan[p];
+                const int NB = D.NB, NC = D.NC, gran = D.gran;
+                int q0, q1;
+                cta_range(NB, NC, gran, virtual_cta(cta, D.rot, n_ctas), n_ctas, q0, q1);
+                if (q0 >= q1) continue;
+                const uint8_t* body = D.packed + kHeaderBytes;
+                const unsigned long long rbb = D.row_block_bytes;
+                const int last_ns = D.NS - 8 * (NC - 1);
+                const uint32_t last_bytes = (uint32_t)(last_ns * kSlabBytes + 16 * (last_ns / C::SPG) * 4);
+                int rb = q0 / NC, j = q0 - rb * NC;
+                for (int q = q0; q < q1; ++q) {
+                    if (wrapped && !*dead && !mbar_test_wait(&empty[slot], use_parity ^ 1u) &&
+                        !mbar_wait_bounded(&empty[slot], use_parity ^ 1u, kMaxBarPolls)) {
+                        *dead = 1;
+                        atomicOr(status, 0x400u | (uint32_t)(p & 0xFF));
+                    }
+                    if (!*dead) {
+                        const uint32_t bytes = (j == NC - 1) ? last_bytes : (uint32_t)C::QB;
+                        mbar_arrive_expect_tx(&full[slot], bytes);
+                        bulk_g2s_hint(ring + (size_t)slot * C::QB, body + (size_t)rb * rbb + (size_t)j * C::QB, bytes,
+                                      &full[slot], stream_policy);
+                        ++issued;
+                    }
+                    if (++slot == S) { slot = 0; use_parity ^= 1u; wrapped = true; }
+                    if (++j == NC) { j = 0; ++rb; }
+                }
+            }
+            // no bulk copy may still be in flight into this CTA's shared memory when it exits
+            for (int n = issued > S ? issued - S : 0; n < issued; ++n)
+                if (!mbar_wait_bounded_compact(&full[n % S], (uint32_t)(n / S) & 1u, kMaxBarPolls)) {
+                    atomicOr(status, 0x800u);
+                    break;
+                }
+        }
+    } else {
+        // =================== consumers ===================
+        const int r = lane >> 2, c = lane & 3;
+        const int tokB = r % MP, gsB = r / MP;   // B-operand role of this lane: column r of the MMA
+        uint32_t B[8][4][2];
+        float C1[C::NSETS][2], C2[C::NSETS][2];
+        int seq_base = 0;                         // quanta of earlier problems that went through this CTA's ring
+        const int ctid = threadIdx.x;             // 0 .. W*32-1
+
+        for (int p = 0; p < H.count; ++p) {
+            const StackProblem& D = plan[p];
+            const int NB = D.NB, NC = D.NC, N = D.N, K = D.K;
+            int q0, q1;
+            const int cv = virtual_cta(cta, D.rot, n_ctas);
+            cta_range(NB, NC, D.gran, cv, n_ctas, q0, q1);
+            const int n = q1 - q0;
+            if (n <= 0) continue;   // uniform over the CTA
+            const int weff = D.weff;
+            const int last_ns = D.NS - 8 * (NC - 1);
+
+            if (warp < weff && warp < n) {
+                // ---- dependencies: the problems whose outputs (or side effects) x depends on ----
+                const int n_deps = D.n_deps;
+                if (n_deps > 0) {
+                    if (lane == 0 && !*dead) {
+                        for (int d = 0; d < n_deps; ++d) {
+                            const int dp = D.deps[d];
+                            const uint32_t target = tag * (uint32_t)plan[dp].NB;
+                            const uint32_t* f = ws.flags + dp;
+                            bool ok = false;
+                            for (uint32_t it = 0; it < kMaxFlagPolls; ++it) {
+                                if (ld_acquire_u32(f) == target) { ok = true; break; }
+                                if ((it & 255u) == 255u && *dead) break;
+                            }
+                            if (!ok) {
+                                if (!*dead) atomicOr(status, 0x100u | (uint32_t)(p & 0xFF));
+                                *dead = 1;
+                                break;
+                            }
+                        }
+                    }
+                    __syncwarp();
+                }
+                const __half* xbase = reinterpret_cast<const __half*>(D.x);
+                int cur_j = -1;
+                for (int i = warp; i < n; i += weff) {
+                    const int q = q0 + i;
+                    const int rb = q / NC, j = q - rb * NC;
+                    const int ns = (j == NC - 1) ? last_ns : 8;
+                    const int ng = ns / C::SPG;
+                    if (j != cur_j) {
+                        cur_j = j;
+                        // ---- activations of k-chunk j -> B fragments and per-group sums (read past L1:
+                        // another SM may have written them during this launch) ----
+                        const __half* xk = xbase + (size_t)j * kChunkK;
+                        // a lane holds the slabs of its groups gsB + GPS * s only (other B entries are zero)
+                        float lo[C::NSETS], hi[C::NSETS];
+                        uint32_t Pm[C::NSETS][C::SPG][4][2];
+#pragma unroll
+                        for (int s = 0; s < C::NSETS; ++s) {
+                            lo[s] = hi[s] = 0.f;
+#pragma unroll
+                            for (int sp = 0; sp < C::SPG; ++sp) {
+                                const int sl = (gsB + C::GPS * s) * C::SPG + sp;
+                                uint4 u0 = make_uint4(0, 0, 0, 0), u1 = u0;
+                                if (sl < ns && tokB < H.M) {
+                                    const uint4* px =
+                                        reinterpret_cast<const uint4*>(xk + (size_t)tokB * K + sl * kSlabK4 + 16 * c);
+                                    u0 = __ldcg(px);
+                                    u1 = __ldcg(px + 1);
+                                }
+                                Pm[s][sp][0][0] = __byte_perm(u0.x, u0.y, 0x5410);
+                                Pm[s][sp][0][1] = __byte_perm(u0.z, u0.w, 0x5410);
+                                Pm[s][sp][1][0] = __byte_perm(u0.x, u0.y, 0x7632);
+                                Pm[s][sp][1][1] = __byte_perm(u0.z, u0.w, 0x7632);
+                                Pm[s][sp][2][0] = __byte_perm(u1.x, u1.y, 0x5410);
+                                Pm[s][sp][2][1] = __byte_perm(u1.z, u1.w, 0x5410);
+                                Pm[s][sp][3][0] = __byte_perm(u1.x, u1.y, 0x7632);
+                                Pm[s][sp][3][1] = __byte_perm(u1.z, u1.w, 0x7632);
+                                float2 f;
+                                f = h2f2(u0.x); lo[s] += f.x + f.y;
+                                f = h2f2(u0.y); lo[s] += f.x + f.y;
+                                f = h2f2(u1.x); lo[s] += f.x + f.y;
+                                f = h2f2(u1.y); lo[s] += f.x + f.y;
+                                f = h2f2(u0.z); hi[s] += f.x + f.y;
+                                f = h2f2(u0.w); hi[s] += f.x + f.y;
+                                f = h2f2(u1.z); hi[s] += f.x + f.y;
+                                f = h2f2(u1.w); hi[s] += f.x + f.y;
+                            }
+                        }
+#pragma unroll
+                        for (int sl = 0; sl < 8; ++sl) {
+                            const int gi = sl / C::SPG;
+                            const bool mine = gsB == gi % C::GPS;
+#pragma unroll
+                            for (int a = 0; a < 4; ++a)
+#pragma unroll
+                                for (int b = 0; b < 2; ++b)
+                                    B[sl][a][b] = mine ? Pm[gi / C::GPS][sl % C::SPG][a][b] : 0u;
+                        }
+#pragma unroll
+                        for (int s = 0; s < C::NSETS; ++s) {
+                            float l = lo[s], h = hi[s];
+                            l += __shfl_xor_sync(0xffffffffu, l, 1);
+                            h += __shfl_xor_sync(0xffffffffu, h, 1);
+                            l += __shfl_xor_sync(0xffffffffu, l, 2);
+                            h += __shfl_xor_sync(0xffffffffu, h, 2);
+                            const float v1 = 1024.f * l + 64.f * h, v2 = l + h;
+                            // correction terms of accumulator column 2c + e sit in the quad with r == that column
+#pragma unroll
+                            for (int e = 0; e < 2; ++e) {
+                                C1[s][e] = __shfl_sync(0xffffffffu, v1, 4 * (2 * c + e));
+                                C2[s][e] = __shfl_sync(0xffffffffu, v2, 4 * (2 * c + e));
+                            }
+                        }
+                    }
+
+                    // ---- this quantum's ring slot ----
+                    const int seq = seq_base + i;
+                    const int use = seq / S, slot = seq - use * S;
+                    if (!*dead && !mbar_test_wait(&full[slot], (uint32_t)use & 1u) &&
+                        !mbar_wait_bounded(&full[slot], (uint32_t)use & 1u, kMaxBarPolls)) {
+                        *dead = 1;
+                        if (lane == 0) atomicOr(status, 0x200u | (uint32_t)(p & 0xFF));
+                    }
+                    const uint8_t* qp = ring + (size_t)slot * C::QB;
+                    const uint4* slabs = reinterpret_cast<const uint4*>(qp);
+                    float Dm[C::NSETS][4];
+                    if (ns == 8) quantum_mma<GROUP, MP, true>(slabs, lane, 8, B, Dm);
+                    else quantum_mma<GROUP, MP, false>(slabs, lane, ns, B, Dm);
+
+                    float out[2][2] = {{0.f, 0.f}, {0.f, 0.f}};   // [row half h][column e]
+                    auto rescale = [&](const int ngc) {
+                        const uint32_t* table = reinterpret_cast<const uint32_t*>(qp + (size_t)ngc * C::SPG * kSlabBytes);
+#pragma unroll
+                        for (int s = 0; s < C::NSETS; ++s)
+#pragma unroll
+                            for (int e = 0; e < 2; ++e) {
+                                const int gi = s * C::GPS + (2 * c + e) / MP;
+                                const bool ok = gi < ngc;
+                                const int gic = ok ? gi : 0;
+#pragma unroll
+                                for (int h = 0; h < 2; ++h) {
+                                    const float2 sz = h2f2(table[(r + 8 * h) * ngc + gic]);
+                                    const float v = sz.x * ((Dm[s][2 * h + e] - C1[s][e]) - sz.y * C2[s][e]);
+                                    out[h][e] += ok ? v : 0.f;
+                                }
+                            }
+                    };
+                    if (ns == 8) rescale(C::GC); else rescale(ng);
+                    // the slot has been read: hand it back to the producer
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&empty[slot]);
+
+                    if (MP == 1) { out[0][0] += out[0][1]; out[1][0] += out[1][1]; }
+#pragma unroll
+                    for (int h = 0; h < 2; ++h)
+#pragma unroll
+                        for (int e = 0; e < 2; ++e) {
+                            if (MP <= 2) out[h][e] += __shfl_xor_sync(0xffffffffu, out[h][e], 1);
+                            if (MP <= 4) out[h][e] += __shfl_xor_sync(0xffffffffu, out[h][e], 2);
+                        }
+                    const bool writer = (MP == 8) || (MP == 4 && c < 2) || (MP <= 2 && c == 0);
+                    if (writer) {
+#pragma unroll
+                        for (int e = 0; e < (MP == 1 ? 1 : 2); ++e) {
+                            const int tok = (2 * c + e) % MP;
+#pragma unroll
+                            for (int h = 0; h < 2; ++h) part[((size_t)i * MP + tok) * 16 + r + 8 * h] = out[h][e];
+                        }
+                    }
+                }
+            }
+            seq_base += n;
+
+            // ---- the CTA's partial sums -> outputs; row blocks shared with other CTAs go through the workspace ----
+            bar_sync(1, W * 32);
+            const int rb_first = q0 / NC, rb_last = (q1 - 1) / NC;
+            const int n_out = (rb_last - rb_first + 1) * MP * 16;
+            unsigned long long* my_parts = ws.parts + ((size_t)p * n_ctas + cv) * (MP * 16);
+            for (int o = ctid; o < n_out; o += W * 32) {
+                const int row = o & 15, tok = (o >> 4) % MP, rb = rb_first + o / (16 * MP);
+                const int qa = rb * NC, qb = qa + NC;          // the row block's quanta
+                const int lo_q = qa > q0 ? qa : q0, hi_q = qb < q1 ? qb : q1;
+                float acc = 0.f;
+                for (int q = lo_q; q < hi_q; ++q) acc += part[((size_t)(q - q0) * MP + tok) * 16 + row];
+                if (qa < q0) {
+                    // the block starts in an earlier CTA, which finishes it: hand the partial sum over
+                    st_relaxed_u64(my_parts + tok * 16 + row,
+                                   ((unsigned long long)tag << 32) | (unsigned long long)__float_as_uint(acc));
+                    continue;
+                }
+                if (qb > q1) {
+                    // this CTA holds the block's first quantum: add the later (virtual) CTAs' parts in order
+                    for (int c2 = cv + 1; c2 < n_ctas; ++c2) {
+                        int r0, r1;
+                        cta_range(NB, NC, D.gran, c2, n_ctas, r0, r1);
+                        if (r0 >= qb) break;
+                        if (r0 >= r1) continue;
+                        const unsigned long long* src = ws.parts + ((size_t)p * n_ctas + c2) * (MP * 16) + tok * 16 + row;
+                        unsigned long long v = 0;
+                        bool ok = false;
+                        if (!*dead) {
+                            for (uint32_t it = 0; it < kMaxFlagPolls; ++it) {
+                                v = ld_relaxed_u64(src);
+                                if ((uint32_t)(v >> 32) == tag) { ok = true; break; }
+                                if ((it & 255u) == 255u && *dead) break;
+                            }
+                            if (!ok) {
+                                if (!*dead) atomicOr(status, 0x1000u | (uint32_t)(p & 0xFF));
+                                *dead = 1;
+                            }
+                        }
+                        acc += __uint_as_float((uint32_t)v);
+                    }
+                }
+                const int nrow = rb * 16 + row;
+                if (nrow < N && tok < H.M) store_out(D.y, D.y_dtype, (size_t)tok * N + nrow, acc);
+            }
+            // ---- completion: row blocks whose first quantum this CTA holds were stored by it ----
+            bar_sync(1, W * 32);
+            if (ctid == 0) {
+                const int stored = (q1 + NC - 1) / NC - (q0 + NC - 1) / NC;
+                if (stored > 0) {
+                    __threadfence();
+                    red_release_add(ws.flags + p, (uint32_t)stored);
+                }
+            }
+        }
+    }
+
+    // ---- end of the launch: the last CTA to finish advances the workspace's launch counter ----
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        const uint32_t old = atomicAdd(ws.done, 1u);
+        if (old == (uint32_t)n_ctas - 1u) {
+            *reinterpret_cast<volatile uint32_t*>(ws.done) = 0u;
+            *reinterpret_cast<volatile uint32_t*>(ws.epoch) = tag;
+        }
+    }
+}
+
+template <int GROUP, int MP>
+size_t smem_of(int slots, int max_quanta) {
+    using C = Cfg<GROUP, MP>;
+    return (size_t)slots * C::QB + (size_t)max_quanta * MP * 16 * 4 + (size_t)2 * slots * 8 + 16;
+}
+
+template <int GROUP, int MP>
+cudaError_t launch_one(const StackHeader& H, const void* plan_dev, const StackWorkspace& ws, uint32_t* status,
+                       cudaStream_t stream) {
+    auto kern = stack_w4a16_kernel<GROUP, MP>;
+    // function attributes belong to a device: set per device, once
+    static bool configured[64];
+    int dev = -1;
+    if (cudaError_t e = cudaGetDevice(&dev); e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (!configured[dev]) {
+        if (cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+            e != cudaSuccess)
+            return e;
+        configured[dev] = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)H.n_ctas);
+    cfg.blockDim = dim3((unsigned)kStackThreads);
+    cfg.dynamicSmemBytes = H.smem_bytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeCooperative;   // all CTAs resident together, or the launch fails
+    attr[0].val.cooperative = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, H, reinterpret_cast<const StackProblem*>(plan_dev), ws, status);
+}
+
+}  // namespace
+
+size_t stack_w4a16_smem(int group, int MP, int slots, int max_quanta) {
+#define MNN_CASE(G, P) if (group == G && MP == P) return smem_of<G, P>(slots, max_quanta);
+    MNN_CASE(64, 1) MNN_CASE(64, 2) MNN_CASE(64, 4) MNN_CASE(64, 8)
+    MNN_CASE(128, 1) MNN_CASE(128, 2) MNN_CASE(128, 4) MNN_CASE(128, 8)
+#undef MNN_CASE
+    return 0;
+}
+
+cudaError_t stack_w4a16_launch(const StackHeader& H, const void* plan_dev, const StackWorkspace& ws, uint32_t* status,
+                               cudaStream_t stream) {
+#define MNN_CASE(G, P) if (H.group == G && H.MP == P) return launch_one<G, P>(H, plan_dev, ws, status, stream);
+    MNN_CASE(64, 1) MNN_CASE(64, 2) MNN_CASE(64, 4) MNN_CASE(64, 8)
+    MNN_CASE(128, 1) MNN_CASE(128, 2) MNN_CASE(128, 4) MNN_CASE(128, 8)
+#undef MNN_CASE
+    return cudaErrorInvalidValue;
+}
+
+}  // namespace mnnllm

@@ -88,6 +88,16 @@ LM_HEAD = dict(N=151936, K=3584, group=128)
 PROMPT_LENGTHS = (64, 256, 1024)
 
 
+def w4_bytes(N: int, K: int, group: int) -> int:
+    """Bytes of int4 codes plus fp16 (scale, zero) pairs of an [N, K] matrix (a byte count only)."""
+    return N * K // 2 + N * (K // group) * 4
+
+
+def linear_bytes(N: int, K: int, group: int, M: int, y_bytes: int = 2) -> int:
+    """Bytes a W4A16 linear has to move: packed weights once, fp16 activations in, outputs out."""
+    return w4_bytes(N, K, group) + 2 * M * K + y_bytes * M * N
+
+
 def stack(model: dict) -> List[Linear]:
     return decoder_layer(model["hidden"], model["kv_dim"], model["inter"])
 

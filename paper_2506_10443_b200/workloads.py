@@ -21,14 +21,8 @@ _INPUT_OF = {"q": 0, "k": 0, "v": 0, "o": 1, "gate": 2, "up": 2, "down": 3}
 _INPUT_SEED_ID = {0: 0, 1: 3, 2: 4, 3: 6}
 
 
-def w4_bytes(N: int, K: int, group: int) -> int:
-    """Bytes of codes plus fp16 (scale, zero) pairs of an [N, K] matrix."""
-    return N * K // 2 + N * (K // group) * 4
-
-
-def linear_bytes(N: int, K: int, group: int, M: int, y_bytes: int = 2) -> int:
-    """Bytes the W4A16 linear has to move: packed weights once, activations in, outputs out."""
-    return w4_bytes(N, K, group) + 2 * M * K + y_bytes * M * N
+w4_bytes = inputs.w4_bytes
+linear_bytes = inputs.linear_bytes
 
 
 @dataclass
@@ -119,6 +113,31 @@ class LinearStack:
     def run_w4a16(self, stream=None) -> None:
         for arr in self._decode_launches():
             B.linear_w4a16_batch(arr, self.M, stream)
+
+    def _stack_plan(self):
+        """The whole stack as ONE launch.  The dependency list is the decoder's: q, k, v wait for the
+        previous layer's down projection, o for q, k, v, gate and up for o, down for gate and up."""
+        if getattr(self, "_plan", None) is None:
+            probs, prev_down = [], None
+            for l, L in enumerate(self.layers):
+                idx = {}
+                for lin in self.linears:
+                    deps = {"q": [prev_down], "k": [prev_down], "v": [prev_down], "o": [idx.get("q"), idx.get("k"), idx.get("v")],
+                            "gate": [idx.get("o")], "up": [idx.get("o")], "down": [idx.get("gate"), idx.get("up")]}[lin.name]
+                    idx[lin.name] = len(probs)
+                    probs.append(dict(x=self.x_view(l, lin.name), packed=L.packed[lin.name], y=self.y_view(l, lin.name),
+                                      N=lin.N, K=lin.K, y_dtype=B.F16, deps=[d for d in deps if d is not None]))
+                prev_down = idx["down"]
+            plan = B.stack_plan_w4a16(probs, self.M, self.group)
+            plan_dev = torch.from_numpy(plan).to(self.device)
+            nbytes = B.stack_workspace_size(plan)
+            ws = torch.zeros(nbytes, dtype=torch.uint8, device=self.device)
+            self._plan = (plan, plan_dev, ws, nbytes)
+        return self._plan
+
+    def run_w4a16_stack(self, stream=None) -> None:
+        plan, plan_dev, ws, nbytes = self._stack_plan()
+        B.linear_w4a16_stack(plan, plan_dev, ws, nbytes, stream)
 
     # ---- prefill ----
     @property
