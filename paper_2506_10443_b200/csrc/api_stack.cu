@@ -2,6 +2,7 @@
 // problem's quanta are dealt to the CTAs) and the launch itself.
 #include <cuda_fp16.h>
 
+#include <cstdlib>
 #include <cstring>
 
 #include "common.h"
@@ -11,6 +12,7 @@ namespace mnnllm {
 namespace {
 
 constexpr size_t kSmemBudget = 227 * 1024;
+constexpr long long kStageBudget = 40 * 1024;   // staged activations per CTA at most
 
 int sm_count_of_current_device() {
     static int cached[64];
@@ -59,7 +61,7 @@ int mnnllm_stack_plan_w4a16(const mnnllm_stack_problem* problems, int count, int
     StackHeader H;
     std::memset(&H, 0, sizeof(H));
     StackProblem* out = reinterpret_cast<StackProblem*>((uint8_t*)plan_out + sizeof(StackHeader));
-    long long max_quanta = 1;
+    long long max_quanta = 1, xs_bytes = 0;
     int rot = 0;
     for (int p = 0; p < count; ++p) {
         const mnnllm_stack_problem& q = problems[p];
@@ -85,6 +87,7 @@ int mnnllm_stack_plan_w4a16(const mnnllm_stack_problem* problems, int count, int
         // shares, blocks shared between neighbours): whichever needs fewer rounds of the CTA's
         // warps, an exchange counting as half a round.
         const long long Q = (long long)D.NB * D.NC;
+        if (Q * n_sms >= (1ll << 31)) return MNNLLM_ERR_UNSUPPORTED;   // the kernel deals quanta in 32-bit arithmetic
         const long long whole = max_share(D.NB, D.NC, n_sms), single = max_share(Q, 1, n_sms);
         const double cost_whole = (double)((whole + D.weff - 1) / D.weff);
         const double cost_single = (double)((single + D.weff - 1) / D.weff) + 0.5;
@@ -92,25 +95,39 @@ int mnnllm_stack_plan_w4a16(const mnnllm_stack_problem* problems, int count, int
         const long long U = Q / D.gran;
         const long long share = D.gran == 1 ? single : whole;
         max_quanta = share > max_quanta ? share : max_quanta;
+        // activations go through shared memory when the chunks one CTA needs are small enough
+        const long long x_need = (share < D.NC ? share : D.NC) * (long long)M * kChunkK * 2;
+        D.stage_x = x_need <= kStageBudget ? 1 : 0;
+        if (D.stage_x && x_need > xs_bytes) xs_bytes = x_need;
         // consecutive small problems start on different SMs
         D.rot = rot;
         rot = (int)((rot + (U < n_sms ? U : 0)) % n_sms);
         D.y_dtype = q.y_dtype;
         D.n_deps = q.n_deps;
-        for (int d = 0; d < q.n_deps; ++d) D.deps[d] = q.deps[d];
+        for (int d = 0; d < q.n_deps; ++d) {
+            D.deps[d] = q.deps[d];
+            D.deps_nb[d] = out[q.deps[d]].NB;
+        }
         out[p] = D;
     }
     // the ring takes what the partial sums leave of the CTA's shared memory
     int slots = 0;
     for (int s = 1; s <= 96; ++s)
-        if (stack_w4a16_smem(group, MP, s, (int)max_quanta) <= kSmemBudget) slots = s;
+        if (stack_w4a16_smem(group, MP, count, s, (int)max_quanta, (int)xs_bytes) <= kSmemBudget) slots = s;
     if (slots < 2) return MNNLLM_ERR_UNSUPPORTED;   // a problem too large for M <= 8 at this shape
     H.magic = kStackMagic; H.version = 1;
     H.count = count; H.M = M; H.group = group; H.MP = MP;
     H.n_ctas = n_sms;
     H.ring_slots = slots;
     H.max_quanta = (int32_t)max_quanta;
-    H.smem_bytes = (uint32_t)stack_w4a16_smem(group, MP, slots, (int)max_quanta);
+    H.xs_bytes = (uint32_t)xs_bytes;
+    H.window = 16;
+    if (const char* env = std::getenv("MNNLLM_STACK_WINDOW")) {   // tuning override
+        const int v = std::atoi(env);
+        if (v >= 1) H.window = v;
+    }
+    if (H.window >= slots) H.window = slots - 1;
+    H.smem_bytes = (uint32_t)stack_w4a16_smem(group, MP, count, slots, (int)max_quanta, (int)xs_bytes);
     std::memcpy(plan_out, &H, sizeof(H));
     return MNNLLM_OK;
 }

@@ -25,7 +25,7 @@ constexpr int kStackMaxDeps = 4;
 constexpr int kStackConsumerWarps = 14;   // + 1 producer warp: 480 threads, 136 registers each
 constexpr int kStackThreads = (kStackConsumerWarps + 1) * 32;
 
-struct StackProblem {            // 96 bytes, 16-byte aligned
+struct StackProblem {            // 112 bytes, 16-byte aligned
     const uint8_t* packed;       // packed buffer (header included)
     const void* x;               // fp16 [M, K]
     void* y;                     // [M, N] of y_dtype
@@ -38,9 +38,11 @@ struct StackProblem {            // 96 bytes, 16-byte aligned
     int y_dtype;
     int n_deps;
     int deps[kStackMaxDeps];     // earlier problems that must be complete before x is read
-    int pad[2];
+    int deps_nb[kStackMaxDeps];  // their row-block counts (the completion counter's increment per launch)
+    int stage_x;                 // 1: the CTA copies the k-chunks of x it needs to shared memory first
+    int pad[1];
 };
-static_assert(sizeof(StackProblem) == 96, "descriptor is 96 bytes");
+static_assert(sizeof(StackProblem) == 112, "descriptor is 112 bytes");
 
 struct StackHeader {             // 64 bytes
     uint32_t magic, version;
@@ -49,7 +51,9 @@ struct StackHeader {             // 64 bytes
     int32_t ring_slots;          // quanta slots of the shared-memory ring
     int32_t max_quanta;          // most quanta one CTA holds of any one problem
     uint32_t smem_bytes;
-    uint32_t reserved[6];
+    int32_t window;              // bulk copies a CTA keeps in flight at most
+    uint32_t xs_bytes;           // shared memory for staged activations
+    uint32_t reserved[4];
 };
 static_assert(sizeof(StackHeader) == 64, "header is 64 bytes");
 
@@ -69,7 +73,8 @@ inline size_t stack_ws_bytes(int count, int n_ctas, int MP) {
 
 cudaError_t stack_w4a16_launch(const StackHeader& H, const void* plan_dev, const StackWorkspace& ws, uint32_t* status,
                                cudaStream_t stream);
-// shared memory of one CTA for a ring of `slots` quanta and partial sums of `max_quanta` quanta
-size_t stack_w4a16_smem(int group, int MP, int slots, int max_quanta);
+// shared memory of one CTA: the plan's `count` descriptors, a ring of `slots` quanta, the
+// partial sums of `max_quanta` quanta and `xs_bytes` of staged activations
+size_t stack_w4a16_smem(int group, int MP, int count, int slots, int max_quanta, int xs_bytes);
 
 }  // namespace mnnllm

@@ -46,6 +46,12 @@ __device__ __forceinline__ unsigned long long ld_relaxed_u64(const unsigned long
 __device__ __forceinline__ void st_relaxed_u64(unsigned long long* p, unsigned long long v) {
     asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
 }
+// generic-address load that is not served from a stale L1 line (shared or global memory)
+__device__ __forceinline__ uint4 ld_volatile_v4(const uint4* p) {
+    uint4 v;
+    asm volatile("ld.volatile.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
+    return v;
+}
 __device__ __forceinline__ void red_release_add(uint32_t* p, uint32_t v) {
     asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
@@ -55,13 +61,13 @@ __device__ __forceinline__ void red_release_add(uint32_t* p, uint32_t v) {
 // With fewer runs than CTAs the first U virtual CTAs take one run each, so that consecutive small
 // problems (rotated against each other by the plan) land on different SMs.
 __device__ __forceinline__ void cta_range(int NB, int NC, int gran, int cv, int n_ctas, int& q0, int& q1) {
-    const long long U = (long long)NB * NC / gran;
-    if (U < n_ctas) {
-        q0 = cv < U ? cv * gran : 0x3fffffff;   // empty, and beyond every row block
-        q1 = cv < U ? q0 + gran : 0x3fffffff;
+    const uint32_t U = (uint32_t)(NB * NC) / (uint32_t)gran;   // the plan guarantees U * n_ctas < 2^31
+    if (U < (uint32_t)n_ctas) {
+        q0 = (uint32_t)cv < U ? cv * gran : 0x3fffffff;   // empty, and beyond every row block
+        q1 = (uint32_t)cv < U ? q0 + gran : 0x3fffffff;
     } else {
-        q0 = (int)(U * cv / n_ctas) * gran;
-        q1 = (int)(U * (cv + 1) / n_ctas) * gran;
+        q0 = (int)(U * (uint32_t)cv / (uint32_t)n_ctas) * gran;
+        q1 = (int)(U * (uint32_t)(cv + 1) / (uint32_t)n_ctas) * gran;
     }
 }
 __device__ __forceinline__ int virtual_cta(int cta, int rot, int n_ctas) {
@@ -82,8 +88,10 @@ stack_w4a16_kernel(const __grid_constant__ StackHeader H, const StackProblem* __
     const int S = H.ring_slots;
 
     uint8_t* ring = smem;
-    float* part = reinterpret_cast<float*>(smem + (size_t)S * C::QB);            // [max_quanta][MP][16]
-    uint64_t* full = reinterpret_cast<uint64_t*>(part + (size_t)H.max_quanta * MP * 16);
+    StackProblem* sD = reinterpret_cast<StackProblem*>(smem + (size_t)S * C::QB);   // the plan, read once
+    float* part = reinterpret_cast<float*>(sD + H.count);                         // [max_quanta][MP][16]
+    uint4* xs = reinterpret_cast<uint4*>(part + (size_t)H.max_quanta * MP * 16);   // staged activations
+    uint64_t* full = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(xs) + H.xs_bytes);
     uint64_t* empty = full + S;
     volatile uint32_t* dead = reinterpret_cast<volatile uint32_t*>(empty + S);   // a bounded wait gave up
 
@@ -91,6 +99,12 @@ stack_w4a16_kernel(const __grid_constant__ StackHeader H, const StackProblem* __
         for (int s = 0; s < S; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
         *dead = 0;
         fence_mbar_init();
+    }
+    {   // descriptors -> shared memory: no global-memory latency at problem boundaries
+        const uint4* src = reinterpret_cast<const uint4*>(plan);
+        uint4* dst = reinterpret_cast<uint4*>(sD);
+        const int n16 = H.count * (int)(sizeof(StackProblem) / 16);
+        for (int i = threadIdx.x; i < n16; i += blockDim.x) dst[i] = __ldg(src + i);
     }
     fence_proxy_async_smem();
     __syncthreads();
@@ -102,10 +116,11 @@ stack_w4a16_kernel(const __grid_constant__ StackHeader H, const StackProblem* __
         if (lane == 0) {
             const uint64_t stream_policy = policy_evict_first();
             int slot = 0, issued = 0;
+            const int window = H.window;
             uint32_t use_parity = 0;   // parity of (uses of this slot so far)
             bool wrapped = false;
             for (int p = 0; p < H.count; ++p) {
-                const StackProblem& D = plan[p];
+                const StackProblem& D = sD[p];
                 const int NB = D.NB, NC = D.NC, gran = D.gran;
                 int q0, q1;
                 cta_range(NB, NC, gran, virtual_cta(cta, D.rot, n_ctas), n_ctas, q0, q1);
@@ -120,6 +135,17 @@ stack_w4a16_kernel(const __grid_constant__ StackHeader H, const StackProblem* __
                         !mbar_wait_bounded(&empty[slot], use_parity ^ 1u, kMaxBarPolls)) {
                         *dead = 1;
                         atomicOr(status, 0x400u | (uint32_t)(p & 0xFF));
+                    }
+                    // Bound the copies in flight: a deep queue of weight requests in front of the memory
+                    // system delays every other access (activations, counters, fences) by its length.
+                    if (issued >= window && !*dead) {
+                        const int n0 = issued - window;
+                        const int u0 = n0 / S;
+                        if (!mbar_test_wait(&full[n0 - u0 * S], (uint32_t)u0 & 1u) &&
+                            !mbar_wait_bounded(&full[n0 - u0 * S], (uint32_t)u0 & 1u, kMaxBarPolls)) {
+                            *dead = 1;
+                            atomicOr(status, 0x400u | (uint32_t)(p & 0xFF));
+                        }
                     }
                     if (!*dead) {
                         const uint32_t bytes = (j == NC - 1) ? last_bytes : (uint32_t)C::QB;
@@ -149,7 +175,7 @@ stack_w4a16_kernel(const __grid_constant__ StackHeader H, const StackProblem* __
         const int ctid = threadIdx.x;             // 0 .. W*32-1
 
         for (int p = 0; p < H.count; ++p) {
-            const StackProblem& D = plan[p];
+            const StackProblem& D = sD[p];
             const int NB = D.NB, NC = D.NC, N = D.N, K = D.K;
             int q0, q1;
             const int cv = virtual_cta(cta, D.rot, n_ctas);
@@ -159,29 +185,48 @@ stack_w4a16_kernel(const __grid_constant__ StackHeader H, const StackProblem* __
             const int weff = D.weff;
             const int last_ns = D.NS - 8 * (NC - 1);
 
-            if (warp < weff && warp < n) {
-                // ---- dependencies: the problems whose outputs (or side effects) x depends on ----
-                const int n_deps = D.n_deps;
-                if (n_deps > 0) {
-                    if (lane == 0 && !*dead) {
-                        for (int d = 0; d < n_deps; ++d) {
-                            const int dp = D.deps[d];
-                            const uint32_t target = tag * (uint32_t)plan[dp].NB;
-                            const uint32_t* f = ws.flags + dp;
-                            bool ok = false;
-                            for (uint32_t it = 0; it < kMaxFlagPolls; ++it) {
-                                if (ld_acquire_u32(f) == target) { ok = true; break; }
-                                if ((it & 255u) == 255u && *dead) break;
-                            }
-                            if (!ok) {
-                                if (!*dead) atomicOr(status, 0x100u | (uint32_t)(p & 0xFF));
-                                *dead = 1;
-                                break;
-                            }
+            // ---- dependencies: the problems whose outputs (or side effects) x depends on.  ONE thread of
+            // the CTA polls their counters: a counter polled by every warp of every SM is a hot spot ----
+            const int n_deps = D.n_deps;
+            if (n_deps > 0) {
+                if (ctid == 0 && !*dead) {
+                    for (int d = 0; d < n_deps; ++d) {
+                        const uint32_t target = tag * (uint32_t)D.deps_nb[d];
+                        const uint32_t* f = ws.flags + D.deps[d];
+                        bool ok = false;
+                        for (uint32_t it = 0; it < kMaxFlagPolls; ++it) {
+                            if (ld_acquire_u32(f) == target) { ok = true; break; }
+                            if ((it & 255u) == 255u && *dead) break;
+                        }
+                        if (!ok) {
+                            if (!*dead) atomicOr(status, 0x100u | (uint32_t)(p & 0xFF));
+                            *dead = 1;
+                            break;
                         }
                     }
-                    __syncwarp();
                 }
+                bar_sync(1, W * 32);
+            }
+            // ---- the k-chunks of x this CTA needs -> shared memory, each 16-byte piece fetched once per
+            // SM (read past L1: another SM may have written x during this launch) ----
+            const int nch = n < NC ? n : NC;                 // distinct chunks among the CTA's quanta
+            const int j_first = n < NC ? q0 % NC : 0;
+            const bool staged = D.stage_x != 0;
+            if (staged) {
+                const int pieces = nch * H.M * 64;
+                for (int idx = ctid; idx < pieces; idx += W * 32) {
+                    const int cl = idx / (H.M * 64), rem = idx - cl * (H.M * 64);
+                    const int tok = rem >> 6, piece = rem & 63;
+                    int j = j_first + cl;
+                    j = j >= NC ? j - NC : j;
+                    const int k = j * kChunkK + piece * 8;
+                    if (k < K)
+                        xs[idx] = __ldcg(reinterpret_cast<const uint4*>(reinterpret_cast<const __half*>(D.x) + (size_t)tok * K + k));
+                }
+                bar_sync(1, W * 32);
+            }
+
+            if (warp < weff && warp < n) {
                 const __half* xbase = reinterpret_cast<const __half*>(D.x);
                 int cur_j = -1;
                 for (int i = warp; i < n; i += weff) {
@@ -193,7 +238,12 @@ stack_w4a16_kernel(const __grid_constant__ StackHeader H, const StackProblem* __
                         cur_j = j;
                         // ---- activations of k-chunk j -> B fragments and per-group sums (read past L1:
                         // another SM may have written them during this launch) ----
-                        const __half* xk = xbase + (size_t)j * kChunkK;
+                        int cl = j - j_first;
+                        cl = cl < 0 ? cl + NC : cl;
+                        // generic pointers: the staged copy in shared memory, or x itself in global memory
+                        const __half* xk = staged ? reinterpret_cast<const __half*>(xs) + (size_t)cl * H.M * kChunkK
+                                                  : xbase + (size_t)j * kChunkK;
+                        const size_t xrow = staged ? (size_t)kChunkK : (size_t)K;   // distance between tokens
                         // a lane holds the slabs of its groups gsB + GPS * s only (other B entries are zero)
                         float lo[C::NSETS], hi[C::NSETS];
                         uint32_t Pm[C::NSETS][C::SPG][4][2];
@@ -206,9 +256,9 @@ stack_w4a16_kernel(const __grid_constant__ StackHeader H, const StackProblem* __
                                 uint4 u0 = make_uint4(0, 0, 0, 0), u1 = u0;
                                 if (sl < ns && tokB < H.M) {
                                     const uint4* px =
-                                        reinterpret_cast<const uint4*>(xk + (size_t)tokB * K + sl * kSlabK4 + 16 * c);
-                                    u0 = __ldcg(px);
-                                    u1 = __ldcg(px + 1);
+                                        reinterpret_cast<const uint4*>(xk + (size_t)tokB * xrow + sl * kSlabK4 + 16 * c);
+                                    u0 = ld_volatile_v4(px);
+                                    u1 = ld_volatile_v4(px + 1);
                                 }
                                 Pm[s][sp][0][0] = __byte_perm(u0.x, u0.y, 0x5410);
                                 Pm[s][sp][0][1] = __byte_perm(u0.z, u0.w, 0x5410);
@@ -363,8 +413,7 @@ stack_w4a16_kernel(const __grid_constant__ StackHeader H, const StackProblem* __
             if (ctid == 0) {
                 const int stored = (q1 + NC - 1) / NC - (q0 + NC - 1) / NC;
                 if (stored > 0) {
-                    __threadfence();
-                    red_release_add(ws.flags + p, (uint32_t)stored);
+                    red_release_add(ws.flags + p, (uint32_t)stored);   // release: the CTA's stores come first
                 }
             }
         }
@@ -383,9 +432,10 @@ stack_w4a16_kernel(const __grid_constant__ StackHeader H, const StackProblem* __
 }
 
 template <int GROUP, int MP>
-size_t smem_of(int slots, int max_quanta) {
+size_t smem_of(int count, int slots, int max_quanta, int xs_bytes) {
     using C = Cfg<GROUP, MP>;
-    return (size_t)slots * C::QB + (size_t)max_quanta * MP * 16 * 4 + (size_t)2 * slots * 8 + 16;
+    return (size_t)slots * C::QB + (size_t)count * sizeof(StackProblem) + (size_t)max_quanta * MP * 16 * 4 +
+           (size_t)xs_bytes + (size_t)2 * slots * 8 + 16;
 }
 
 template <int GROUP, int MP>
@@ -418,8 +468,8 @@ cudaError_t launch_one(const StackHeader& H, const void* plan_dev, const StackWo
 
 }  // namespace
 
-size_t stack_w4a16_smem(int group, int MP, int slots, int max_quanta) {
-#define MNN_CASE(G, P) if (group == G && MP == P) return smem_of<G, P>(slots, max_quanta);
+size_t stack_w4a16_smem(int group, int MP, int count, int slots, int max_quanta, int xs_bytes) {
+#define MNN_CASE(G, P) if (group == G && MP == P) return smem_of<G, P>(count, slots, max_quanta, xs_bytes);
     MNN_CASE(64, 1) MNN_CASE(64, 2) MNN_CASE(64, 4) MNN_CASE(64, 8)
     MNN_CASE(128, 1) MNN_CASE(128, 2) MNN_CASE(128, 4) MNN_CASE(128, 8)
 #undef MNN_CASE
