@@ -58,11 +58,6 @@ int mnnllm_stack_plan_w4a16(const mnnllm_stack_problem* problems, int count, int
     const int MP = mp_of(M);
     const int W = kStackConsumerWarps;
 
-    StackHeader H;
-    std::memset(&H, 0, sizeof(H));
-    StackProblem* out = reinterpret_cast<StackProblem*>((uint8_t*)plan_out + sizeof(StackHeader));
-    long long max_quanta = 1, xs_bytes = 0;
-    int rot = 0;
     for (int p = 0; p < count; ++p) {
         const mnnllm_stack_problem& q = problems[p];
         if (!q.x || !q.packed || !q.y || q.N < 1 || q.K < 1) return MNNLLM_ERR_INVALID_ARG;
@@ -72,16 +67,68 @@ int mnnllm_stack_plan_w4a16(const mnnllm_stack_problem* problems, int count, int
         if (q.n_deps < 0 || q.n_deps > MNNLLM_STACK_MAX_DEPS) return MNNLLM_ERR_INVALID_ARG;
         for (int d = 0; d < q.n_deps; ++d)
             if (q.deps[d] < 0 || q.deps[d] >= p) return MNNLLM_ERR_INVALID_ARG;   // only earlier problems
+    }
 
-        const W4Geometry g = w4_geometry(q.N, q.K, group);
-        StackProblem D;
-        std::memset(&D, 0, sizeof(D));
-        D.packed = (const uint8_t*)q.packed;
-        D.x = q.x;
-        D.y = q.y;
-        D.row_block_bytes = g.row_block_bytes;
-        D.N = q.N; D.K = q.K;
-        D.NB = g.n_row_blocks; D.NC = g.n_chunks; D.NS = g.n_slabs;
+    StackHeader H;
+    std::memset(&H, 0, sizeof(H));
+    StackProblem* out = reinterpret_cast<StackProblem*>((uint8_t*)plan_out + sizeof(StackHeader));
+    std::memset(out, 0, (size_t)count * sizeof(StackProblem));
+    int fused_of[MNNLLM_STACK_MAX_PROBLEMS];   // caller's problem -> problem of the plan
+    int n_plan = 0;
+    auto same_deps = [&](const mnnllm_stack_problem& a, const mnnllm_stack_problem& b) {
+        if (a.n_deps != b.n_deps) return false;
+        for (int i = 0; i < a.n_deps; ++i) {
+            bool found = false;
+            for (int j = 0; j < b.n_deps; ++j) found |= a.deps[i] == b.deps[j];
+            if (!found) return false;
+        }
+        return true;
+    };
+    // Neighbours in the list that read the same activations and wait for the same predecessors
+    // (q, k, v; gate, up) become ONE problem of the plan: their row blocks are dealt to the CTAs
+    // together, so they cost one pass of the problem loop instead of one each.
+    for (int p = 0; p < count;) {
+        int e = p + 1;
+        while (e < count && e - p < kStackMaxSub && problems[e].x == problems[p].x && problems[e].K == problems[p].K &&
+               same_deps(problems[e], problems[p]))
+            ++e;
+        StackProblem& D = out[n_plan];
+        const W4Geometry g0 = w4_geometry(problems[p].N, problems[p].K, group);
+        D.x = problems[p].x;
+        D.K = problems[p].K;
+        D.row_block_bytes = g0.row_block_bytes;
+        D.NC = g0.n_chunks; D.NS = g0.n_slabs;
+        int nb = 0;
+        for (int i = p; i < e; ++i) {
+            const W4Geometry g = w4_geometry(problems[i].N, problems[i].K, group);
+            nb += g.n_row_blocks;
+            D.packed[i - p] = (const uint8_t*)problems[i].packed;
+            D.y[i - p] = problems[i].y;
+            D.N[i - p] = problems[i].N;
+            D.nb_end[i - p] = nb;
+            D.y_dtypes |= problems[i].y_dtype << (8 * (i - p));
+            fused_of[i] = n_plan;
+        }
+        for (int i = e - p; i < kStackMaxSub; ++i) D.nb_end[i] = nb;
+        D.NB = nb;
+        for (int d = 0; d < problems[p].n_deps; ++d) {      // predecessors in the plan's numbering, once each
+            const int f = fused_of[problems[p].deps[d]];
+            bool have = false;
+            for (int j = 0; j < D.n_deps; ++j) have |= D.deps[j] == f;
+            if (!have) {
+                D.deps[D.n_deps] = f;
+                D.deps_nb[D.n_deps] = out[f].NB;
+                ++D.n_deps;
+            }
+        }
+        ++n_plan;
+        p = e;
+    }
+
+    long long max_quanta = 1, xs_bytes = 0;
+    int rot = 0;
+    for (int p = 0; p < n_plan; ++p) {
+        StackProblem& D = out[p];
         D.weff = D.NC <= W ? (W / D.NC) * D.NC : W;
         // Whole 16-row blocks per CTA (no exchange between CTAs) or runs of single quanta (even
         // shares, blocks shared between neighbours): whichever needs fewer rounds of the CTA's
@@ -102,21 +149,14 @@ int mnnllm_stack_plan_w4a16(const mnnllm_stack_problem* problems, int count, int
         // consecutive small problems start on different SMs
         D.rot = rot;
         rot = (int)((rot + (U < n_sms ? U : 0)) % n_sms);
-        D.y_dtype = q.y_dtype;
-        D.n_deps = q.n_deps;
-        for (int d = 0; d < q.n_deps; ++d) {
-            D.deps[d] = q.deps[d];
-            D.deps_nb[d] = out[q.deps[d]].NB;
-        }
-        out[p] = D;
     }
     // the ring takes what the partial sums leave of the CTA's shared memory
     int slots = 0;
     for (int s = 1; s <= 96; ++s)
-        if (stack_w4a16_smem(group, MP, count, s, (int)max_quanta, (int)xs_bytes) <= kSmemBudget) slots = s;
+        if (stack_w4a16_smem(group, MP, n_plan, s, (int)max_quanta, (int)xs_bytes) <= kSmemBudget) slots = s;
     if (slots < 2) return MNNLLM_ERR_UNSUPPORTED;   // a problem too large for M <= 8 at this shape
     H.magic = kStackMagic; H.version = 1;
-    H.count = count; H.M = M; H.group = group; H.MP = MP;
+    H.count = n_plan; H.M = M; H.group = group; H.MP = MP;
     H.n_ctas = n_sms;
     H.ring_slots = slots;
     H.max_quanta = (int32_t)max_quanta;
@@ -127,7 +167,7 @@ int mnnllm_stack_plan_w4a16(const mnnllm_stack_problem* problems, int count, int
         if (v >= 1) H.window = v;
     }
     if (H.window >= slots) H.window = slots - 1;
-    H.smem_bytes = (uint32_t)stack_w4a16_smem(group, MP, count, slots, (int)max_quanta, (int)xs_bytes);
+    H.smem_bytes = (uint32_t)stack_w4a16_smem(group, MP, n_plan, slots, (int)max_quanta, (int)xs_bytes);
     std::memcpy(plan_out, &H, sizeof(H));
     return MNNLLM_OK;
 }

@@ -22,31 +22,37 @@ namespace mnnllm {
 
 constexpr uint32_t kStackMagic = 0x4B54534Du;  // "MSTK"
 constexpr int kStackMaxDeps = 4;
-constexpr int kStackConsumerWarps = 14;   // + 1 producer warp: 480 threads, 136 registers each
-constexpr int kStackThreads = (kStackConsumerWarps + 1) * 32;
+constexpr int kStackConsumerWarps = 14;   // + producer warp + signaller warp: 512 threads, 128 registers each
+constexpr int kStackThreads = (kStackConsumerWarps + 2) * 32;
 
-struct StackProblem {            // 112 bytes, 16-byte aligned
-    const uint8_t* packed;       // packed buffer (header included)
-    const void* x;               // fp16 [M, K]
-    void* y;                     // [M, N] of y_dtype
+constexpr int kStackMaxSub = 4;           // weight matrices fused into one problem (q+k+v, gate+up)
+
+// One problem of the plan: up to kStackMaxSub weight matrices that multiply the same activations and
+// wait for the same predecessors; their 16-row blocks are numbered through (matrix 0 first).
+struct StackProblem {            // 192 bytes, 16-byte aligned
+    const uint8_t* packed[kStackMaxSub];   // packed buffers (header included)
+    void* y[kStackMaxSub];                 // [M, N[i]] of the matrix's output dtype
+    const void* x;                         // fp16 [M, K]
     unsigned long long row_block_bytes;
-    int N, K;
-    int NB, NC, NS;              // 16-row blocks, 512-k chunks, 64-k slabs per row
+    int N[kStackMaxSub];
+    int nb_end[kStackMaxSub];    // row blocks of matrices 0..i (cumulative); unused entries = NB
+    int K;
+    int NB, NC, NS;              // 16-row blocks (all matrices), 512-k chunks, 64-k slabs per row
     int gran;                    // CTAs receive runs of quanta that are multiples of gran (1 or NC)
     int rot;                     // CTA `cta` plays the role of virtual CTA (cta - rot) mod n_ctas
     int weff;                    // consumer warps used (a multiple of NC where NC <= the warp count)
-    int y_dtype;
+    int y_dtypes;                // output dtype of matrix i in bits 8i .. 8i+7
     int n_deps;
-    int deps[kStackMaxDeps];     // earlier problems that must be complete before x is read
-    int deps_nb[kStackMaxDeps];  // their row-block counts (the completion counter's increment per launch)
     int stage_x;                 // 1: the CTA copies the k-chunks of x it needs to shared memory first
-    int pad[1];
+    int deps[kStackMaxDeps];     // earlier problems (of the plan) that must be complete before x is read
+    int deps_nb[kStackMaxDeps];  // their row-block counts (the completion counter's increment per launch)
+    int pad[2];
 };
-static_assert(sizeof(StackProblem) == 112, "descriptor is 112 bytes");
+static_assert(sizeof(StackProblem) == 192, "descriptor is 192 bytes");
 
 struct StackHeader {             // 64 bytes
     uint32_t magic, version;
-    int32_t count, M, group, MP;
+    int32_t count, M, group, MP; // count = problems of the plan (after fusing matrices that share x)
     int32_t n_ctas;              // grid size the plan was made for
     int32_t ring_slots;          // quanta slots of the shared-memory ring
     int32_t max_quanta;          // most quanta one CTA holds of any one problem

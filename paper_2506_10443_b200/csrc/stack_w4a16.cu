@@ -52,6 +52,14 @@ __device__ __forceinline__ uint4 ld_volatile_v4(const uint4* p) {
     asm volatile("ld.volatile.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
     return v;
 }
+__device__ __forceinline__ uint32_t ld_acquire_cta_u32(const uint32_t* smem_word) {
+    uint32_t v;
+    asm volatile("ld.acquire.cta.shared.u32 %0, [%1];" : "=r"(v) : "r"(smem_u32(smem_word)) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release_cta_u32(uint32_t* smem_word, uint32_t v) {
+    asm volatile("st.release.cta.shared.u32 [%0], %1;" ::"r"(smem_u32(smem_word)), "r"(v) : "memory");
+}
 __device__ __forceinline__ void red_release_add(uint32_t* p, uint32_t v) {
     asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
@@ -91,13 +99,17 @@ stack_w4a16_kernel(const __grid_constant__ StackHeader H, const StackProblem* __
     StackProblem* sD = reinterpret_cast<StackProblem*>(smem + (size_t)S * C::QB);   // the plan, read once
     float* part = reinterpret_cast<float*>(sD + H.count);                         // [max_quanta][MP][16]
     uint4* xs = reinterpret_cast<uint4*>(part + (size_t)H.max_quanta * MP * 16);   // staged activations
-    uint64_t* full = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(xs) + H.xs_bytes);
+    // per staged (chunk, token): GC pairs (1024 X_lo + 64 X_hi, X_lo + X_hi) of the group sums of x
+    float2* xsum = reinterpret_cast<float2*>(reinterpret_cast<uint8_t*>(xs) + H.xs_bytes);
+    uint64_t* full = reinterpret_cast<uint64_t*>(xsum + (size_t)(H.xs_bytes / 1024) * C::GC);
     uint64_t* empty = full + S;
     volatile uint32_t* dead = reinterpret_cast<volatile uint32_t*>(empty + S);   // a bounded wait gave up
+    uint32_t* finished = const_cast<uint32_t*>(dead) + 1;   // problems whose outputs this CTA has stored (mailbox)
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
         *dead = 0;
+        *finished = 0;
         fence_mbar_init();
     }
     {   // descriptors -> shared memory: no global-memory latency at problem boundaries
@@ -125,11 +137,13 @@ stack_w4a16_kernel(const __grid_constant__ StackHeader H, const StackProblem* __
                 int q0, q1;
                 cta_range(NB, NC, gran, virtual_cta(cta, D.rot, n_ctas), n_ctas, q0, q1);
                 if (q0 >= q1) continue;
-                const uint8_t* body = D.packed + kHeaderBytes;
                 const unsigned long long rbb = D.row_block_bytes;
                 const int last_ns = D.NS - 8 * (NC - 1);
                 const uint32_t last_bytes = (uint32_t)(last_ns * kSlabBytes + 16 * (last_ns / C::SPG) * 4);
                 int rb = q0 / NC, j = q0 - rb * NC;
+                int sub = 0;
+                while (rb >= D.nb_end[sub]) ++sub;            // the matrix that row block rb belongs to
+                const uint8_t* body = D.packed[sub] + kHeaderBytes - (size_t)(sub ? D.nb_end[sub - 1] : 0) * rbb;
                 for (int q = q0; q < q1; ++q) {
                     if (wrapped && !*dead && !mbar_test_wait(&empty[slot], use_parity ^ 1u) &&
                         !mbar_wait_bounded(&empty[slot], use_parity ^ 1u, kMaxBarPolls)) {
@@ -155,7 +169,14 @@ stack_w4a16_kernel(const __grid_constant__ StackHeader H, const StackProblem* __
                         ++issued;
                     }
                     if (++slot == S) { slot = 0; use_parity ^= 1u; wrapped = true; }
-                    if (++j == NC) { j = 0; ++rb; }
+                    if (++j == NC) {
+                        j = 0;
+                        ++rb;
+                        if (rb >= D.nb_end[sub] && rb < NB) {
+                            while (rb >= D.nb_end[sub]) ++sub;
+                            body = D.packed[sub] + kHeaderBytes - (size_t)D.nb_end[sub - 1] * rbb;
+                        }
+                    }
                 }
             }
             // no bulk copy may still be in flight into this CTA's shared memory when it exits
@@ -165,6 +186,30 @@ stack_w4a16_kernel(const __grid_constant__ StackHeader H, const StackProblem* __
                     break;
                 }
         }
+    } else if (warp == W + 1) {
+        // =================== signaller: publishes "problem p complete" off the consumers' critical path ===========
+        // The release-ordered add waits until the CTA's output stores are visible GPU-wide (most of a
+        // microsecond); the consumers only leave a note in shared memory and move on.
+        if (lane == 0) {
+            uint32_t seen = 0;
+            for (int p = 0; p < H.count; ++p) {
+                const StackProblem& D = sD[p];
+                const int NC = D.NC;
+                int q0, q1;
+                cta_range(D.NB, NC, D.gran, virtual_cta(cta, D.rot, n_ctas), n_ctas, q0, q1);
+                if (q0 >= q1) continue;
+                const int stored = (q1 + NC - 1) / NC - (q0 + NC - 1) / NC;   // row blocks whose first quantum is here
+                ++seen;
+                bool ok = false;
+                for (uint32_t it = 0; it < (1u << 24); ++it) {
+                    if (ld_acquire_cta_u32(finished) >= seen) { ok = true; break; }
+                    if (*dead) break;
+                    __nanosleep(20);
+                }
+                if (!ok) break;   // a wait elsewhere in the CTA gave up (or this one did: ~0.5 s)
+                if (stored > 0) red_release_add(ws.flags + p, (uint32_t)stored);
+            }
+        }
     } else {
         // =================== consumers ===================
         const int r = lane >> 2, c = lane & 3;
@@ -172,11 +217,12 @@ stack_w4a16_kernel(const __grid_constant__ StackHeader H, const StackProblem* __
         uint32_t B[8][4][2];
         float C1[C::NSETS][2], C2[C::NSETS][2];
         int seq_base = 0;                         // quanta of earlier problems that went through this CTA's ring
+        uint32_t n_finished = 0;                  // problems this CTA has stored outputs of
         const int ctid = threadIdx.x;             // 0 .. W*32-1
 
         for (int p = 0; p < H.count; ++p) {
             const StackProblem& D = sD[p];
-            const int NB = D.NB, NC = D.NC, N = D.N, K = D.K;
+            const int NB = D.NB, NC = D.NC, K = D.K;
             int q0, q1;
             const int cv = virtual_cta(cta, D.rot, n_ctas);
             cta_range(NB, NC, D.gran, cv, n_ctas, q0, q1);
@@ -213,15 +259,27 @@ stack_w4a16_kernel(const __grid_constant__ StackHeader H, const StackProblem* __
             const int j_first = n < NC ? q0 % NC : 0;
             const bool staged = D.stage_x != 0;
             if (staged) {
-                const int pieces = nch * H.M * 64;
+                // piece = 8 consecutive k (16 bytes); 8 * SPG consecutive pieces = one group, held by
+                // neighbouring lanes, which add up the group's sums of x on the way
+                const int pieces = nch * H.M * 64;   // a multiple of 64: whole warps run each iteration
                 for (int idx = ctid; idx < pieces; idx += W * 32) {
                     const int cl = idx / (H.M * 64), rem = idx - cl * (H.M * 64);
                     const int tok = rem >> 6, piece = rem & 63;
                     int j = j_first + cl;
                     j = j >= NC ? j - NC : j;
                     const int k = j * kChunkK + piece * 8;
-                    if (k < K)
-                        xs[idx] = __ldcg(reinterpret_cast<const uint4*>(reinterpret_cast<const __half*>(D.x) + (size_t)tok * K + k));
+                    uint4 u = make_uint4(0, 0, 0, 0);
+                    if (k < K) u = __ldcg(reinterpret_cast<const uint4*>(reinterpret_cast<const __half*>(D.x) + (size_t)tok * K + k));
+                    xs[idx] = u;
+                    const float2 a0 = h2f2(u.x), a1 = h2f2(u.y), b0 = h2f2(u.z), b1 = h2f2(u.w);
+                    float lo = (a0.x + a0.y) + (a1.x + a1.y), hi = (b0.x + b0.y) + (b1.x + b1.y);
+#pragma unroll
+                    for (int m = 1; m < 8 * C::SPG; m <<= 1) {
+                        lo += __shfl_xor_sync(0xffffffffu, lo, m);
+                        hi += __shfl_xor_sync(0xffffffffu, hi, m);
+                    }
+                    if ((piece & (8 * C::SPG - 1)) == 0)
+                        xsum[(size_t)(idx >> 6) * C::GC + piece / (8 * C::SPG)] = make_float2(1024.f * lo + 64.f * hi, lo + hi);
                 }
                 bar_sync(1, W * 32);
             }
@@ -268,15 +326,17 @@ stack_w4a16_kernel(const __grid_constant__ StackHeader H, const StackProblem* __
                                 Pm[s][sp][2][1] = __byte_perm(u1.z, u1.w, 0x5410);
                                 Pm[s][sp][3][0] = __byte_perm(u1.x, u1.y, 0x7632);
                                 Pm[s][sp][3][1] = __byte_perm(u1.z, u1.w, 0x7632);
-                                float2 f;
-                                f = h2f2(u0.x); lo[s] += f.x + f.y;
-                                f = h2f2(u0.y); lo[s] += f.x + f.y;
-                                f = h2f2(u1.x); lo[s] += f.x + f.y;
-                                f = h2f2(u1.y); lo[s] += f.x + f.y;
-                                f = h2f2(u0.z); hi[s] += f.x + f.y;
-                                f = h2f2(u0.w); hi[s] += f.x + f.y;
-                                f = h2f2(u1.z); hi[s] += f.x + f.y;
-                                f = h2f2(u1.w); hi[s] += f.x + f.y;
+                                if (!staged) {   // the staged copy comes with its group sums
+                                    float2 f;
+                                    f = h2f2(u0.x); lo[s] += f.x + f.y;
+                                    f = h2f2(u0.y); lo[s] += f.x + f.y;
+                                    f = h2f2(u1.x); lo[s] += f.x + f.y;
+                                    f = h2f2(u1.y); lo[s] += f.x + f.y;
+                                    f = h2f2(u0.z); hi[s] += f.x + f.y;
+                                    f = h2f2(u0.w); hi[s] += f.x + f.y;
+                                    f = h2f2(u1.z); hi[s] += f.x + f.y;
+                                    f = h2f2(u1.w); hi[s] += f.x + f.y;
+                                }
                             }
                         }
 #pragma unroll
@@ -289,6 +349,19 @@ stack_w4a16_kernel(const __grid_constant__ StackHeader H, const StackProblem* __
                                 for (int b = 0; b < 2; ++b)
                                     B[sl][a][b] = mine ? Pm[gi / C::GPS][sl % C::SPG][a][b] : 0u;
                         }
+                        if (staged) {
+                            // correction terms of accumulator column 2c + e = (token, group slot) of tile s
+#pragma unroll
+                            for (int s = 0; s < C::NSETS; ++s)
+#pragma unroll
+                                for (int e = 0; e < 2; ++e) {
+                                    const int tok = (2 * c + e) % MP, gi = s * C::GPS + (2 * c + e) / MP;
+                                    float2 v = make_float2(0.f, 0.f);
+                                    if (tok < H.M && gi < ng) v = xsum[((size_t)cl * H.M + tok) * C::GC + gi];
+                                    C1[s][e] = v.x;
+                                    C2[s][e] = v.y;
+                                }
+                        } else
 #pragma unroll
                         for (int s = 0; s < C::NSETS; ++s) {
                             float l = lo[s], h = hi[s];
@@ -405,17 +478,15 @@ stack_w4a16_kernel(const __grid_constant__ StackHeader H, const StackProblem* __
                         acc += __uint_as_float((uint32_t)v);
                     }
                 }
-                const int nrow = rb * 16 + row;
-                if (nrow < N && tok < H.M) store_out(D.y, D.y_dtype, (size_t)tok * N + nrow, acc);
+                int sub = 0;
+                while (rb >= D.nb_end[sub]) ++sub;            // the matrix that row block rb belongs to
+                const int nrow = (rb - (sub ? D.nb_end[sub - 1] : 0)) * 16 + row, Ns = D.N[sub];
+                if (nrow < Ns && tok < H.M)
+                    store_out(D.y[sub], (D.y_dtypes >> (8 * sub)) & 0xFF, (size_t)tok * Ns + nrow, acc);
             }
             // ---- completion: row blocks whose first quantum this CTA holds were stored by it ----
             bar_sync(1, W * 32);
-            if (ctid == 0) {
-                const int stored = (q1 + NC - 1) / NC - (q0 + NC - 1) / NC;
-                if (stored > 0) {
-                    red_release_add(ws.flags + p, (uint32_t)stored);   // release: the CTA's stores come first
-                }
-            }
+            if (ctid == 0) st_release_cta_u32(finished, ++n_finished);   // the signaller warp takes it from here
         }
     }
 
@@ -435,7 +506,7 @@ template <int GROUP, int MP>
 size_t smem_of(int count, int slots, int max_quanta, int xs_bytes) {
     using C = Cfg<GROUP, MP>;
     return (size_t)slots * C::QB + (size_t)count * sizeof(StackProblem) + (size_t)max_quanta * MP * 16 * 4 +
-           (size_t)xs_bytes + (size_t)2 * slots * 8 + 16;
+           (size_t)xs_bytes + (size_t)(xs_bytes / 1024) * C::GC * 8 + (size_t)2 * slots * 8 + 16;
 }
 
 template <int GROUP, int MP>
