@@ -57,8 +57,8 @@ struct StackHeader {             // 64 bytes
     int32_t ring_slots;          // quanta slots of the shared-memory ring
     int32_t max_quanta;          // most quanta one CTA holds of any one problem
     uint32_t smem_bytes;
-    int32_t window;              // bulk copies a CTA keeps in flight at most
     uint32_t xs_bytes;           // shared memory for staged activations
+    int32_t producer_lanes;      // lanes of the producer warp that issue copies; divides ring_slots
     uint32_t reserved[4];
 };
 static_assert(sizeof(StackHeader) == 64, "header is 64 bytes");

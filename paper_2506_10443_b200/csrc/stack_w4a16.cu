@@ -125,66 +125,62 @@ stack_w4a16_kernel(const __grid_constant__ StackHeader H, const StackProblem* __
 
     if (warp == W) {
         // =================== producer: every problem's weights, in order, never waits for x ===================
-        if (lane == 0) {
-            const uint64_t stream_policy = policy_evict_first();
-            int slot = 0, issued = 0;
-            const int window = H.window;
-            uint32_t use_parity = 0;   // parity of (uses of this slot so far)
-            bool wrapped = false;
-            for (int p = 0; p < H.count; ++p) {
-                const StackProblem& D = sD[p];
-                const int NB = D.NB, NC = D.NC, gran = D.gran;
-                int q0, q1;
-                cta_range(NB, NC, gran, virtual_cta(cta, D.rot, n_ctas), n_ctas, q0, q1);
-                if (q0 >= q1) continue;
-                const unsigned long long rbb = D.row_block_bytes;
-                const int last_ns = D.NS - 8 * (NC - 1);
-                const uint32_t last_bytes = (uint32_t)(last_ns * kSlabBytes + 16 * (last_ns / C::SPG) * 4);
-                int rb = q0 / NC, j = q0 - rb * NC;
+        // One thread cannot issue copies fast enough (a copy costs it some hundreds of cycles of waits
+        // and address arithmetic), so the warp's 32 lanes take the CTA's quanta round-robin.
+        const uint64_t stream_policy = policy_evict_first();
+        int seq_base = 0;   // quanta of earlier problems
+        // Lane L issues the copies whose sequence number is L modulo PL, and PL divides the slot count:
+        // every use of a slot is issued by the same lane, in order, so that a lane's wait for "the
+        // previous occupant has been read" always refers to the barrier phase it means (a parity wait
+        // issued two phases early would succeed at once).
+        const int PL = H.producer_lanes;
+        for (int p = 0; p < H.count && lane < PL; ++p) {
+            const StackProblem& D = sD[p];
+            const int NB = D.NB, NC = D.NC;
+            int q0, q1;
+            cta_range(NB, NC, D.gran, virtual_cta(cta, D.rot, n_ctas), n_ctas, q0, q1);
+            if (q0 >= q1) continue;
+            const unsigned long long rbb = D.row_block_bytes;
+            const int last_ns = D.NS - 8 * (NC - 1);
+            const uint32_t last_bytes = (uint32_t)(last_ns * kSlabBytes + 16 * (last_ns / C::SPG) * 4);
+            int first = lane - seq_base % PL;
+            first = first < 0 ? first + PL : first;
+            for (int q = q0 + first; q < q1; q += PL) {
+                const int seq = seq_base + (q - q0);
+                const int use = seq / S, slot = seq - use * S;
+                const int rb = q / NC, j = q - rb * NC;
                 int sub = 0;
                 while (rb >= D.nb_end[sub]) ++sub;            // the matrix that row block rb belongs to
-                const uint8_t* body = D.packed[sub] + kHeaderBytes - (size_t)(sub ? D.nb_end[sub - 1] : 0) * rbb;
-                for (int q = q0; q < q1; ++q) {
-                    if (wrapped && !*dead && !mbar_test_wait(&empty[slot], use_parity ^ 1u) &&
-                        !mbar_wait_bounded(&empty[slot], use_parity ^ 1u, kMaxBarPolls)) {
-                        *dead = 1;
-                        atomicOr(status, 0x400u | (uint32_t)(p & 0xFF));
-                    }
-                    // Bound the copies in flight: a deep queue of weight requests in front of the memory
-                    // system delays every other access (activations, counters, fences) by its length.
-                    if (issued >= window && !*dead) {
-                        const int n0 = issued - window;
-                        const int u0 = n0 / S;
-                        if (!mbar_test_wait(&full[n0 - u0 * S], (uint32_t)u0 & 1u) &&
-                            !mbar_wait_bounded(&full[n0 - u0 * S], (uint32_t)u0 & 1u, kMaxBarPolls)) {
-                            *dead = 1;
-                            atomicOr(status, 0x400u | (uint32_t)(p & 0xFF));
-                        }
-                    }
-                    if (!*dead) {
-                        const uint32_t bytes = (j == NC - 1) ? last_bytes : (uint32_t)C::QB;
-                        mbar_arrive_expect_tx(&full[slot], bytes);
-                        bulk_g2s_hint(ring + (size_t)slot * C::QB, body + (size_t)rb * rbb + (size_t)j * C::QB, bytes,
-                                      &full[slot], stream_policy);
-                        ++issued;
-                    }
-                    if (++slot == S) { slot = 0; use_parity ^= 1u; wrapped = true; }
-                    if (++j == NC) {
-                        j = 0;
-                        ++rb;
-                        if (rb >= D.nb_end[sub] && rb < NB) {
-                            while (rb >= D.nb_end[sub]) ++sub;
-                            body = D.packed[sub] + kHeaderBytes - (size_t)D.nb_end[sub - 1] * rbb;
-                        }
-                    }
+                const uint8_t* src = D.packed[sub] + kHeaderBytes + (size_t)(rb - (sub ? D.nb_end[sub - 1] : 0)) * rbb +
+                                     (size_t)j * C::QB;
+                // the slot's previous occupant must have been read
+                if (use > 0 && !*dead && !mbar_test_wait(&empty[slot], (uint32_t)(use - 1) & 1u) &&
+                    !mbar_wait_bounded(&empty[slot], (uint32_t)(use - 1) & 1u, kMaxBarPolls)) {
+                    *dead = 1;
+                    atomicOr(status, 0x400u | (uint32_t)(p & 0xFF));
+                }
+                if (!*dead) {
+                    const uint32_t bytes = (j == NC - 1) ? last_bytes : (uint32_t)C::QB;
+                    mbar_arrive_expect_tx(&full[slot], bytes);
+                    bulk_g2s_hint(ring + (size_t)slot * C::QB, src, bytes, &full[slot], stream_policy);
                 }
             }
-            // no bulk copy may still be in flight into this CTA's shared memory when it exits
-            for (int n = issued > S ? issued - S : 0; n < issued; ++n)
-                if (!mbar_wait_bounded_compact(&full[n % S], (uint32_t)(n / S) & 1u, kMaxBarPolls)) {
-                    atomicOr(status, 0x800u);
-                    break;
+            seq_base += q1 - q0;
+        }
+        // no bulk copy may still be in flight into this CTA's shared memory when it exits: wait for
+        // the last use of every slot (a copy that was never issued, after a give-up, cannot be waited for)
+        if (!*dead) {
+            const int start = seq_base > S ? seq_base - S : 0;   // the last use of each slot: the last S copies
+            if (lane < PL)
+                for (int seq = start / PL * PL + lane; seq < seq_base; seq += PL) {
+                    if (seq < start) continue;
+                    if (!mbar_wait_bounded_compact(&full[seq % S], (uint32_t)(seq / S) & 1u, kMaxBarPolls)) {
+                        atomicOr(status, 0x800u);
+                        break;
+                    }
                 }
+        } else {
+            for (int i = 0; i < 50; ++i) __nanosleep(1000);   // ~50 us: far longer than a copy takes
         }
     } else if (warp == W + 1) {
         // =================== signaller: publishes "problem p complete" off the consumers' critical path ===========
@@ -284,10 +280,18 @@ stack_w4a16_kernel(const __grid_constant__ StackHeader H, const StackProblem* __
                 bar_sync(1, W * 32);
             }
 
-            if (warp < weff && warp < n) {
-                const __half* xbase = reinterpret_cast<const __half*>(D.x);
-                int cur_j = -1;
-                for (int i = warp; i < n; i += weff) {
+            // A wait on a slot tells "the copy I mean" from "the copy before it" only by a parity bit, so
+            // no warp may reach use u of a slot before use u-1 has been read: a problem with more quanta
+            // than the ring has slots is taken in batches of at most that many, a CTA barrier between them
+            // (between problems the barrier before the reduction does the same).
+            const int batch = S >= weff ? (S / weff) * weff : S;
+            const __half* xbase = reinterpret_cast<const __half*>(D.x);
+            int cur_j = -1;
+            for (int base = 0; base < n; base += batch) {
+                if (base > 0) bar_sync(1, W * 32);
+                const int end = base + batch < n ? base + batch : n;
+                if (warp < weff)
+                for (int i = base + warp; i < end; i += weff) {
                     const int q = q0 + i;
                     const int rb = q / NC, j = q - rb * NC;
                     const int ns = (j == NC - 1) ? last_ns : 8;
