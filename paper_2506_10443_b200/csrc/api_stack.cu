@@ -150,22 +150,17 @@ int mnnllm_stack_plan_w4a16(const mnnllm_stack_problem* problems, int count, int
         rot = (int)((rot + (U < n_sms ? U : 0)) % n_sms);
     }
     // the ring takes what the partial sums leave of the CTA's shared memory
-    int slots = 0, lanes = 0;
-    for (int s = 1; s <= 96; ++s)
-        if (stack_w4a16_smem(group, MP, n_plan, s, (int)max_quanta, (int)xs_bytes) <= kSmemBudget) slots = s;
-    if (slots < 2) return MNNLLM_ERR_UNSUPPORTED;   // a problem too large for M <= 8 at this shape
-    // the producer warp's lanes share the slots: a slot count with a divisor between 16 and 32
-    for (; slots >= 32 && !lanes; --slots)
-        for (int d = 32; d >= 16 && !lanes; --d)
-            if (slots % d == 0) lanes = d;
-    if (lanes) ++slots; else lanes = slots < 32 ? slots : 32;   // fewer than 32 slots: one lane each
+    // the ring takes what is left of the CTA's shared memory: the same number of slots for each consumer warp
+    int slots = 0;
+    for (int r = 1; r <= 8; ++r)
+        if (stack_w4a16_smem(group, MP, n_plan, r * W, (int)max_quanta, (int)xs_bytes) <= kSmemBudget) slots = r * W;
+    if (slots < W) return MNNLLM_ERR_UNSUPPORTED;   // a problem too large for M <= 8 at this shape
     H.magic = kStackMagic; H.version = 1;
     H.count = n_plan; H.M = M; H.group = group; H.MP = MP;
     H.n_ctas = n_sms;
     H.ring_slots = slots;
     H.max_quanta = (int32_t)max_quanta;
     H.xs_bytes = (uint32_t)xs_bytes;
-    H.producer_lanes = lanes;
     H.smem_bytes = (uint32_t)stack_w4a16_smem(group, MP, n_plan, slots, (int)max_quanta, (int)xs_bytes);
     std::memcpy(plan_out, &H, sizeof(H));
     return MNNLLM_OK;

@@ -54,12 +54,11 @@ struct StackHeader {             // 64 bytes
     uint32_t magic, version;
     int32_t count, M, group, MP; // count = problems of the plan (after fusing matrices that share x)
     int32_t n_ctas;              // grid size the plan was made for
-    int32_t ring_slots;          // quanta slots of the shared-memory ring
+    int32_t ring_slots;          // quanta slots of the shared-memory ring, a multiple of the consumer warps
     int32_t max_quanta;          // most quanta one CTA holds of any one problem
     uint32_t smem_bytes;
     uint32_t xs_bytes;           // shared memory for staged activations
-    int32_t producer_lanes;      // lanes of the producer warp that issue copies; divides ring_slots
-    uint32_t reserved[4];
+    uint32_t reserved[5];
 };
 static_assert(sizeof(StackHeader) == 64, "header is 64 bytes");
 

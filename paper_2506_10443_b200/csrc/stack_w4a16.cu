@@ -78,6 +78,11 @@ __device__ __forceinline__ void cta_range(int NB, int NC, int gran, int cv, int 
         q1 = (int)(U * (uint32_t)(cv + 1) / (uint32_t)n_ctas) * gran;
     }
 }
+// cached read of a pointer field of the (read-only) plan
+template <typename T, typename P>
+__device__ __forceinline__ T* ldg_ptr(P* const* field) {
+    return reinterpret_cast<T*>(__ldg(reinterpret_cast<const unsigned long long*>(field)));
+}
 __device__ __forceinline__ int virtual_cta(int cta, int rot, int n_ctas) {
     const int v = cta - rot;
     return v < 0 ? v + n_ctas : v;
@@ -95,9 +100,10 @@ stack_w4a16_kernel(const __grid_constant__ StackHeader H, const StackProblem* __
     const int cta = blockIdx.x, n_ctas = gridDim.x;
     const int S = H.ring_slots;
 
+    const int R = S / W;                      // every consumer warp owns R slots of the ring
     uint8_t* ring = smem;
-    StackProblem* sD = reinterpret_cast<StackProblem*>(smem + (size_t)S * C::QB);   // the plan, read once
-    float* part = reinterpret_cast<float*>(sD + H.count);                         // [max_quanta][MP][16]
+    const StackProblem* sD = plan;            // read-only for the whole launch: cached loads, prefetched ahead
+    float* part = reinterpret_cast<float*>(smem + (size_t)S * C::QB);             // [max_quanta][MP][16]
     uint4* xs = reinterpret_cast<uint4*>(part + (size_t)H.max_quanta * MP * 16);   // staged activations
     // per staged (chunk, token): GC pairs (1024 X_lo + 64 X_hi, X_lo + X_hi) of the group sums of x
     float2* xsum = reinterpret_cast<float2*>(reinterpret_cast<uint8_t*>(xs) + H.xs_bytes);
@@ -112,12 +118,6 @@ stack_w4a16_kernel(const __grid_constant__ StackHeader H, const StackProblem* __
         *finished = 0;
         fence_mbar_init();
     }
-    {   // descriptors -> shared memory: no global-memory latency at problem boundaries
-        const uint4* src = reinterpret_cast<const uint4*>(plan);
-        uint4* dst = reinterpret_cast<uint4*>(sD);
-        const int n16 = H.count * (int)(sizeof(StackProblem) / 16);
-        for (int i = threadIdx.x; i < n16; i += blockDim.x) dst[i] = __ldg(src + i);
-    }
     fence_proxy_async_smem();
     __syncthreads();
 
@@ -125,62 +125,63 @@ stack_w4a16_kernel(const __grid_constant__ StackHeader H, const StackProblem* __
 
     if (warp == W) {
         // =================== producer: every problem's weights, in order, never waits for x ===================
-        // One thread cannot issue copies fast enough (a copy costs it some hundreds of cycles of waits
-        // and address arithmetic), so the warp's 32 lanes take the CTA's quanta round-robin.
-        const uint64_t stream_policy = policy_evict_first();
-        int seq_base = 0;   // quanta of earlier problems
-        // Lane L issues the copies whose sequence number is L modulo PL, and PL divides the slot count:
-        // every use of a slot is issued by the same lane, in order, so that a lane's wait for "the
-        // previous occupant has been read" always refers to the barrier phase it means (a parity wait
-        // issued two phases early would succeed at once).
-        const int PL = H.producer_lanes;
-        for (int p = 0; p < H.count && lane < PL; ++p) {
-            const StackProblem& D = sD[p];
-            const int NB = D.NB, NC = D.NC;
-            int q0, q1;
-            cta_range(NB, NC, D.gran, virtual_cta(cta, D.rot, n_ctas), n_ctas, q0, q1);
-            if (q0 >= q1) continue;
-            const unsigned long long rbb = D.row_block_bytes;
-            const int last_ns = D.NS - 8 * (NC - 1);
-            const uint32_t last_bytes = (uint32_t)(last_ns * kSlabBytes + 16 * (last_ns / C::SPG) * 4);
-            int first = lane - seq_base % PL;
-            first = first < 0 ? first + PL : first;
-            for (int q = q0 + first; q < q1; q += PL) {
-                const int seq = seq_base + (q - q0);
-                const int use = seq / S, slot = seq - use * S;
-                const int rb = q / NC, j = q - rb * NC;
-                int sub = 0;
-                while (rb >= D.nb_end[sub]) ++sub;            // the matrix that row block rb belongs to
-                const uint8_t* src = D.packed[sub] + kHeaderBytes + (size_t)(rb - (sub ? D.nb_end[sub - 1] : 0)) * rbb +
-                                     (size_t)j * C::QB;
-                // the slot's previous occupant must have been read
-                if (use > 0 && !*dead && !mbar_test_wait(&empty[slot], (uint32_t)(use - 1) & 1u) &&
-                    !mbar_wait_bounded(&empty[slot], (uint32_t)(use - 1) & 1u, kMaxBarPolls)) {
-                    *dead = 1;
-                    atomicOr(status, 0x400u | (uint32_t)(p & 0xFF));
-                }
-                if (!*dead) {
-                    const uint32_t bytes = (j == NC - 1) ? last_bytes : (uint32_t)C::QB;
-                    mbar_arrive_expect_tx(&full[slot], bytes);
-                    bulk_g2s_hint(ring + (size_t)slot * C::QB, src, bytes, &full[slot], stream_policy);
+        // Lane L streams the quanta of consumer warp L (quantum i of a problem goes to warp i mod weff)
+        // through that warp's own R slots.  A slot is thus always filled by one lane and read by one warp,
+        // both in order, so the parity waits on its barriers can never mistake one use for another; and
+        // one thread could not issue the CTA's copies fast enough anyway.
+        if (lane < W) {
+            const uint64_t stream_policy = policy_evict_first();
+            uint8_t* my_ring = ring + (size_t)lane * R * C::QB;
+            uint64_t* my_full = full + lane * R;
+            uint64_t* my_empty = empty + lane * R;
+            int slot = 0;
+            uint32_t parity = 0;      // parity of the slot's use count
+            bool wrapped = false;
+            int issued = 0;
+            for (int p = 0; p < H.count; ++p) {
+                const StackProblem& D = sD[p];
+                const int weff = __ldg(&D.weff);
+                if (lane >= weff) continue;
+                const int NB = __ldg(&D.NB), NC = __ldg(&D.NC);
+                int q0, q1;
+                cta_range(NB, NC, __ldg(&D.gran), virtual_cta(cta, __ldg(&D.rot), n_ctas), n_ctas, q0, q1);
+                if (q0 + lane >= q1) continue;
+                const unsigned long long rbb = __ldg(&D.row_block_bytes);
+                const int last_ns = __ldg(&D.NS) - 8 * (NC - 1);
+                const uint32_t last_bytes = (uint32_t)(last_ns * kSlabBytes + 16 * (last_ns / C::SPG) * 4);
+                for (int q = q0 + lane; q < q1; q += weff) {
+                    const int rb = q / NC, j = q - rb * NC;
+                    int sub = 0;
+                    while (rb >= __ldg(&D.nb_end[sub])) ++sub;            // the matrix that row block rb belongs to
+                    const uint8_t* src = ldg_ptr<const uint8_t>(&D.packed[sub]) + kHeaderBytes +
+                                         (size_t)(rb - (sub ? __ldg(&D.nb_end[sub - 1]) : 0)) * rbb + (size_t)j * C::QB;
+                    // the slot's previous occupant must have been read
+                    if (wrapped && !*dead && !mbar_test_wait(&my_empty[slot], parity ^ 1u) &&
+                        !mbar_wait_bounded(&my_empty[slot], parity ^ 1u, kMaxBarPolls)) {
+                        *dead = 1;
+                        atomicOr(status, 0x400u | (uint32_t)(p & 0xFF));
+                    }
+                    if (!*dead) {
+                        const uint32_t bytes = (j == NC - 1) ? last_bytes : (uint32_t)C::QB;
+                        mbar_arrive_expect_tx(&my_full[slot], bytes);
+                        bulk_g2s_hint(my_ring + (size_t)slot * C::QB, src, bytes, &my_full[slot], stream_policy);
+                        ++issued;
+                    }
+                    if (++slot == R) { slot = 0; parity ^= 1u; wrapped = true; }
                 }
             }
-            seq_base += q1 - q0;
-        }
-        // no bulk copy may still be in flight into this CTA's shared memory when it exits: wait for
-        // the last use of every slot (a copy that was never issued, after a give-up, cannot be waited for)
-        if (!*dead) {
-            const int start = seq_base > S ? seq_base - S : 0;   // the last use of each slot: the last S copies
-            if (lane < PL)
-                for (int seq = start / PL * PL + lane; seq < seq_base; seq += PL) {
-                    if (seq < start) continue;
-                    if (!mbar_wait_bounded_compact(&full[seq % S], (uint32_t)(seq / S) & 1u, kMaxBarPolls)) {
+            // no bulk copy may still be in flight into this CTA's shared memory when it exits: wait for
+            // the last use of each of the lane's slots (after a give-up nothing more was issued: sleep
+            // instead, far longer than a copy takes)
+            if (!*dead) {
+                for (int n = issued > R ? issued - R : 0; n < issued; ++n)
+                    if (!mbar_wait_bounded_compact(&my_full[n % R], (uint32_t)(n / R) & 1u, kMaxBarPolls)) {
                         atomicOr(status, 0x800u);
                         break;
                     }
-                }
-        } else {
-            for (int i = 0; i < 50; ++i) __nanosleep(1000);   // ~50 us: far longer than a copy takes
+            } else {
+                for (int i = 0; i < 50; ++i) __nanosleep(1000);
+            }
         }
     } else if (warp == W + 1) {
         // =================== signaller: publishes "problem p complete" off the consumers' critical path ===========
@@ -190,9 +191,9 @@ stack_w4a16_kernel(const __grid_constant__ StackHeader H, const StackProblem* __
             uint32_t seen = 0;
             for (int p = 0; p < H.count; ++p) {
                 const StackProblem& D = sD[p];
-                const int NC = D.NC;
+                const int NC = __ldg(&D.NC);
                 int q0, q1;
-                cta_range(D.NB, NC, D.gran, virtual_cta(cta, D.rot, n_ctas), n_ctas, q0, q1);
+                cta_range(__ldg(&D.NB), NC, __ldg(&D.gran), virtual_cta(cta, __ldg(&D.rot), n_ctas), n_ctas, q0, q1);
                 if (q0 >= q1) continue;
                 const int stored = (q1 + NC - 1) / NC - (q0 + NC - 1) / NC;   // row blocks whose first quantum is here
                 ++seen;
@@ -212,29 +213,38 @@ stack_w4a16_kernel(const __grid_constant__ StackHeader H, const StackProblem* __
         const int tokB = r % MP, gsB = r / MP;   // B-operand role of this lane: column r of the MMA
         uint32_t B[8][4][2];
         float C1[C::NSETS][2], C2[C::NSETS][2];
-        int seq_base = 0;                         // quanta of earlier problems that went through this CTA's ring
         uint32_t n_finished = 0;                  // problems this CTA has stored outputs of
+        // this warp's slots of the ring, used in order across problems
+        const uint8_t* my_ring = ring + (size_t)warp * R * C::QB;
+        uint64_t* my_full = full + warp * R;
+        uint64_t* my_empty = empty + warp * R;
+        int slot = 0;
+        uint32_t parity = 0;
         const int ctid = threadIdx.x;             // 0 .. W*32-1
 
         for (int p = 0; p < H.count; ++p) {
+            // the next descriptors into L1 (192 bytes = two lines each), off the critical path
+            if (ctid < 8 && p + 1 + (ctid >> 1) < H.count)
+                asm volatile("prefetch.global.L1 [%0];" ::"l"(reinterpret_cast<const uint8_t*>(sD + p + 1 + (ctid >> 1)) + 128 * (ctid & 1)));
             const StackProblem& D = sD[p];
-            const int NB = D.NB, NC = D.NC, K = D.K;
+            const int NB = __ldg(&D.NB), NC = __ldg(&D.NC), K = __ldg(&D.K), gran = __ldg(&D.gran);
             int q0, q1;
-            const int cv = virtual_cta(cta, D.rot, n_ctas);
-            cta_range(NB, NC, D.gran, cv, n_ctas, q0, q1);
+            const int cv = virtual_cta(cta, __ldg(&D.rot), n_ctas);
+            cta_range(NB, NC, gran, cv, n_ctas, q0, q1);
             const int n = q1 - q0;
             if (n <= 0) continue;   // uniform over the CTA
-            const int weff = D.weff;
-            const int last_ns = D.NS - 8 * (NC - 1);
+            const int weff = __ldg(&D.weff);
+            const int last_ns = __ldg(&D.NS) - 8 * (NC - 1);
+            const __half* xbase = ldg_ptr<const __half>(&D.x);
 
             // ---- dependencies: the problems whose outputs (or side effects) x depends on.  ONE thread of
             // the CTA polls their counters: a counter polled by every warp of every SM is a hot spot ----
-            const int n_deps = D.n_deps;
+            const int n_deps = __ldg(&D.n_deps);
             if (n_deps > 0) {
                 if (ctid == 0 && !*dead) {
                     for (int d = 0; d < n_deps; ++d) {
-                        const uint32_t target = tag * (uint32_t)D.deps_nb[d];
-                        const uint32_t* f = ws.flags + D.deps[d];
+                        const uint32_t target = tag * (uint32_t)__ldg(&D.deps_nb[d]);
+                        const uint32_t* f = ws.flags + __ldg(&D.deps[d]);
                         bool ok = false;
                         for (uint32_t it = 0; it < kMaxFlagPolls; ++it) {
                             if (ld_acquire_u32(f) == target) { ok = true; break; }
@@ -253,7 +263,7 @@ stack_w4a16_kernel(const __grid_constant__ StackHeader H, const StackProblem* __
             // SM (read past L1: another SM may have written x during this launch) ----
             const int nch = n < NC ? n : NC;                 // distinct chunks among the CTA's quanta
             const int j_first = n < NC ? q0 % NC : 0;
-            const bool staged = D.stage_x != 0;
+            const bool staged = __ldg(&D.stage_x) != 0;
             if (staged) {
                 // piece = 8 consecutive k (16 bytes); 8 * SPG consecutive pieces = one group, held by
                 // neighbouring lanes, which add up the group's sums of x on the way
@@ -265,7 +275,7 @@ stack_w4a16_kernel(const __grid_constant__ StackHeader H, const StackProblem* __
                     j = j >= NC ? j - NC : j;
                     const int k = j * kChunkK + piece * 8;
                     uint4 u = make_uint4(0, 0, 0, 0);
-                    if (k < K) u = __ldcg(reinterpret_cast<const uint4*>(reinterpret_cast<const __half*>(D.x) + (size_t)tok * K + k));
+                    if (k < K) u = __ldcg(reinterpret_cast<const uint4*>(xbase + (size_t)tok * K + k));
                     xs[idx] = u;
                     const float2 a0 = h2f2(u.x), a1 = h2f2(u.y), b0 = h2f2(u.z), b1 = h2f2(u.w);
                     float lo = (a0.x + a0.y) + (a1.x + a1.y), hi = (b0.x + b0.y) + (b1.x + b1.y);
@@ -280,18 +290,10 @@ stack_w4a16_kernel(const __grid_constant__ StackHeader H, const StackProblem* __
                 bar_sync(1, W * 32);
             }
 
-            // A wait on a slot tells "the copy I mean" from "the copy before it" only by a parity bit, so
-            // no warp may reach use u of a slot before use u-1 has been read: a problem with more quanta
-            // than the ring has slots is taken in batches of at most that many, a CTA barrier between them
-            // (between problems the barrier before the reduction does the same).
-            const int batch = S >= weff ? (S / weff) * weff : S;
-            const __half* xbase = reinterpret_cast<const __half*>(D.x);
             int cur_j = -1;
-            for (int base = 0; base < n; base += batch) {
-                if (base > 0) bar_sync(1, W * 32);
-                const int end = base + batch < n ? base + batch : n;
+            {
                 if (warp < weff)
-                for (int i = base + warp; i < end; i += weff) {
+                for (int i = warp; i < n; i += weff) {
                     const int q = q0 + i;
                     const int rb = q / NC, j = q - rb * NC;
                     const int ns = (j == NC - 1) ? last_ns : 8;
@@ -384,14 +386,12 @@ stack_w4a16_kernel(const __grid_constant__ StackHeader H, const StackProblem* __
                     }
 
                     // ---- this quantum's ring slot ----
-                    const int seq = seq_base + i;
-                    const int use = seq / S, slot = seq - use * S;
-                    if (!*dead && !mbar_test_wait(&full[slot], (uint32_t)use & 1u) &&
-                        !mbar_wait_bounded(&full[slot], (uint32_t)use & 1u, kMaxBarPolls)) {
+                    if (!*dead && !mbar_test_wait(&my_full[slot], parity) &&
+                        !mbar_wait_bounded(&my_full[slot], parity, kMaxBarPolls)) {
                         *dead = 1;
                         if (lane == 0) atomicOr(status, 0x200u | (uint32_t)(p & 0xFF));
                     }
-                    const uint8_t* qp = ring + (size_t)slot * C::QB;
+                    const uint8_t* qp = my_ring + (size_t)slot * C::QB;
                     const uint4* slabs = reinterpret_cast<const uint4*>(qp);
                     float Dm[C::NSETS][4];
                     if (ns == 8) quantum_mma<GROUP, MP, true>(slabs, lane, 8, B, Dm);
@@ -418,7 +418,8 @@ stack_w4a16_kernel(const __grid_constant__ StackHeader H, const StackProblem* __
                     if (ns == 8) rescale(C::GC); else rescale(ng);
                     // the slot has been read: hand it back to the producer
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(&empty[slot]);
+                    if (lane == 0) mbar_arrive(&my_empty[slot]);
+                    if (++slot == R) { slot = 0; parity ^= 1u; }
 
                     if (MP == 1) { out[0][0] += out[0][1]; out[1][0] += out[1][1]; }
 #pragma unroll
@@ -439,7 +440,6 @@ stack_w4a16_kernel(const __grid_constant__ StackHeader H, const StackProblem* __
                     }
                 }
             }
-            seq_base += n;
 
             // ---- the CTA's partial sums -> outputs; row blocks shared with other CTAs go through the workspace ----
             bar_sync(1, W * 32);
@@ -462,7 +462,7 @@ stack_w4a16_kernel(const __grid_constant__ StackHeader H, const StackProblem* __
                     // this CTA holds the block's first quantum: add the later (virtual) CTAs' parts in order
                     for (int c2 = cv + 1; c2 < n_ctas; ++c2) {
                         int r0, r1;
-                        cta_range(NB, NC, D.gran, c2, n_ctas, r0, r1);
+                        cta_range(NB, NC, gran, c2, n_ctas, r0, r1);
                         if (r0 >= qb) break;
                         if (r0 >= r1) continue;
                         const unsigned long long* src = ws.parts + ((size_t)p * n_ctas + c2) * (MP * 16) + tok * 16 + row;
@@ -483,10 +483,10 @@ stack_w4a16_kernel(const __grid_constant__ StackHeader H, const StackProblem* __
                     }
                 }
                 int sub = 0;
-                while (rb >= D.nb_end[sub]) ++sub;            // the matrix that row block rb belongs to
-                const int nrow = (rb - (sub ? D.nb_end[sub - 1] : 0)) * 16 + row, Ns = D.N[sub];
+                while (rb >= __ldg(&D.nb_end[sub])) ++sub;    // the matrix that row block rb belongs to
+                const int nrow = (rb - (sub ? __ldg(&D.nb_end[sub - 1]) : 0)) * 16 + row, Ns = __ldg(&D.N[sub]);
                 if (nrow < Ns && tok < H.M)
-                    store_out(D.y[sub], (D.y_dtypes >> (8 * sub)) & 0xFF, (size_t)tok * Ns + nrow, acc);
+                    store_out(ldg_ptr<void>(&D.y[sub]), (__ldg(&D.y_dtypes) >> (8 * sub)) & 0xFF, (size_t)tok * Ns + nrow, acc);
             }
             // ---- completion: row blocks whose first quantum this CTA holds were stored by it ----
             bar_sync(1, W * 32);
@@ -509,7 +509,8 @@ stack_w4a16_kernel(const __grid_constant__ StackHeader H, const StackProblem* __
 template <int GROUP, int MP>
 size_t smem_of(int count, int slots, int max_quanta, int xs_bytes) {
     using C = Cfg<GROUP, MP>;
-    return (size_t)slots * C::QB + (size_t)count * sizeof(StackProblem) + (size_t)max_quanta * MP * 16 * 4 +
+    (void)count;   // the descriptors stay in global memory
+    return (size_t)slots * C::QB + (size_t)max_quanta * MP * 16 * 4 +
            (size_t)xs_bytes + (size_t)(xs_bytes / 1024) * C::GC * 8 + (size_t)2 * slots * 8 + 16;
 }
 

@@ -7,7 +7,7 @@ import pytest
 from paper_2506_10443_b200 import binding as B
 from paper_2506_10443_b200 import inputs
 
-HDR = struct.Struct("<IIiiiiiiiIIi")          # magic, version, count, M, group, MP, n_ctas, slots, max_quanta, smem, xs, lanes
+HDR = struct.Struct("<IIiiiiiiiII")           # magic, version, count, M, group, MP, n_ctas, slots, max_quanta, smem, xs
 PROB = struct.Struct("<4Q4QQQ" + "4i4i" + "i" * 10 + "4i4i" + "ii")
 
 
@@ -32,7 +32,7 @@ def fake_problems(model, layers=2):
 def parse(plan):
     raw = plan.tobytes()
     h = HDR.unpack_from(raw, 0)
-    hdr = dict(zip("magic version count M group MP n_ctas slots max_quanta smem xs lanes".split(), h))
+    hdr = dict(zip("magic version count M group MP n_ctas slots max_quanta smem xs".split(), h))
     probs = []
     for p in range(hdr["count"]):
         f = PROB.unpack_from(raw, 64 + 192 * p)
@@ -58,8 +58,8 @@ def test_plan_covers_every_quantum_once_and_fits_shared_memory(model, M, n_sms):
     hdr, out = parse(B.stack_plan_w4a16(probs, M, 64, n_sms=n_sms))
     # q+k+v and gate+up share their input and their predecessors: 4 problems per layer in the plan
     assert hdr["count"] == 8 and hdr["n_ctas"] == n_sms and hdr["M"] == M
-    assert hdr["slots"] >= 2 and hdr["smem"] <= 227 * 1024
-    assert 1 <= hdr["lanes"] <= 32 and hdr["slots"] % hdr["lanes"] == 0   # a slot is always refilled by the same lane
+    assert hdr["slots"] >= 14 and hdr["smem"] <= 227 * 1024
+    assert hdr["slots"] % 14 == 0   # every consumer warp owns the same number of slots
     groups = [[0, 1, 2], [3], [4, 5], [6], [7, 8, 9], [10], [11, 12], [13]]
     for members, d in zip(groups, out):
         want = [probs[i] for i in members]
