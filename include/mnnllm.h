@@ -78,7 +78,8 @@ int mnnllm_pack_w4(const float* W, int N, int K, int group, void* packed_out);
  * N, K and group are taken from the header. */
 int mnnllm_unpack_w4(const void* packed, uint8_t* q, uint16_t* scale_bits, uint16_t* zero_bits);
 
-/* Reads N, K and group of a packed buffer (host); any output pointer may be null. */
+/* Reads N, K and group of a packed buffer (host); any output pointer may be null.  (A helper of this
+ * library's buffer format; the paper has no counterpart.) */
 int mnnllm_packed_info(const void* packed, int* N, int* K, int* group, int* bits);
 
 /* int8 per-channel variant (Section 4.2: the LM head is kept in int8): Eq. 1 with clip_max = 255,
@@ -102,13 +103,17 @@ int mnnllm_unpack_w8(const void* packed, uint8_t* q, uint16_t* scale_bits, uint1
 int mnnllm_linear_w4a16(const void* x, const void* packed, void* y, int M, int N, int K, int group,
                         void* stream);
 
-/* Same with explicit dtypes: x_dtype MNNLLM_F16; y_dtype MNNLLM_F16, MNNLLM_BF16 or MNNLLM_F32
- * (fp32 logits for the LM head). */
+/* Same with explicit dtypes (Section 4.2: floating-point activations on GPUs): x_dtype MNNLLM_F16 or
+ * MNNLLM_BF16; y_dtype MNNLLM_F16, MNNLLM_BF16 or MNNLLM_F32 (fp32 logits for the LM head).  bf16
+ * activations are converted to fp16 as the kernel loads them, which is exact for magnitudes in
+ * [2^-17, 65504]; larger values saturate at +-65504, smaller ones lose low bits. */
 int mnnllm_linear_w4a16_ex(const void* x, const void* packed, void* y, int M, int N, int K, int group,
                            int x_dtype, int y_dtype, void* stream);
 
 /* Several independent W4A16 problems that share M (for example q, k, v of one layer, or gate and
- * up) in ONE launch.  `problems` is a host array of `count` (1..MNNLLM_MAX_BATCH) descriptors; it
+ * up) in ONE launch: each computes exactly what mnnllm_linear_w4a16_ex computes (Section 4.2, W4A16);
+ * putting them in one launch is this library's, as the paper's GPU path adjusts its parallelism to
+ * the problem's dimensions (Section 5.1).  `problems` is a host array of `count` (1..MNNLLM_MAX_BATCH) descriptors; it
  * is copied into the launch and may be reused when the call returns. */
 #define MNNLLM_MAX_BATCH 8
 typedef struct {
@@ -172,7 +177,7 @@ int mnnllm_linear_w8a16(const void* x, const void* packed, void* y, int M, int N
                         void* stream);
 
 /* ------------------------------------------------------------------------------------------------
- * W4A8 (Section 4.2: "activation values are quantized to int8 ... W4A8"):
+ * W4A8 (Section 4.2: per-token int8 activation quantisation in front of integer matrix instructions):
  *   per token m:   amax = max_k |x[m, k]|,  a_scale[m] = amax / 127,
  *                  a_q[m, k] = clamp(round(x[m, k] * (127 / amax)), -127, 127)   (0 if amax == 0)
  *   per group g:   P[m, n, g] = sum_{k in g} a_q[m, k] * q[n, k]      (int32, exact)
@@ -181,6 +186,10 @@ int mnnllm_linear_w8a16(const void* x, const void* packed, void* y, int M, int N
  *
  *   x          device [M, K] of x_dtype (MNNLLM_F16 or MNNLLM_BF16)
  *   y          device [M, N] of y_dtype, overwritten
+ *   weights    the zero-point term sum_g scale*zero*A is evaluated on the tensor cores from a two-term
+ *              fp16 split of scale*zero (about the group's |w_min|): every group needs |w_min| < 256,
+ *              and the term is carried to 2^-33 absolute, i.e. without loss for weights whose typical
+ *              magnitude is above ~1e-5 (the W4A16 path has neither limit)
  *   workspace  device scratch, 256-byte aligned; holds a_q, a_scale, A between the two kernels.
  *              mnnllm_workspace_size_w4a8(M, N, K, group) is the size to allocate.  It includes
  *              about 20 MB in which a problem with fewer 128 x 128 output tiles than the GPU has
@@ -193,6 +202,8 @@ int mnnllm_linear_w8a16(const void* x, const void* packed, void* y, int M, int N
  *              the call would reject.
  * ---------------------------------------------------------------------------------------------- */
 size_t mnnllm_workspace_size_w4a8(int M, int N, int K, int group);
+/* Smallest workspace mnnllm_linear_w4a8 accepts (no room for splitting tiles along K); a sizing
+ * helper of this library, the paper has no counterpart. */
 size_t mnnllm_workspace_min_w4a8(int M, int N, int K, int group);
 int mnnllm_linear_w4a8(const void* x, const void* packed, void* y, int M, int N, int K, int group,
                        int x_dtype, int y_dtype, void* workspace, size_t workspace_bytes, void* stream);
@@ -251,6 +262,14 @@ int mnnllm_debug_w4a8_partials(const void* x, int x_dtype, const void* packed, i
  * instead of spinning.  This call synchronises `stream`, reads the word, clears it and returns
  * MNNLLM_OK or MNNLLM_ERR_TIMEOUT (detail, if not null, receives the raw word). */
 int mnnllm_read_status(void* stream, uint32_t* detail);
+
+/* Exercises the time-out path without any of the library's kernels having to fail: enqueues a
+ * one-warp kernel that waits, with the kernels' own bounded wait, on a barrier nobody arrives at
+ * (max_polls tries of at most 20 microseconds each, 1..1000), records MNNLLM_DEBUG_TIMEOUT_DETAIL in
+ * the status word and ends normally.  mnnllm_read_status then reports MNNLLM_ERR_TIMEOUT once.
+ * (Failure reporting is this library's; the paper has no counterpart.) */
+#define MNNLLM_DEBUG_TIMEOUT_DETAIL 0x2000u
+int mnnllm_debug_wait_timeout(int max_polls, void* stream);
 
 /* 1 if the current CUDA device can run the kernels (compute capability 10.x), else 0. */
 int mnnllm_device_supported(void);

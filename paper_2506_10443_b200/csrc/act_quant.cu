@@ -1,5 +1,5 @@
 // Dynamic per-token int8 activation quantisation, the first kernel of the W4A8 path
-// (Section 4.2: "activation values are quantized to int8").  For every token m:
+// (Section 4.2: per-token int8 activation quantisation).  For every token m:
 //     amax = max_k |x[m,k]|,  a_scale = amax / 127,  a_q = clamp(rint(x * (127 / amax)), -127, 127)
 // and, for the zero-point correction of the asymmetric weights, the group sums A[m,g] = sum a_q.
 // One CTA per token; the row is read twice (the second read hits L2).  HBM-bound and tiny next to
@@ -12,6 +12,7 @@
 #include <cuda_fp16.h>
 
 #include "act_quant.h"
+#include "common.h"
 #include "ptx.cuh"
 
 namespace mnnllm {
@@ -128,17 +129,20 @@ __global__ void __launch_bounds__(kThreads) act_quant_kernel(const T* __restrict
 cudaError_t act_quant_launch(const void* x, int x_dtype, int M, int K, int group, int8_t* a_q, float* a_scale,
                              int32_t* A, void* AC, bool offset128, uint32_t* clear, int n_clear, cudaStream_t stream) {
     if (!clear) n_clear = 0;
-    static bool carveout_set = false;
-    if (!carveout_set) {
-        // the GEMM that follows needs the largest shared-memory carve-out: ask for the same here, so
-        // that the SMs are not re-partitioned between the two kernels of a call
-        cudaFuncSetAttribute(act_quant_kernel<__half>, cudaFuncAttributePreferredSharedMemoryCarveout,
-                             (int)cudaSharedmemCarveoutMaxShared);
-        cudaFuncSetAttribute(act_quant_kernel<__nv_bfloat16>, cudaFuncAttributePreferredSharedMemoryCarveout,
-                             (int)cudaSharedmemCarveoutMaxShared);
-        (void)cudaGetLastError();
-        carveout_set = true;
-    }
+    static PerDevice<bool> carveout_set;
+    (void)carveout_set.with([](bool& done) {
+        if (!done) {
+            // the GEMM that follows needs the largest shared-memory carve-out: ask for the same here, so
+            // that the SMs are not re-partitioned between the two kernels of a call
+            cudaFuncSetAttribute(act_quant_kernel<__half>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                 (int)cudaSharedmemCarveoutMaxShared);
+            cudaFuncSetAttribute(act_quant_kernel<__nv_bfloat16>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                 (int)cudaSharedmemCarveoutMaxShared);
+            (void)cudaGetLastError();
+            done = true;
+        }
+        return cudaSuccess;
+    });
     const uint32_t code_xor = offset128 ? 0x80808080u : 0u;
     const int G4 = (K / group + 3) / 4 * 4;
     uint2* ac = reinterpret_cast<uint2*>(AC);

@@ -13,18 +13,6 @@ namespace {
 constexpr size_t kSmemBudget = 227 * 1024;
 constexpr long long kStageBudget = 40 * 1024;   // staged activations per CTA at most
 
-int sm_count_of_current_device() {
-    static int cached[64];
-    int dev = -1;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
-    if (!cached[dev]) {
-        int n = 0;
-        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
-        cached[dev] = n;
-    }
-    return cached[dev];
-}
-
 int mp_of(int M) { return M <= 1 ? 1 : (M <= 2 ? 2 : (M <= 4 ? 4 : 8)); }
 
 // most quanta a CTA receives when U runs of `gran` quanta are dealt evenly to n CTAs
@@ -51,7 +39,7 @@ int mnnllm_stack_plan_w4a16(const mnnllm_stack_problem* problems, int count, int
     if (M > 8 || (group != 64 && group != 128)) return MNNLLM_ERR_UNSUPPORTED;
     if (n_sms == 0) {
         if (!device_is_supported()) return MNNLLM_ERR_UNSUPPORTED;
-        n_sms = sm_count_of_current_device();
+        n_sms = device_sm_count();
     }
     if (n_sms < 1) return MNNLLM_ERR_INVALID_ARG;
     const int MP = mp_of(M);
@@ -193,7 +181,7 @@ int mnnllm_linear_w4a16_stack(const void* plan_host, const void* plan_dev, void*
     if (!workspace || workspace_bytes < stack_ws_bytes(H.count, H.n_ctas, H.MP)) return MNNLLM_ERR_WORKSPACE;
     if ((uintptr_t)workspace & 255) return MNNLLM_ERR_ALIGNMENT;
     if (!device_is_supported()) return MNNLLM_ERR_UNSUPPORTED;
-    if (H.n_ctas > sm_count_of_current_device()) return MNNLLM_ERR_UNSUPPORTED;   // all CTAs must be resident
+    if (H.n_ctas > device_sm_count()) return MNNLLM_ERR_UNSUPPORTED;   // all CTAs must be resident
     uint32_t* status = status_word_ptr();
     if (!status) return MNNLLM_ERR_CUDA;
     StackWorkspace ws;

@@ -8,36 +8,68 @@
 
 #include "common.h"
 #include "gemv.h"
+#include "ptx.cuh"
 
 namespace mnnllm {
 
 __device__ uint32_t g_status_word = 0;
 
-static int g_cc_major[64];
-static bool g_cc_known[64];
-static uint32_t* g_status_ptr[64];
+namespace {
+struct DeviceFacts {
+    bool known;
+    int cc_major, sm_count;
+    uint32_t* status_ptr;
+};
+PerDevice<DeviceFacts> g_facts;
+
+// the current device's facts, asked of the runtime on first use
+cudaError_t device_facts(DeviceFacts& out) {
+    return g_facts.with([&](DeviceFacts& f) {
+        if (!f.known) {
+            const int dev = current_device();
+            void* p = nullptr;
+            cudaError_t e = cudaDeviceGetAttribute(&f.cc_major, cudaDevAttrComputeCapabilityMajor, dev);
+            if (e == cudaSuccess) e = cudaDeviceGetAttribute(&f.sm_count, cudaDevAttrMultiProcessorCount, dev);
+            if (e == cudaSuccess) e = cudaGetSymbolAddress(&p, g_status_word);
+            if (e != cudaSuccess) return e;
+            f.status_ptr = (uint32_t*)p;
+            f.known = true;
+        }
+        out = f;
+        return cudaSuccess;
+    });
+}
+}  // namespace
 
 int device_is_supported() {
-    int dev = -1;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
-    if (!g_cc_known[dev]) {
-        int major = 0;
-        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return 0;
-        g_cc_major[dev] = major;
-        g_cc_known[dev] = true;
-    }
-    return g_cc_major[dev] == 10;
+    DeviceFacts f;
+    if (device_facts(f) != cudaSuccess) { (void)cudaGetLastError(); return 0; }
+    return f.cc_major == 10;
+}
+
+int device_sm_count() {
+    DeviceFacts f;
+    if (device_facts(f) != cudaSuccess) { (void)cudaGetLastError(); return 0; }
+    return f.sm_count;
 }
 
 uint32_t* status_word_ptr() {
-    int dev = -1;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
-    if (!g_status_ptr[dev]) {
-        void* p = nullptr;
-        if (cudaGetSymbolAddress(&p, g_status_word) != cudaSuccess) return nullptr;
-        g_status_ptr[dev] = (uint32_t*)p;
+    DeviceFacts f;
+    if (device_facts(f) != cudaSuccess) { (void)cudaGetLastError(); return nullptr; }
+    return f.status_ptr;
+}
+
+// One warp waits on a barrier that nobody will ever arrive at, with the same bounded wait the
+// kernels use; when the wait runs out it records a code in the status word and returns normally.
+__global__ void wait_timeout_kernel(uint32_t max_polls, uint32_t* status) {
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        ptx::mbar_init(&bar, 1);
+        ptx::fence_mbar_init();
     }
-    return g_status_ptr[dev];
+    __syncwarp();
+    if (!ptx::mbar_wait_bounded_compact(&bar, 0, max_polls) && threadIdx.x == 0)
+        atomicOr(status, MNNLLM_DEBUG_TIMEOUT_DETAIL);
 }
 
 namespace {
@@ -47,20 +79,29 @@ struct Plan {
     int clusters;  // total clusters of the launch (persistent: about one resident set)
 };
 
-// Resident CTAs per SM, asked of the runtime once per configuration and cached.
+// Resident CTAs per SM, asked of the runtime once per configuration and device, and cached.
 int cached_occupancy(int bits, int group, int MP, int W, int SR, int S) {
     struct Entry { int key[6]; int occ; };
-    static Entry cache[64];
-    static int n_cached = 0;
+    struct Table { Entry e[64]; int n; };
+    static PerDevice<Table> tables;
     const int key[6] = {bits, group, MP, W, SR, S};
-    for (int i = 0; i < n_cached; ++i)
-        if (!std::memcmp(cache[i].key, key, sizeof(key))) return cache[i].occ;
-    int occ = bits == 4 ? gemv_w4a16_occupancy(group, MP, W, SR, S) : gemv_w8a16_occupancy(W, SR, S);
+    int occ = 0;
+    (void)tables.with([&](Table& t) {
+        for (int i = 0; i < t.n; ++i)
+            if (!std::memcmp(t.e[i].key, key, sizeof(key))) { occ = t.e[i].occ; return cudaSuccess; }
+        return cudaSuccess;
+    });
+    if (occ) return occ;
+    // asked outside the table's lock: the query itself takes the kernels' own per-device locks
+    occ = bits == 4 ? gemv_w4a16_occupancy(group, MP, W, SR, S) : gemv_w8a16_occupancy(W, SR, S);
     if (occ < 1) occ = 1;
-    if (n_cached < 64) {
-        std::memcpy(cache[n_cached].key, key, sizeof(key));
-        cache[n_cached++].occ = occ;
-    }
+    (void)tables.with([&](Table& t) {
+        if (t.n < 64) {
+            std::memcpy(t.e[t.n].key, key, sizeof(key));
+            t.e[t.n++].occ = occ;
+        }
+        return cudaSuccess;
+    });
     return occ;
 }
 
@@ -78,7 +119,8 @@ Plan make_plan(int nb_total, int nc_max, int group, int MP, int bits = 4) {
     p.WC = (nc_max + p.CS - 1) / p.CS;
     if (p.WC > kGemvMaxWarps) p.WC = kGemvMaxWarps;
     p.SR = kGemvMaxWarps / p.WC;
-    while (p.SR > 1 && nb_total * p.CS < kNumSMs * p.SR) --p.SR;
+    const int n_sms = device_sm_count() > 0 ? device_sm_count() : 148;
+    while (p.SR > 1 && nb_total * p.CS < n_sms * p.SR) --p.SR;
     p.stages = 3;
     p.RBI = 0;
     int forced_clusters = 0;
@@ -99,7 +141,7 @@ Plan make_plan(int nb_total, int nc_max, int group, int MP, int bits = 4) {
     };
     while (p.stages > 1 && smem(p.stages) > 220 * 1024) --p.stages;
     const int occ = cached_occupancy(bits, group, MP, p.WC * p.SR, p.SR, p.stages);
-    int clusters = kNumSMs * occ / p.CS;
+    int clusters = n_sms * occ / p.CS;
     const int max_useful = (nb_total + p.SR - 1) / p.SR;  // at least SR row blocks per cluster
     if (clusters > max_useful) clusters = max_useful;
     if (forced_clusters) clusters = forced_clusters;
@@ -140,7 +182,7 @@ int check_problem(const mnnllm_w4a16_problem& q, int M) {
     return MNNLLM_OK;
 }
 
-int run_batch(const mnnllm_w4a16_problem* problems, int count, int M, cudaStream_t stream) {
+int run_batch(const mnnllm_w4a16_problem* problems, int count, int M, int x_dtype, cudaStream_t stream) {
     if (!problems || count < 1 || count > MNNLLM_MAX_BATCH) return MNNLLM_ERR_INVALID_ARG;
     const int group = problems[0].group;
     for (int i = 0; i < count; ++i) {
@@ -182,6 +224,7 @@ int run_batch(const mnnllm_w4a16_problem* problems, int count, int M, cudaStream
             P.cluster_begin = clusters;
             P.n_clusters = ncl[i];
             P.y_dtype = q.y_dtype;
+            P.x_dtype = x_dtype;
             P.row_block_bytes = g.row_block_bytes;
             clusters += ncl[i];
         }
@@ -213,8 +256,18 @@ int mnnllm_read_status(void* stream, uint32_t* detail) {
     return v ? MNNLLM_ERR_TIMEOUT : MNNLLM_OK;
 }
 
+int mnnllm_debug_wait_timeout(int max_polls, void* stream) {
+    if (max_polls < 1 || max_polls > 1000) return MNNLLM_ERR_INVALID_ARG;
+    if (!device_is_supported()) return MNNLLM_ERR_UNSUPPORTED;
+    uint32_t* status = status_word_ptr();
+    if (!status) return MNNLLM_ERR_CUDA;
+    wait_timeout_kernel<<<1, 32, 0, (cudaStream_t)stream>>>((uint32_t)max_polls, status);
+    if (cudaGetLastError() != cudaSuccess) return MNNLLM_ERR_CUDA;
+    return MNNLLM_OK;
+}
+
 int mnnllm_linear_w4a16_batch(const mnnllm_w4a16_problem* problems, int count, int M, void* stream) {
-    return run_batch(problems, count, M, (cudaStream_t)stream);
+    return run_batch(problems, count, M, MNNLLM_F16, (cudaStream_t)stream);
 }
 
 int mnnllm_linear_w8a16(const void* x, const void* packed, void* y, int M, int N, int K, int y_dtype, void* stream) {
@@ -251,11 +304,11 @@ int mnnllm_linear_w8a16(const void* x, const void* packed, void* y, int M, int N
 
 int mnnllm_linear_w4a16_ex(const void* x, const void* packed, void* y, int M, int N, int K, int group, int x_dtype,
                            int y_dtype, void* stream) {
-    if (x_dtype != MNNLLM_F16) return x_dtype == MNNLLM_BF16 || x_dtype == MNNLLM_F32 ? MNNLLM_ERR_UNSUPPORTED
-                                                                                     : MNNLLM_ERR_INVALID_ARG;
+    if (x_dtype != MNNLLM_F16 && x_dtype != MNNLLM_BF16)
+        return x_dtype == MNNLLM_F32 ? MNNLLM_ERR_UNSUPPORTED : MNNLLM_ERR_INVALID_ARG;
     mnnllm_w4a16_problem p;
     p.x = x; p.packed = packed; p.y = y; p.N = N; p.K = K; p.group = group; p.y_dtype = y_dtype;
-    return run_batch(&p, 1, M, (cudaStream_t)stream);
+    return run_batch(&p, 1, M, x_dtype, (cudaStream_t)stream);
 }
 
 int mnnllm_linear_w4a16(const void* x, const void* packed, void* y, int M, int N, int K, int group, void* stream) {

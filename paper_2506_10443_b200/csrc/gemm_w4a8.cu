@@ -47,6 +47,7 @@
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
+#include "common.h"
 #include "gemm_w4a8.h"
 #include "layout.h"
 #include "ptx.cuh"
@@ -163,28 +164,23 @@ EncodeTiledFn encode_fn() {
 
 // SMs of the current device (one persistent CTA each), asked once per device.
 int sm_count() {
-    static int cached[64];
-    int dev = -1;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
-    if (!cached[dev]) {
-        int n = 0;
-        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
-        cached[dev] = n;
-    }
-    return cached[dev];
+    return device_sm_count();
 }
 
 template <int GROUP, bool PARTIALS, bool SPLIT>
 cudaError_t launch(const CUtensorMap& tm_act, const CUtensorMap& tm_ac, const WeightMaps& wmaps, const Params& p,
                    dim3 grid, uint32_t* status, cudaStream_t stream) {
-    static bool configured = false;
+    static PerDevice<bool> configured;   // per instantiation and device
     void (*kern)(CUtensorMap, CUtensorMap, WeightMaps, Params, uint32_t*) =
         SPLIT ? gemm_w4a8_split_kernel<GROUP, PARTIALS> : gemm_w4a8_kernel<GROUP, PARTIALS>;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
-        if (e != cudaSuccess) return e;
-        configured = true;
-    }
+    if (cudaError_t e = configured.with([&](bool& done) {
+            if (done) return cudaSuccess;
+            cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+            done = err == cudaSuccess;
+            return err;
+        });
+        e != cudaSuccess)
+        return e;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
     cfg.blockDim = dim3(kThreads);

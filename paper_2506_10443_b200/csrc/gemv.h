@@ -11,7 +11,6 @@ namespace mnnllm {
 constexpr int kGemvMaxWarps = 7;    // warps per CTA (7 * 32 threads leave 144 registers each at 2 CTAs per SM)
 constexpr int kGemvMaxStages = 4;   // ring slots per warp
 constexpr int kGemvMaxRBI = 8;      // 16-row blocks a warp walks through per k-chunk
-constexpr int kNumSMs = 148;
 
 struct GemvProblem {
     const uint8_t* packed;  // start of the packed buffer (header included)
@@ -22,6 +21,7 @@ struct GemvProblem {
     int cluster_begin;      // first cluster of this problem in the launch
     int n_clusters;         // clusters that share this problem's row blocks evenly
     int y_dtype;
+    int x_dtype;            // MNNLLM_F16, or MNNLLM_BF16 (converted to fp16 as the fragments are built)
     unsigned long long row_block_bytes;
     unsigned long long table_offset;  // W8: per-row (scale, zero) table, from the buffer start
 };

@@ -19,6 +19,7 @@
 #include <cuda_fp16.h>
 #include <cuda_bf16.h>
 
+#include "common.h"
 #include "gemv.h"
 #include "gemv_w4a16_core.cuh"
 #include "ptx.cuh"
@@ -102,8 +103,9 @@ gemv_w4a16_kernel(const __grid_constant__ GemvLaunch L, uint32_t* __restrict__ s
     // push the activations (written by the previous kernel, read by the next) out of L2
     const uint64_t stream_policy = policy_evict_first();
     // every lane keeps the (uniform) producer state; one elected lane issues the copy
+    bool dead = false;   // a bounded wait gave up: nothing more is copied or waited for
     auto issue_next = [&]() {
-        if (i_rd >= n_rounds) return;
+        if (i_rd >= n_rounds || dead) return;
         if (elect_one()) {
             mbar_arrive_expect_tx(&bars[i_slot], i_bytes);
             bulk_g2s_hint(ring + (size_t)i_slot * C::QB, i_src, i_bytes, &bars[i_slot], stream_policy);
@@ -129,9 +131,9 @@ gemv_w4a16_kernel(const __grid_constant__ GemvLaunch L, uint32_t* __restrict__ s
     pdl_wait();
 
     const int tokB = r % MP, gsB = r / MP;  // B-operand role of this lane: column r of the MMA
+    const bool x_bf16 = P.x_dtype == MNNLLM_BF16;
     uint32_t B[8][4][2];
     float C1[C::NSETS][2], C2[C::NSETS][2];
-    bool dead = false;
     int cur_j = -1, slot = 0;
     uint32_t phase = 0;
     const int wc_used = (P.NC - rank * L.WC) < L.WC ? (P.NC - rank * L.WC) : L.WC;  // warps that own a chunk
@@ -159,6 +161,7 @@ gemv_w4a16_kernel(const __grid_constant__ GemvLaunch L, uint32_t* __restrict__ s
                                 reinterpret_cast<const uint4*>(xk + (size_t)tokB * P.K + sl * kSlabK4 + 16 * c);
                             u0 = px[0];
                             u1 = px[1];
+                            if (x_bf16) { u0 = bf16x8_to_f16x8(u0); u1 = bf16x8_to_f16x8(u1); }
                         }
                         B[sl][0][0] = __byte_perm(u0.x, u0.y, 0x5410);
                         B[sl][0][1] = __byte_perm(u0.z, u0.w, 0x5410);
@@ -181,7 +184,8 @@ gemv_w4a16_kernel(const __grid_constant__ GemvLaunch L, uint32_t* __restrict__ s
                             for (int sp = 0; sp < C::SPG; ++sp) {
                                 const uint4* px = reinterpret_cast<const uint4*>(
                                     xk + (size_t)tokB * P.K + (gi * C::SPG + sp) * kSlabK4 + 16 * c);
-                                const uint4 u0 = px[0], u1 = px[1];
+                                uint4 u0 = px[0], u1 = px[1];
+                                if (x_bf16) { u0 = bf16x8_to_f16x8(u0); u1 = bf16x8_to_f16x8(u1); }
                                 float2 f;
                                 f = h2f2(u0.x); lo += f.x + f.y;
                                 f = h2f2(u0.y); lo += f.x + f.y;
@@ -309,6 +313,8 @@ gemv_w4a16_kernel(const __grid_constant__ GemvLaunch L, uint32_t* __restrict__ s
             }
         }
     }
+    if (dead)   // copies issued before the give-up may still be in flight into this CTA's shared memory
+        for (int i = 0; i < 50; ++i) __nanosleep(1000);
     if (CS > 1) cluster_sync();  // peers may still be reading this CTA's shared memory
 }
 
@@ -322,23 +328,26 @@ size_t smem_bytes(int W, int SR, int S) {
 // Raises the kernel's dynamic shared memory limit when a launch needs more than any before it.
 template <int GROUP, int MP>
 cudaError_t ensure_smem(size_t smem) {
-    static size_t configured = 0;  // per instantiation
-    static bool carveout_set = false;
-    if (!carveout_set) {
-        // every launch of the library asks for the same (largest) shared-memory carve-out, so that
-        // an SM does not have to re-partition its L1 between consecutive dependent launches
-        cudaError_t e = cudaFuncSetAttribute(gemv_w4a16_kernel<GROUP, MP>, cudaFuncAttributePreferredSharedMemoryCarveout,
-                                             (int)cudaSharedmemCarveoutMaxShared);
-        if (e != cudaSuccess) return e;
-        carveout_set = true;
-    }
-    if (smem > configured) {
-        cudaError_t e = cudaFuncSetAttribute(gemv_w4a16_kernel<GROUP, MP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)smem);
-        if (e != cudaSuccess) return e;
-        configured = smem;
-    }
-    return cudaSuccess;
+    struct State { size_t configured; bool carveout_set; };
+    static PerDevice<State> state;   // per instantiation and device
+    return state.with([&](State& st) {
+        if (!st.carveout_set) {
+            // every launch of the library asks for the same (largest) shared-memory carve-out, so that
+            // an SM does not have to re-partition its L1 between consecutive dependent launches
+            cudaError_t e = cudaFuncSetAttribute(gemv_w4a16_kernel<GROUP, MP>,
+                                                 cudaFuncAttributePreferredSharedMemoryCarveout,
+                                                 (int)cudaSharedmemCarveoutMaxShared);
+            if (e != cudaSuccess) return e;
+            st.carveout_set = true;
+        }
+        if (smem > st.configured) {
+            cudaError_t e = cudaFuncSetAttribute(gemv_w4a16_kernel<GROUP, MP>,
+                                                 cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e != cudaSuccess) return e;
+            st.configured = smem;
+        }
+        return cudaSuccess;
+    });
 }
 
 template <int GROUP, int MP>

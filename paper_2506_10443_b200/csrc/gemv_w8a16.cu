@@ -7,6 +7,7 @@
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
+#include "common.h"
 #include "gemv.h"
 #include "ptx.cuh"
 
@@ -75,8 +76,9 @@ gemv_w8a16_kernel(const __grid_constant__ GemvLaunch L, uint32_t* __restrict__ s
     int i_rd = 0, i_t = 0, i_it = 0, i_nit = nit_of(0), i_slot = 0;
     while (i_rd < n_rounds && i_nit == 0) { ++i_rd; i_nit = i_rd < n_rounds ? nit_of(i_rd) : 0; }
     const uint64_t stream_policy = policy_evict_first();  // weights are read once: keep them from displacing x in L2
+    bool dead = false;   // a bounded wait gave up: nothing more is copied or waited for
     auto issue_next = [&]() {
-        if (i_rd >= n_rounds) return;
+        if (i_rd >= n_rounds || dead) return;
         const int j = j0 + i_t * jstride;
         const int rb = rb_begin + i_rd * per_round + i_it * SR + sr;
         const int ns = (j == P.NC - 1) ? last_ns : 16;
@@ -101,7 +103,6 @@ gemv_w8a16_kernel(const __grid_constant__ GemvLaunch L, uint32_t* __restrict__ s
 
     uint32_t B[16][2][2];
     float X0 = 0.f, X1 = 0.f;  // sum of x over the current chunk for tokens 2c and 2c + 1
-    bool dead = false;
     int cur_j = -1, slot = 0;
     uint32_t phase = 0;
     const int wc_used = (P.NC - rank * L.WC) < L.WC ? (P.NC - rank * L.WC) : L.WC;
@@ -215,26 +216,31 @@ gemv_w8a16_kernel(const __grid_constant__ GemvLaunch L, uint32_t* __restrict__ s
             }
         }
     }
+    if (dead)   // copies issued before the give-up may still be in flight into this CTA's shared memory
+        for (int i = 0; i < 50; ++i) __nanosleep(1000);
     if (CS > 1) cluster_sync();
 }
 
 }  // namespace
 
 static cudaError_t ensure_smem_w8(size_t smem) {
-    static size_t configured = 0;
-    static bool carveout_set = false;
-    if (!carveout_set) {   // the same carve-out as every other kernel of the library
-        cudaError_t e = cudaFuncSetAttribute(gemv_w8a16_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
-                                             (int)cudaSharedmemCarveoutMaxShared);
-        if (e != cudaSuccess) return e;
-        carveout_set = true;
-    }
-    if (smem > configured) {
-        cudaError_t e = cudaFuncSetAttribute(gemv_w8a16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        configured = smem;
-    }
-    return cudaSuccess;
+    struct State { size_t configured; bool carveout_set; };
+    static PerDevice<State> state;
+    return state.with([&](State& st) {
+        if (!st.carveout_set) {   // the same carve-out as every other kernel of the library
+            cudaError_t e = cudaFuncSetAttribute(gemv_w8a16_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                                 (int)cudaSharedmemCarveoutMaxShared);
+            if (e != cudaSuccess) return e;
+            st.carveout_set = true;
+        }
+        if (smem > st.configured) {
+            cudaError_t e =
+                cudaFuncSetAttribute(gemv_w8a16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e != cudaSuccess) return e;
+            st.configured = smem;
+        }
+        return cudaSuccess;
+    });
 }
 
 size_t gemv_w8a16_smem(int W, int SR, int S) {

@@ -1,6 +1,6 @@
 // Host-side weight packer: Eq. 1 quantisation (Section 4.2) and the reorder of codes and
 // (scale, zero) pairs into the bulk-copy friendly layout of layout.h.  Runs once at model load
-// ("weights are determined when the model is loaded", Section 5.1); no GPU involved.
+// (packing happens once, at model load, Section 5.1); no GPU involved.
 //
 // Built with floating-point contraction off: each fp32 operation below rounds once, as written.
 #include <cmath>

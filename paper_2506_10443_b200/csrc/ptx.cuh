@@ -62,15 +62,9 @@ __device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity) {
 // together (the W4A8 GEMM: up to 12 % faster; a polling loop in a function of its own was slower
 // than either).
 __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, uint32_t max_polls) {
-#ifdef MNNLLM_SPIN_WAIT
-    for (uint32_t i = 0; i < max_polls * 64u; ++i)
-        if (mbar_test_wait(bar, parity)) return true;
-    return false;
-#else
     for (uint32_t i = 0; i < max_polls; ++i)
         if (mbar_try_wait(bar, parity)) return true;
     return false;
-#endif
 }
 __device__ __forceinline__ bool mbar_wait_bounded_compact(uint64_t* bar, uint32_t parity, uint32_t max_polls) {
 #pragma unroll 1

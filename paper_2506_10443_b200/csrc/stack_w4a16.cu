@@ -21,6 +21,7 @@
 
 #include "gemv_w4a16_core.cuh"
 #include "ptx.cuh"
+#include "common.h"
 #include "stack.h"
 
 namespace mnnllm {
@@ -519,16 +520,15 @@ cudaError_t launch_one(const StackHeader& H, const void* plan_dev, const StackWo
                        cudaStream_t stream) {
     auto kern = stack_w4a16_kernel<GROUP, MP>;
     // function attributes belong to a device: set per device, once
-    static bool configured[64];
-    int dev = -1;
-    if (cudaError_t e = cudaGetDevice(&dev); e != cudaSuccess) return e;
-    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-    if (!configured[dev]) {
-        if (cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-            e != cudaSuccess)
-            return e;
-        configured[dev] = true;
-    }
+    static PerDevice<bool> configured;   // per instantiation and device
+    if (cudaError_t e = configured.with([&](bool& done) {
+            if (done) return cudaSuccess;
+            cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+            done = err == cudaSuccess;
+            return err;
+        });
+        e != cudaSuccess)
+        return e;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)H.n_ctas);
     cfg.blockDim = dim3((unsigned)kStackThreads);

@@ -1,5 +1,5 @@
 """Device-resident synthetic workloads shaped like the paper's evaluation models (Section 6): the
-linear layers of a decoder stack, packed once ("weights are determined when the model is loaded",
+linear layers of a decoder stack, packed once (packing happens once, at model load,
 Section 5.1) and then driven token by token (decode) or prompt by prompt (prefill).
 
 Only plumbing lives here: seeded arrays from ``inputs`` are packed with the library's host packer,

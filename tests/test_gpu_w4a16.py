@@ -77,9 +77,19 @@ def test_w4a16_output_dtypes():
     assert_close(run_w4a16(x, packed, M, N, K, group, B.F32), ref)
     assert_close(run_w4a16(x, packed, M, N, K, group, B.F32), ref, 2e-4)   # fp32 logits are much tighter
     y_bf16 = run_w4a16(x, packed, M, N, K, group, B.BF16)
-    y_f32 = run_w4a16(x, packed, M, N, K, group, B.F32)
-    assert_bf16_within_1ulp(y_bf16, y_f32.astype(np.float64))
-    assert_close(y_bf16, ref, 2.0 ** -8 + 2e-4)
+    assert_bf16_within_1ulp(y_bf16, ref)
+
+
+@pytest.mark.parametrize("N,K,M,group", [(256, 1536, 1, 64), (1536, 8960, 1, 64), (777, 1024, 3, 64), (1000, 3584, 4, 128),
+                                         (300, 1536, 11, 64)])
+def test_w4a16_bf16_activations_match_oracle(N, K, M, group):
+    W, packed, (q, s, z) = quantized(N + 3 * K + M, N, K, group)
+    xb = inputs.activations(N + K + 5 * M, M, K, dtype="bf16")      # fp32 array of bf16-exact values
+    xd = dev(inputs.bf16_bits(xb)).view(torch.bfloat16)
+    y = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
+    B.linear_w4a16_ex(xd, dev(packed), y, M, N, K, group, B.BF16, B.F32)
+    assert B.read_status() == 0
+    assert_close(y.cpu().numpy(), oracle.linear_wa16(xb, q, s, z, group), 2e-4)
 
 
 def test_w4a16_batch_qkv_one_launch():
@@ -123,7 +133,8 @@ def test_w4a16_argument_errors_on_gpu():
     st = B.lib.mnnllm_linear_w4a16(y.data_ptr() + 2, y.data_ptr(), y.data_ptr(), 1, 16, 64, 64, None)
     assert st == 3
     assert B.lib.mnnllm_linear_w4a16(y.data_ptr(), y.data_ptr(), y.data_ptr(), 1, 16, 64, 32, None) == 2
-    assert B.lib.mnnllm_linear_w4a16_ex(y.data_ptr(), y.data_ptr(), y.data_ptr(), 1, 16, 64, 64, B.BF16, B.F16, None) == 2
+    assert B.lib.mnnllm_linear_w4a16_ex(y.data_ptr(), y.data_ptr(), y.data_ptr(), 1, 16, 64, 64, B.F32, B.F16, None) == 2
+    assert B.lib.mnnllm_linear_w4a16_ex(y.data_ptr(), y.data_ptr(), y.data_ptr(), 1, 16, 64, 64, 7, B.F16, None) == 1
 
 
 @pytest.mark.parametrize("N,K,M", [(16, 32, 1), (37, 96, 3), (1000, 3584, 1), (4096, 3584, 4), (200, 544, 8), (64, 1024, 9)])

@@ -75,10 +75,22 @@ def test_w4a8_output_and_input_dtypes():
     y32 = run_w4a8(dev(x), packed, M, N, K, group, B.F32)
     assert_close(y32, ref, 2e-4)
     assert_close(run_w4a8(dev(x), packed, M, N, K, group, B.F16), ref)
-    assert_bf16_within_1ulp(run_w4a8(dev(x), packed, M, N, K, group, B.BF16), y32.astype(np.float64))
+    assert_bf16_within_1ulp(run_w4a8(dev(x), packed, M, N, K, group, B.BF16), ref)
     xb = inputs.activations(13, M, K, outliers=True, dtype="bf16")
     yb = run_w4a8(dev(inputs.bf16_bits(xb)).view(torch.bfloat16), packed, M, N, K, group, B.F32, x_dtype=B.BF16)
     assert_close(yb, oracle.linear_w4a8(xb, q, s, z, group))
+
+
+@pytest.mark.parametrize("std", [1e-5, 2e-3, 3.0])
+def test_w4a8_zero_point_term_over_the_weight_range(std):
+    # tiny, small and large weights against activations with a non-zero mean (large group sums A, so
+    # that the zero-point term dominates and cancels against the integer partials)
+    M, N, K, group = 96, 144, 1536, 64
+    W = inputs.weights(21, N, K, std=std)
+    packed, (q, s, z) = B.pack_w4(W, group), oracle.quantize_w4(W, group)
+    x = (inputs.activations(22, M, K).astype(np.float32) + 1.0).astype(np.float16)
+    y = run_w4a8(dev(x), packed, M, N, K, group, B.F32)
+    assert_close(y, oracle.linear_w4a8(x.astype(np.float32), q, s, z, group))
 
 
 def test_w4a8_unusual_zero_points():

@@ -28,6 +28,16 @@ def test_worked_group_from_golden_file():
     assert (np.rint(t) == want).all()
 
 
+def test_scale_and_zero_saturate_at_fp16_max_golden_file():
+    for line in open(os.path.join(GOLDEN, "eq1_saturation.txt")):
+        if not line.strip() or line.startswith("#"):
+            continue
+        w, sb, zb, codes = [f.split() for f in line.split("|")]
+        q, s, z = oracle.quantize_w4(np.array([[float(v) for v in w]], np.float32), 4)
+        assert s[0, 0] == int(sb[0], 16) and z[0, 0] == int(zb[0], 16), line
+        assert q[0].tolist() == [int(c) for c in codes], line
+
+
 @pytest.mark.parametrize("group", [64, 128])
 def test_eq1_endpoints_and_monotone(group):
     W = inputs.weights(11, 24, 4 * group)

@@ -14,6 +14,7 @@ import torch
 
 from paper_2506_10443_b200 import binding as B
 from paper_2506_10443_b200 import inputs
+import oracle
 from gpu_util import TOL, assert_close, dev
 
 
@@ -46,3 +47,7 @@ def test_static_entry_matches_the_workspace_entry_on_two_calls_in_a_row():
         assert B.read_status() == 0
         assert_close(y.cpu().numpy(), y_ref.cpu().numpy().astype(np.float64), TOL)
         assert torch.equal(y, y_ref)   # same kernels, same inputs: in fact identical
+        # and against the CPU oracle, like every other entry point
+        q, s, z = oracle.quantize_w4(W, group)
+        x = inputs.activations(910 + i, M, K, outliers=True).astype(np.float32)
+        assert_close(y.cpu().numpy(), oracle.linear_w4a8(x, q, s, z, group), TOL)
