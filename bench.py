@@ -29,12 +29,50 @@ FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1590.0        # burst; about 1400 sustained
 INT8_OVER_BF16 = 2.0                 # nominal dense tensor-rate ratio (4.5 POPS int8 : 2.25 PFLOPS bf16)
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel from the committed
-# ncu capture (profiles/), keyed by workload; None when no capture matches the current kernel.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {
-    # mean of one layer's four launches (q+k+v, o, gate+up, down), profiles/gemv_w4a16_decode_qwen2_1p5b.txt
-    "decode_qwen2_1p5b_w4a16_g64": 6629760,
+PROFILE_OF = {   # committed ncu summary of the dominant kernel of a workload (profiles/)
+    "decode_qwen2_1p5b_w4a16_g64": "gemv_w4a16_decode_qwen2_1p5b.txt",
+    "decode_qwen2_7b_w4a16_g64": "gemv_w4a16_decode_qwen2_7b.txt",
+    "prefill_qwen2_1p5b_w4a8_g64_m1024": "gemm_w4a8_prefill_qwen2_1p5b_m1024.txt",
+    "prefill_qwen2_1p5b_w4a8_g64_m64": "gemm_w4a8_prefill_qwen2_1p5b_m64.txt",
+    "prefill_qwen2_7b_w4a8_g64_m512": "gemm_w4a8_prefill_qwen2_7b_m512.txt",
 }
+
+
+def kernel_sources_sha1(names):
+    """sha1 over the named files of csrc/: a profile summary records it, so that counters taken
+    from another version of the kernel are recognised."""
+    import hashlib
+
+    h = hashlib.sha1()
+    for n in sorted(names):
+        with open(os.path.join(ROOT, "paper_2506_10443_b200", "csrc", n), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
+
+
+def traffic_from_profile(workload):
+    """dram__bytes_read.sum + dram__bytes_write.sum per launch of the workload's dominant kernel, read
+    from the committed ncu summary; None when there is none or the kernel's sources have changed
+    since (the summary carries 'traffic_bytes_per_launch = N', 'kernel_sources = a.cu b.cuh ...' and
+    'kernel_sources_sha1 = ...' lines)."""
+    import re
+
+    name = PROFILE_OF.get(workload)
+    path = os.path.join(ROOT, "profiles", name) if name else None
+    if not path or not os.path.exists(path):
+        return None
+    text = open(path).read()
+    m = re.search(r"^traffic_bytes_per_launch\s*=\s*(\d+)", text, re.M)
+    src = re.search(r"^kernel_sources\s*=\s*(.+)$", text, re.M)
+    sha = re.search(r"^kernel_sources_sha1\s*=\s*([0-9a-f]{40})", text, re.M)
+    if not (m and src and sha):
+        return None
+    try:
+        if kernel_sources_sha1(src.group(1).split()) != sha.group(1):
+            return None
+    except OSError:
+        return None
+    return int(m.group(1))
 
 
 def measured_peaks():
@@ -269,10 +307,78 @@ def _time_steps(step, steps, warmup):
     return e0.elapsed_time(e1) / steps
 
 
-def secondary_measurements(stack, model, peaks):
-    """The other rows of the hot path on the same GPU, reported beside the headline: the W4A8
-    prefill of a 1024-token prompt over the same packed weights, and the LM-head GEMVs (int4 group
-    128 and int8 per channel, fp32 logits).  Each entry carries its own roofline fraction."""
+def _graph_of(run):
+    """Captures `run(stream)` into a CUDA graph (after one eager call that resolves per-device state)."""
+    import torch
+
+    run()
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    cap = torch.cuda.Stream()
+    cap.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.graph(g, stream=cap):
+        run(cap)
+    torch.cuda.synchronize()
+    return g
+
+
+def _hbm_entry(kernel, nbytes, ms, hbm, **extra):
+    gbs = nbytes / (ms * 1e-3) / 1e9
+    e = {"metric": "decode W4 GEMV GB/s", "value": gbs, "unit": "GB/s", "ms_per_step": ms,
+         "roofline": {"bound": "hbm", "kernel": kernel, "achieved": gbs, "peak": hbm, "unit": "GB/s", "frac": gbs / hbm}}
+    e.update(extra)
+    return e
+
+
+def _tensor_entry(ops, ms, M, int8_peak, ceiling, **extra):
+    tops = ops / (ms * 1e-3) / 1e12
+    roof = {"bound": "tensor", "kernel": "gemm_w4a8_kernel", "achieved": tops, "peak": int8_peak, "unit": "TOP/s",
+            "frac": tops / int8_peak, "frac_of_nominal_4500": tops / 4500.0,
+            "frac_of_measured_int8_mma_ceiling": (tops / ceiling) if ceiling else None}
+    e = {"metric": "prefill W4A8 TOPS", "value": tops, "unit": "TOPS", "ms_per_step": ms,
+         "tokens_per_s": M / (ms * 1e-3), "roofline": roof}
+    e.update(extra)
+    return e
+
+
+def int8_mma_ceiling(device_index):
+    """tcgen05.mma kind::i8 issued back to back on resident shared-memory tiles for >= 100 ms: the
+    ceiling of the instruction at the clock the GPU holds meanwhile (see mnnllm_bench_mma_i8)."""
+    import torch
+
+    from paper_2506_10443_b200 import binding as B
+
+    sms = torch.cuda.get_device_properties(torch.cuda.current_device()).multi_processor_count
+    sampler = ClockSampler(device_index, period_s=0.005)
+    sampler.start()
+    cycles = torch.zeros(sms, dtype=torch.int64, device="cuda")
+    B.bench_mma_i8(40000, cycles)   # warm-up
+    torch.cuda.synchronize()
+    mmas = 3_200_000                # x 64 cycles at full rate: ~0.1-0.15 s
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = time.perf_counter()
+    e0.record()
+    B.bench_mma_i8(mmas, cycles)
+    e1.record()
+    torch.cuda.synchronize()
+    t1 = time.perf_counter()
+    assert B.read_status() == 0
+    ms = e0.elapsed_time(e1)
+    ops = 2.0 * 128 * 128 * 32 * mmas * sms
+    cyc = float(cycles.max().item())
+    sampler.stop()
+    clk = sampler.summary(t0, t1)
+    return {"metric": "tcgen05.mma kind::i8 issue ceiling", "value": ops / (ms * 1e-3) / 1e12, "unit": "TOP/s",
+            "ms": ms, "mmas_per_sm": mmas, "shape": "128x128x32, operands resident in shared memory",
+            "mac_per_clk_per_sm": 128.0 * 128 * 32 * mmas / cyc, "sm_mhz_from_cycles": cyc / (ms * 1e-3) / 1e6,
+            "clocks": clk}
+
+
+def secondary_measurements(stack, model, peaks, device_index):
+    """The other rows of the hot path on the same GPU, reported beside the headline, each with its
+    own roofline: the one-launch form of the same decode step, the single-GEMV workload (cold L2), the
+    W4A8 prefill of 64 / 256 / 1024-token prompts over the same packed weights, the Qwen2-7B decode
+    and prefill stacks, the LM-head GEMVs, and the measured int8 tensor-core ceiling."""
     import torch
 
     from paper_2506_10443_b200 import binding as B
@@ -283,23 +389,78 @@ def secondary_measurements(stack, model, peaks):
     hbm = float(peaks["hbm_gbs"])
     int8_peak = float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])) * INT8_OVER_BF16
 
-    M = 1024
-    pre = LinearStack(model, 3, M, GROUP, outliers=True, weights_from=stack)
-    pre.run_w4a8()
-    assert B.read_status() == 0
-    g = torch.cuda.CUDAGraph()
-    cap = torch.cuda.Stream()
-    cap.wait_stream(torch.cuda.current_stream())
-    with torch.cuda.graph(g, stream=cap):
-        pre.run_w4a8(cap)
-    ms = _time_steps(g.replay, 20, 3)
-    tops = pre.ops / (ms * 1e-3) / 1e12
-    out["prefill_w4a8_m1024"] = {
-        "metric": "prefill W4A8 TOPS", "value": tops, "unit": "TOPS", "ms_per_step": ms, "tokens_per_s": M / (ms * 1e-3),
-        "roofline": {"bound": "tensor", "kernel": "gemm_w4a8_kernel", "achieved": tops, "peak": int8_peak,
-                     "frac": tops / int8_peak, "frac_of_nominal_4500": tops / 4500.0}}
-    del g, pre
+    out["int8_mma_ceiling"] = ceil = int8_mma_ceiling(device_index)
+    ceiling = ceil["value"]
 
+    # the same decode step through the one-launch entry point (mnnllm_linear_w4a16_stack)
+    g = _graph_of(stack.run_w4a16_stack)
+    ms = _time_steps(g.replay, 300, 20)
+    out["decode_one_launch_qwen2_1p5b"] = _hbm_entry(
+        "stack_w4a16_kernel", stack.algorithmic_bytes_w4a16, ms, hbm, launches_per_step=1,
+        note="whole stack as one persistent cooperative launch with device-side dependency counters")
+    del g
+
+    # the single-GEMV workload: x [1, 1536], W [1536, 1536]; L2 flushed before every launch
+    lin = stack.linears[0]
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    xq, pq, yq = stack.x_view(0, "q"), stack.layers[0].packed["q"], stack.y_view(0, "q")
+    times = []
+    for i in range(60):
+        flush.fill_(i & 0xFF)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        B.linear_w4a16(xq, pq, yq, 1, lin.N, lin.K, GROUP)
+        e1.record()
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1))
+    ms = float(np.median(times[10:]))
+    out["single_gemv_1536x1536_m1"] = _hbm_entry(
+        "gemv_w4a16_kernel", inputs.linear_bytes(lin.N, lin.K, GROUP, 1), ms, hbm,
+        note="latency-bound: 1.3 MB is 0.2 us of HBM time; one launch timed alone with events, L2 flushed "
+             "(256 MB written) before each; median of 50")
+    del flush
+
+    for M, reps in ((64, 50), (256, 30), (1024, 20)):
+        pre = LinearStack(model, 3, M, GROUP, outliers=True, weights_from=stack, distinct=4)
+        g = _graph_of(pre.run_w4a8)
+        assert B.read_status() == 0
+        ms = _time_steps(g.replay, reps, 3)
+        e = _tensor_entry(pre.ops, ms, M, int8_peak, ceiling,
+                          note="activations of 4 distinct layers, reused by the others")
+        if M == 64:   # 4 M = 256 int8 operations per weight byte: below the ridge, graded on bytes
+            nbytes = pre.weight_bytes + sum(2 * M * (t.K + t.N) for t in pre.linears) * pre.n_layers
+            gbs = nbytes / (ms * 1e-3) / 1e9
+            e["roofline_hbm"] = {"bound": "hbm", "achieved": gbs, "peak": hbm, "unit": "GB/s", "frac": gbs / hbm}
+        out["prefill_w4a8_m%d" % M] = e
+        del g, pre
+    torch.cuda.empty_cache()
+
+    # Qwen2-7B: decode and a 512-token prefill.  Four layers of distinct weights (524 MB, four times
+    # L2), reused in turn by the 28 layers: every pass streams its weights from DRAM.
+    m7 = inputs.QWEN2_7B
+    s7 = LinearStack(m7, 4, 1, GROUP, distinct=4)
+    g = _graph_of(s7.run_w4a16)
+    ms = _time_steps(g.replay, 100, 10)
+    out["decode_qwen2_7b"] = _hbm_entry(
+        "gemv_w4a16_kernel", s7.algorithmic_bytes_w4a16, ms, hbm, launches_per_step=s7.launches_per_step_w4a16,
+        tokens_per_s=1.0 / (ms * 1e-3), traffic=traffic_from_profile("decode_qwen2_7b_w4a16_g64"),
+        note="28 layers over 4 layers of distinct weights and inputs")
+    del g
+    g = _graph_of(s7.run_w4a16_stack)
+    ms = _time_steps(g.replay, 100, 10)
+    out["decode_one_launch_qwen2_7b"] = _hbm_entry("stack_w4a16_kernel", s7.algorithmic_bytes_w4a16, ms, hbm,
+                                                   launches_per_step=1)
+    del g
+    p7 = LinearStack(m7, 4, 512, GROUP, outliers=True, weights_from=s7, distinct=4)
+    g = _graph_of(p7.run_w4a8)
+    ms = _time_steps(g.replay, 10, 3)
+    out["prefill_qwen2_7b_w4a8_m512"] = _tensor_entry(p7.ops, ms, 512, int8_peak, ceiling,
+                                                      note="28 layers over 4 layers of distinct weights and inputs")
+    assert B.read_status() == 0
+    del g, p7, s7
+    torch.cuda.empty_cache()
+
+    # LM head: int4 group 128 and int8 per channel, fp32 logits
     N, K, grp = inputs.LM_HEAD["N"], inputs.LM_HEAD["K"], inputs.LM_HEAD["group"]
     W = inputs.weights(inputs.seed_for(5, 0, 0, 0), N, K)
     x = torch.from_numpy(inputs.activations(inputs.seed_for(5, 0, 0, 1), 4, K)).cuda()
@@ -307,20 +468,15 @@ def secondary_measurements(stack, model, peaks):
     p4 = torch.from_numpy(B.pack_w4(W, grp)).cuda()
     for Mh in (1, 4):
         ms = _time_steps(lambda: B.linear_w4a16_ex(x, p4, y, Mh, N, K, grp, B.F16, B.F32), 50, 5)
-        nbytes = w4_bytes(N, K, grp) + 2 * Mh * K + 4 * Mh * N
-        gbs = nbytes / (ms * 1e-3) / 1e9
-        out["lm_head_w4a16_g128_m%d" % Mh] = {
-            "metric": "decode W4 GEMV GB/s", "value": gbs, "unit": "GB/s", "us": 1e3 * ms,
-            "roofline": {"bound": "hbm", "kernel": "gemv_w4a16_kernel", "achieved": gbs, "peak": hbm, "frac": gbs / hbm}}
+        out["lm_head_w4a16_g128_m%d" % Mh] = _hbm_entry("gemv_w4a16_kernel", w4_bytes(N, K, grp) + 2 * Mh * K + 4 * Mh * N,
+                                                        ms, hbm)
     del p4
     p8 = torch.from_numpy(B.pack_w8(W)).cuda()
     del W
     ms = _time_steps(lambda: B.linear_w8a16(x, p8, y, 1, N, K, B.F32), 50, 5)
-    nbytes = N * K + 4 * N + 2 * K + 4 * N
-    gbs = nbytes / (ms * 1e-3) / 1e9
-    out["lm_head_w8a16_m1"] = {
-        "metric": "decode W8 GEMV GB/s", "value": gbs, "unit": "GB/s", "us": 1e3 * ms,
-        "roofline": {"bound": "hbm", "kernel": "gemv_w8a16_kernel", "achieved": gbs, "peak": hbm, "frac": gbs / hbm}}
+    e = _hbm_entry("gemv_w8a16_kernel", N * K + 4 * N + 2 * K + 4 * N, ms, hbm)
+    e["metric"] = "decode W8 GEMV GB/s"
+    out["lm_head_w8a16_m1"] = e
     assert B.read_status() == 0
     return out
 
@@ -442,7 +598,7 @@ def run_ours(args):
         roof.update({"frac": roof["achieved"] / roof["peak"], "launches_per_step": launches,
                      "avg_launch_us": 1e3 * ms_per_step / launches,
                      "algorithmic_units_per_launch": step_units / launches,
-                     "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(args.workload)})
+                     "traffic": traffic_from_profile(args.workload)})
         line = {
             "metric": metric, "value": value, "unit": unit, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
@@ -462,7 +618,7 @@ def run_ours(args):
             "roofline": roof,
         }
         if world == 1 and kind == "decode" and not args.no_secondary:
-            line["secondary"] = secondary_measurements(stack, model, peaks)
+            line["secondary"] = secondary_measurements(stack, model, peaks, local_rank)
         if world == 1 and not args.no_cpu_baseline:
             sample, what, threads = oracle_sample(wl, model, args.cpu_seconds)
             t = time.perf_counter()

@@ -271,6 +271,14 @@ int mnnllm_read_status(void* stream, uint32_t* detail);
 #define MNNLLM_DEBUG_TIMEOUT_DETAIL 0x2000u
 int mnnllm_debug_wait_timeout(int max_polls, void* stream);
 
+/* Measurement aid for the prefill roofline (Section 4.2 puts W4A8 on integer matrix instructions;
+ * the measurement itself is this library's): one CTA per SM issues mmas_per_sm (rounded down to a
+ * multiple of 4) back-to-back 128 x 128 x 32 tcgen05.mma kind::i8 on operand tiles resident in
+ * shared memory, nothing else.  Integer operations performed = SMs * mmas * 2 * 128 * 128 * 32; time
+ * it with events on `stream`.  cycles_out: device, one entry per SM (the issuing thread's elapsed SM
+ * clock cycles), or null. */
+int mnnllm_bench_mma_i8(unsigned long long mmas_per_sm, unsigned long long* cycles_out, void* stream);
+
 /* 1 if the current CUDA device can run the kernels (compute capability 10.x), else 0. */
 int mnnllm_device_supported(void);
 

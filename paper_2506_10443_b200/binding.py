@@ -88,6 +88,7 @@ _sig("mnnllm_quantize_activations", _c.c_int, [_P, _c.c_int, _c.c_int, _c.c_int,
 _sig("mnnllm_debug_w4a8_partials", _c.c_int,
      [_P, _c.c_int, _P, _P, _P, _P, _P, _c.c_int, _c.c_int, _c.c_int, _c.c_int, _P])
 _sig("mnnllm_debug_wait_timeout", _c.c_int, [_c.c_int, _P])
+_sig("mnnllm_bench_mma_i8", _c.c_int, [_c.c_ulonglong, _P, _P])
 _sig("mnnllm_read_status", _c.c_int, [_P, _c.POINTER(_c.c_uint32)])
 _sig("mnnllm_device_supported", _c.c_int, [])
 
@@ -96,7 +97,7 @@ EXPORTS = [
     "mnnllm_packed_size_w8", "mnnllm_pack_w8", "mnnllm_unpack_w8", "mnnllm_linear_w4a16", "mnnllm_linear_w4a16_ex",
     "mnnllm_linear_w4a16_batch", "mnnllm_stack_plan_size", "mnnllm_stack_plan_w4a16", "mnnllm_stack_workspace_size",
     "mnnllm_stack_workspace_init", "mnnllm_linear_w4a16_stack", "mnnllm_linear_w8a16", "mnnllm_workspace_size_w4a8", "mnnllm_workspace_min_w4a8", "mnnllm_linear_w4a8", "mnnllm_linear_w4a8_batch", "mnnllm_linear_w4a8_static",
-    "mnnllm_quantize_activations", "mnnllm_debug_w4a8_partials", "mnnllm_debug_wait_timeout", "mnnllm_read_status", "mnnllm_device_supported",
+    "mnnllm_quantize_activations", "mnnllm_debug_w4a8_partials", "mnnllm_debug_wait_timeout", "mnnllm_bench_mma_i8", "mnnllm_read_status", "mnnllm_device_supported",
 ]
 
 
@@ -310,6 +311,11 @@ DEBUG_TIMEOUT_DETAIL = 0x2000
 def debug_wait_timeout(max_polls: int = 3, stream=None) -> None:
     """Enqueues a kernel whose bounded wait runs out on purpose (it records a status code and ends)."""
     _check(lib.mnnllm_debug_wait_timeout(max_polls, _stream(stream)), "debug_wait_timeout")
+
+
+def bench_mma_i8(mmas_per_sm: int, cycles_out=None, stream=None) -> None:
+    """Enqueues the int8 tensor-rate ceiling kernel (see mnnllm_bench_mma_i8)."""
+    _check(lib.mnnllm_bench_mma_i8(mmas_per_sm, _ptr(cycles_out), _stream(stream)), "bench_mma_i8")
 
 
 def read_status_code(stream=None):

@@ -115,14 +115,6 @@ struct WeightMaps {   // the packed bodies as 2-D tensors: codes box and table b
     CUtensorMap pk[kGemmMaxBatch], tab[kGemmMaxBatch];
 };
 
-// K-major operand tile whose rows are 128 bytes, 128B swizzle: 8-row groups are 1024 bytes apart.
-__device__ __forceinline__ uint64_t desc_sw128(uint32_t smem_addr) {
-    return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
-}
-// K-major operand tile whose rows are 32 bytes, 32B swizzle: 8-row groups are 256 bytes apart.
-__device__ __forceinline__ uint64_t desc_sw32(uint32_t smem_addr) {
-    return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | (1ull << 16) | (16ull << 32) | (1ull << 46) | (6ull << 61);
-}
 // instruction descriptors: D format (bits 4-5), A/B formats (7-9, 10-12), both K-major, N >> 3 at
 // bit 17, M >> 4 at bit 24
 // (kind::i8 formats: 0 = unsigned, 1 = signed 8 bit; codes 0..15 and activations a_q + 128 are both unsigned)

@@ -33,7 +33,7 @@ namespace {
 
 constexpr uint32_t kMaxPolls = 1u << 15;  // x 20 us per try: gives up after ~0.65 s
 
-template <int GROUP, int MP>
+template <int GROUP, int MP, bool XBF>   // XBF: activations are bf16 (converted to fp16 as the fragments are built)
 __global__ void __launch_bounds__(kGemvMaxWarps * 32, (MP <= 2 ? 2 : 1))
 gemv_w4a16_kernel(const __grid_constant__ GemvLaunch L, uint32_t* __restrict__ status) {
     using C = Cfg<GROUP, MP>;
@@ -131,7 +131,7 @@ gemv_w4a16_kernel(const __grid_constant__ GemvLaunch L, uint32_t* __restrict__ s
     pdl_wait();
 
     const int tokB = r % MP, gsB = r / MP;  // B-operand role of this lane: column r of the MMA
-    const bool x_bf16 = P.x_dtype == MNNLLM_BF16;
+    constexpr bool x_bf16 = XBF;
     uint32_t B[8][4][2];
     float C1[C::NSETS][2], C2[C::NSETS][2];
     int cur_j = -1, slot = 0;
@@ -326,7 +326,7 @@ size_t smem_bytes(int W, int SR, int S) {
 }
 
 // Raises the kernel's dynamic shared memory limit when a launch needs more than any before it.
-template <int GROUP, int MP>
+template <int GROUP, int MP, bool XBF>
 cudaError_t ensure_smem(size_t smem) {
     struct State { size_t configured; bool carveout_set; };
     static PerDevice<State> state;   // per instantiation and device
@@ -334,14 +334,14 @@ cudaError_t ensure_smem(size_t smem) {
         if (!st.carveout_set) {
             // every launch of the library asks for the same (largest) shared-memory carve-out, so that
             // an SM does not have to re-partition its L1 between consecutive dependent launches
-            cudaError_t e = cudaFuncSetAttribute(gemv_w4a16_kernel<GROUP, MP>,
+            cudaError_t e = cudaFuncSetAttribute(gemv_w4a16_kernel<GROUP, MP, XBF>,
                                                  cudaFuncAttributePreferredSharedMemoryCarveout,
                                                  (int)cudaSharedmemCarveoutMaxShared);
             if (e != cudaSuccess) return e;
             st.carveout_set = true;
         }
         if (smem > st.configured) {
-            cudaError_t e = cudaFuncSetAttribute(gemv_w4a16_kernel<GROUP, MP>,
+            cudaError_t e = cudaFuncSetAttribute(gemv_w4a16_kernel<GROUP, MP, XBF>,
                                                  cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
             if (e != cudaSuccess) return e;
             st.configured = smem;
@@ -350,12 +350,12 @@ cudaError_t ensure_smem(size_t smem) {
     });
 }
 
-template <int GROUP, int MP>
+template <int GROUP, int MP, bool XBF>
 cudaError_t launch_one(const GemvLaunch& L, int n_clusters, int CS, uint32_t* status, cudaStream_t stream) {
     const int W = L.WC * L.SR;
     const size_t smem = smem_bytes<GROUP, MP>(W, L.SR, L.stages);
-    auto kern = gemv_w4a16_kernel<GROUP, MP>;
-    if (cudaError_t e = ensure_smem<GROUP, MP>(smem); e != cudaSuccess) return e;
+    auto kern = gemv_w4a16_kernel<GROUP, MP, XBF>;
+    if (cudaError_t e = ensure_smem<GROUP, MP, XBF>(smem); e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(n_clusters * CS));
     cfg.blockDim = dim3((unsigned)(W * 32));
@@ -373,12 +373,12 @@ cudaError_t launch_one(const GemvLaunch& L, int n_clusters, int CS, uint32_t* st
     return cudaLaunchKernelEx(&cfg, kern, L, status);
 }
 
-template <int GROUP, int MP>
+template <int GROUP, int MP, bool XBF = false>
 int occupancy_of(int W, int SR, int S) {
     int n = 0;
     const size_t smem = smem_bytes<GROUP, MP>(W, SR, S);
-    auto kern = gemv_w4a16_kernel<GROUP, MP>;
-    if (ensure_smem<GROUP, MP>(smem) != cudaSuccess) return 0;
+    auto kern = gemv_w4a16_kernel<GROUP, MP, XBF>;
+    if (ensure_smem<GROUP, MP, XBF>(smem) != cudaSuccess) return 0;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kern, W * 32, smem) != cudaSuccess) return 0;
     return n;
 }
@@ -404,7 +404,10 @@ size_t gemv_w4a16_smem(int group, int MP, int W, int SR, int S) {
 
 cudaError_t gemv_w4a16_launch(const GemvLaunch& L, int group, int MP, int n_clusters, int CS, uint32_t* status,
                               cudaStream_t stream) {
-#define MNN_CASE(G, P) if (group == G && MP == P) return launch_one<G, P>(L, n_clusters, CS, status, stream);
+#define MNN_CASE(G, P)                                                                                   \
+    if (group == G && MP == P)                                                                          \
+        return L.prob[0].x_dtype == MNNLLM_BF16 ? launch_one<G, P, true>(L, n_clusters, CS, status, stream) \
+                                                : launch_one<G, P, false>(L, n_clusters, CS, status, stream);
     MNN_CASE(64, 1) MNN_CASE(64, 2) MNN_CASE(64, 4) MNN_CASE(64, 8)
     MNN_CASE(128, 1) MNN_CASE(128, 2) MNN_CASE(128, 4) MNN_CASE(128, 8)
 #undef MNN_CASE

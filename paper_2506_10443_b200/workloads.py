@@ -42,7 +42,12 @@ class LinearStack:
     """
 
     def __init__(self, model: dict, config: int, M: int, group: int = 64, layers: Optional[int] = None,
-                 outliers: bool = False, device: str = "cuda", weights_from: "Optional[LinearStack]" = None):
+                 outliers: bool = False, device: str = "cuda", weights_from: "Optional[LinearStack]" = None,
+                 distinct: Optional[int] = None):
+        """``distinct`` = d < layers: only the first d layers get arrays of their own; layer l reuses
+        the packed weights and the input activations of layer l mod d (outputs stay separate).  With
+        d layers of weights well above the L2 size every pass still streams from DRAM; it bounds the
+        host time spent drawing random numbers for the large models."""
         self.model, self.config, self.M, self.group = model, config, M, group
         self.n_layers = model["layers"] if layers is None else layers
         self.linears = inputs.stack(model)
@@ -53,16 +58,22 @@ class LinearStack:
         self.weight_bytes = 0
         self.algorithmic_bytes_w4a16 = 0
         self.ops = 0
+        self.distinct = self.n_layers if distinct is None else max(1, min(distinct, self.n_layers))
         for l in range(self.n_layers):
             L = _Layer()
+            src = self.layers[l % self.distinct] if l >= self.distinct else None
             for lin in self.linears:
                 if weights_from is not None:   # same packed weights, other activations
                     L.packed[lin.name] = weights_from.layers[l].packed[lin.name]
+                elif src is not None:
+                    L.packed[lin.name] = src.packed[lin.name]
                 else:
                     W = inputs.weights(inputs.seed_for(config, l, lin.matrix_id, 0), lin.N, lin.K)
                     L.packed[lin.name] = torch.from_numpy(B.pack_w4(W, group)).to(self.device)
                     del W
                 iid = _INPUT_OF[lin.name]
+                if src is not None:
+                    L.x_off[iid] = src.x_off[iid]
                 if iid not in L.x_off:
                     x = inputs.activations(inputs.seed_for(config, l, _INPUT_SEED_ID[iid], 1), M, lin.K,
                                            outliers=outliers)
