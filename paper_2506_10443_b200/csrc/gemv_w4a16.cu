@@ -151,58 +151,52 @@ gemv_w4a16_kernel(const __grid_constant__ GemvLaunch L, uint32_t* __restrict__ s
                     cur_j = j;
                     // ---- new k-chunk: activations -> B fragments, group sums -> correction terms ----
                     const __half* xk = P.x + (size_t)j * kChunkK;
-#pragma unroll
-                    for (int sl = 0; sl < 8; ++sl) {
-                        uint4 u0 = make_uint4(0, 0, 0, 0), u1 = u0;
-                        const int gi = sl / C::SPG;
-                        const bool mine = (sl < ns) && (tokB < L.M) && (gsB == gi % C::GPS);
-                        if (mine) {
-                            const uint4* px =
-                                reinterpret_cast<const uint4*>(xk + (size_t)tokB * P.K + sl * kSlabK4 + 16 * c);
-                            u0 = px[0];
-                            u1 = px[1];
-                            if (x_bf16) { u0 = bf16x8_to_f16x8(u0); u1 = bf16x8_to_f16x8(u1); }
-                        }
-                        B[sl][0][0] = __byte_perm(u0.x, u0.y, 0x5410);
-                        B[sl][0][1] = __byte_perm(u0.z, u0.w, 0x5410);
-                        B[sl][1][0] = __byte_perm(u0.x, u0.y, 0x7632);
-                        B[sl][1][1] = __byte_perm(u0.z, u0.w, 0x7632);
-                        B[sl][2][0] = __byte_perm(u1.x, u1.y, 0x5410);
-                        B[sl][2][1] = __byte_perm(u1.z, u1.w, 0x5410);
-                        B[sl][3][0] = __byte_perm(u1.x, u1.y, 0x7632);
-                        B[sl][3][1] = __byte_perm(u1.z, u1.w, 0x7632);
-                    }
-                    // group sums of the activations: lane (r, c) adds up its 16-k pieces of group
-                    // gsB + GPS * i of token tokB, the four lanes of a quad complete the sum
+                    // a lane holds the slabs of its groups gsB + GPS * s only (its other B entries are
+                    // zero): load those once, take the group sums from the same registers
                     float v1[C::NSETS], v2[C::NSETS];
+                    uint32_t Pm[C::NSETS][C::SPG][4][2];
 #pragma unroll
-                    for (int i = 0; i < C::NSETS; ++i) {
-                        const int gi = gsB + C::GPS * i;
+                    for (int s = 0; s < C::NSETS; ++s) {
                         float lo = 0.f, hi = 0.f;
-                        if (gi < ng && tokB < L.M) {
 #pragma unroll
-                            for (int sp = 0; sp < C::SPG; ++sp) {
-                                const uint4* px = reinterpret_cast<const uint4*>(
-                                    xk + (size_t)tokB * P.K + (gi * C::SPG + sp) * kSlabK4 + 16 * c);
-                                uint4 u0 = px[0], u1 = px[1];
+                        for (int sp = 0; sp < C::SPG; ++sp) {
+                            const int sl = (gsB + C::GPS * s) * C::SPG + sp;
+                            uint4 u0 = make_uint4(0, 0, 0, 0), u1 = u0;
+                            if (sl < ns && tokB < L.M) {
+                                const uint4* px =
+                                    reinterpret_cast<const uint4*>(xk + (size_t)tokB * P.K + sl * kSlabK4 + 16 * c);
+                                u0 = px[0];
+                                u1 = px[1];
                                 if (x_bf16) { u0 = bf16x8_to_f16x8(u0); u1 = bf16x8_to_f16x8(u1); }
-                                float2 f;
-                                f = h2f2(u0.x); lo += f.x + f.y;
-                                f = h2f2(u0.y); lo += f.x + f.y;
-                                f = h2f2(u1.x); lo += f.x + f.y;
-                                f = h2f2(u1.y); lo += f.x + f.y;
-                                f = h2f2(u0.z); hi += f.x + f.y;
-                                f = h2f2(u0.w); hi += f.x + f.y;
-                                f = h2f2(u1.z); hi += f.x + f.y;
-                                f = h2f2(u1.w); hi += f.x + f.y;
                             }
+                            Pm[s][sp][0][0] = __byte_perm(u0.x, u0.y, 0x5410);
+                            Pm[s][sp][0][1] = __byte_perm(u0.z, u0.w, 0x5410);
+                            Pm[s][sp][1][0] = __byte_perm(u0.x, u0.y, 0x7632);
+                            Pm[s][sp][1][1] = __byte_perm(u0.z, u0.w, 0x7632);
+                            Pm[s][sp][2][0] = __byte_perm(u1.x, u1.y, 0x5410);
+                            Pm[s][sp][2][1] = __byte_perm(u1.z, u1.w, 0x5410);
+                            Pm[s][sp][3][0] = __byte_perm(u1.x, u1.y, 0x7632);
+                            Pm[s][sp][3][1] = __byte_perm(u1.z, u1.w, 0x7632);
+                            const float2 a0 = h2f2(u0.x), a1 = h2f2(u0.y), a2 = h2f2(u1.x), a3 = h2f2(u1.y);
+                            const float2 b0 = h2f2(u0.z), b1 = h2f2(u0.w), b2 = h2f2(u1.z), b3 = h2f2(u1.w);
+                            lo += ((a0.x + a0.y) + (a1.x + a1.y)) + ((a2.x + a2.y) + (a3.x + a3.y));
+                            hi += ((b0.x + b0.y) + (b1.x + b1.y)) + ((b2.x + b2.y) + (b3.x + b3.y));
                         }
                         lo += __shfl_xor_sync(0xffffffffu, lo, 1);
                         hi += __shfl_xor_sync(0xffffffffu, hi, 1);
                         lo += __shfl_xor_sync(0xffffffffu, lo, 2);
                         hi += __shfl_xor_sync(0xffffffffu, hi, 2);
-                        v1[i] = 1024.f * lo + 64.f * hi;
-                        v2[i] = lo + hi;
+                        v1[s] = 1024.f * lo + 64.f * hi;
+                        v2[s] = lo + hi;
+                    }
+#pragma unroll
+                    for (int sl = 0; sl < 8; ++sl) {
+                        const int gi = sl / C::SPG;
+                        const bool mine = gsB == gi % C::GPS;
+#pragma unroll
+                        for (int a = 0; a < 4; ++a)
+#pragma unroll
+                            for (int b = 0; b < 2; ++b) B[sl][a][b] = mine ? Pm[gi / C::GPS][sl % C::SPG][a][b] : 0u;
                     }
                     // the correction terms of accumulator column 2c + e = (token, group slot) sit in
                     // the quad whose row index r equals that column
