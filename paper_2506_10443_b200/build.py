@@ -24,6 +24,7 @@ SOURCES = [
     "api_stack.cu",
     "act_quant.cu",
     "gemm_w4a8.cu",
+    "gemm_small_w4a8.cu",
     "api_w4a8.cu",
     "bench_mma_i8.cu",
 ]

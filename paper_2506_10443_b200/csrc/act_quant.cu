@@ -47,7 +47,8 @@ template <typename T>
 __global__ void __launch_bounds__(kThreads) act_quant_kernel(const T* __restrict__ x, int K, int group,
                                                              int8_t* __restrict__ a_q, float* __restrict__ a_scale,
                                                              int32_t* __restrict__ A, uint2* __restrict__ AC, int G4,
-                                                             uint32_t code_xor, uint32_t* __restrict__ clear, int n_clear) {
+                                                             uint32_t code_xor, uint32_t* __restrict__ clear, int n_clear,
+                                                             float* __restrict__ sums_t) {
     __shared__ float warp_max[kThreads / 32];
     ptx::pdl_launch_dependents();
     ptx::pdl_wait();
@@ -112,6 +113,7 @@ __global__ void __launch_bounds__(kThreads) act_quant_kernel(const T* __restrict
             const int g = v / lanes_per_group;
             if (g < G) {
                 if (A != nullptr) A[(size_t)m * G + g] = sum;
+                if (sums_t != nullptr) sums_t[(size_t)g * 64 + m] = (float)sum;   // [G][64], for at most 64 tokens
                 if (AC != nullptr) {
                     const int h = (sum + 32) >> 6;  // floor((sum + 32) / 64)
                     const int l = sum - 64 * h;
@@ -127,7 +129,9 @@ __global__ void __launch_bounds__(kThreads) act_quant_kernel(const T* __restrict
 }  // namespace
 
 cudaError_t act_quant_launch(const void* x, int x_dtype, int M, int K, int group, int8_t* a_q, float* a_scale,
-                             int32_t* A, void* AC, bool offset128, uint32_t* clear, int n_clear, cudaStream_t stream) {
+                             int32_t* A, void* AC, bool offset128, uint32_t* clear, int n_clear, cudaStream_t stream,
+                             float* sums_t) {
+    if (sums_t && M > 64) return cudaErrorInvalidValue;
     if (!clear) n_clear = 0;
     static PerDevice<bool> carveout_set;
     (void)carveout_set.with([](bool& done) {
@@ -157,9 +161,9 @@ cudaError_t act_quant_launch(const void* x, int x_dtype, int M, int K, int group
     cfg.numAttrs = 1;
     if (x_dtype == MNNLLM_F16)
         return cudaLaunchKernelEx(&cfg, act_quant_kernel<__half>, (const __half*)x, K, group, a_q, a_scale, A, ac,
-                                  G4, code_xor, clear, n_clear);
+                                  G4, code_xor, clear, n_clear, sums_t);
     return cudaLaunchKernelEx(&cfg, act_quant_kernel<__nv_bfloat16>, (const __nv_bfloat16*)x, K, group, a_q, a_scale,
-                              A, ac, G4, code_xor, clear, n_clear);
+                              A, ac, G4, code_xor, clear, n_clear, sums_t);
 }
 
 }  // namespace mnnllm

@@ -12,8 +12,11 @@ namespace mnnllm {
 // [M, G4] x 8 bytes with G4 = K / group rounded up to a multiple of 4 (padding written as zeros).
 // With offset128 the codes are stored as unsigned bytes a_q + 128 (what the GEMM multiplies); the
 // sums A and AC are those of the signed codes either way.  `clear` (may be null) is an array of
-// n_clear words that the kernel sets to zero: the counters of the GEMM that follows.
+// n_clear words that the kernel sets to zero: the counters of the GEMM that follows.  `sums_t` (may be
+// null; M <= 64 only) receives the group sums as fp32, transposed: [K / group][64], token fastest
+// (entries of tokens >= M are left as they are).
 cudaError_t act_quant_launch(const void* x, int x_dtype, int M, int K, int group, int8_t* a_q, float* a_scale,
-                             int32_t* A, void* AC, bool offset128, uint32_t* clear, int n_clear, cudaStream_t stream);
+                             int32_t* A, void* AC, bool offset128, uint32_t* clear, int n_clear, cudaStream_t stream,
+                             float* sums_t = nullptr);
 
 }  // namespace mnnllm

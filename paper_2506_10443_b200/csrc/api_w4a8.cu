@@ -2,6 +2,7 @@
 // launches (activation quantiser, then the tensor-core GEMM).
 #include "act_quant.h"
 #include "common.h"
+#include "gemm_small_w4a8.h"
 #include "gemm_w4a8.h"
 #include "layout.h"
 
@@ -19,7 +20,8 @@ int check_xq(const void* x, int x_dtype, int M, int K, int group) {
 
 size_t round256(size_t v) { return (v + 255) & ~(size_t)255; }
 
-// workspace: a_q int8 [M, K] | a_scale fp32 [M] | fp16 group-sum quadruples [M, G4] x 8 bytes
+// workspace: a_q int8 [M, K] | a_scale fp32 [M] | group sums: fp16 quadruples [M, G4] x 8 bytes for the
+//            tensor-memory GEMM, fp32 [G][64] for the short-prompt kernel (M <= 64)
 //            | optional: counters | fp32 parts of tiles that several CTAs share
 struct Workspace {
     size_t a_q, a_scale, ac, total;   // total: what every call needs
@@ -31,7 +33,8 @@ Workspace workspace_layout(int M, int K, int group) {
     w.a_q = 0;
     w.a_scale = round256((size_t)M * K);
     w.ac = w.a_scale + round256((size_t)M * 4);
-    w.total = w.ac + round256((size_t)M * G4 * 8);
+    const size_t sums = (size_t)M * G4 * 8, sums_small = M <= kGemmSmallMaxTokens ? G4 * 64 * 4 : 0;
+    w.total = w.ac + round256(sums > sums_small ? sums : sums_small);
     w.counters = w.total;
     w.scratch = w.counters + round256((size_t)kGemmCounters * 4);
     w.total_split = w.scratch + kGemmScratchBytes;
@@ -111,6 +114,29 @@ int mnnllm_linear_w4a8_batch(const mnnllm_w4a8_problem* problems, int count, con
     float* a_scale = (float*)(ws + w.a_scale);
     void* ac = ws + w.ac;
     uint32_t* counters = split ? (uint32_t*)(ws + w.counters) : nullptr;
+    if (M <= kGemmSmallMaxTokens) {
+        // short prompts: bound by HBM, not by the tensor cores; the GEMV-shaped kernel streams the weights once
+        if (act_quant_launch(x, x_dtype, M, K, group, a_q, a_scale, nullptr, nullptr, false, counters, kGemmCounters,
+                             (cudaStream_t)stream, (float*)ac) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return MNNLLM_ERR_CUDA;
+        }
+        GemmSmallArgs a;
+        a.count = count;
+        for (int i = 0; i < count; ++i) {
+            a.packed[i] = problems[i].packed; a.y[i] = problems[i].y; a.N[i] = problems[i].N; a.y_dtype[i] = problems[i].y_dtype;
+        }
+        a.a_q = a_q; a.a_scale = a_scale; a.a_sums_t = (const float*)ac; a.P = nullptr;
+        a.scratch = split ? (float*)(ws + w.scratch) : nullptr;
+        a.scratch_bytes = kGemmScratchBytes;
+        a.counters = counters; a.n_counters = kGemmCounters;
+        a.M = M; a.K = K; a.group = group;
+        if (gemm_small_w4a8_launch(a, status, (cudaStream_t)stream) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return MNNLLM_ERR_CUDA;
+        }
+        return MNNLLM_OK;
+    }
     // the activations are quantised once for all the matrices of the batch (the same kernel clears
     // the counters of the GEMM)
     if (act_quant_launch(x, x_dtype, M, K, group, a_q, a_scale, nullptr, ac, true, counters, kGemmCounters,
@@ -153,6 +179,24 @@ int mnnllm_debug_w4a8_partials(const void* x, int x_dtype, const void* packed, i
     if (!device_is_supported()) return MNNLLM_ERR_UNSUPPORTED;
     uint32_t* status = status_word_ptr();
     if (!status) return MNNLLM_ERR_CUDA;
+    if (M <= kGemmSmallMaxTokens) {   // the short-prompt kernel multiplies the signed codes as they are
+        if (act_quant_launch(x, x_dtype, M, K, group, a_q, a_scale, A, nullptr, false, nullptr, 0, (cudaStream_t)stream) !=
+            cudaSuccess) {
+            (void)cudaGetLastError();
+            return MNNLLM_ERR_CUDA;
+        }
+        GemmSmallArgs a;
+        a.count = 1;
+        a.packed[0] = packed; a.y[0] = nullptr; a.N[0] = N; a.y_dtype[0] = MNNLLM_F32;
+        a.a_q = a_q; a.a_scale = a_scale; a.a_sums_t = nullptr; a.P = P;
+        a.scratch = nullptr; a.scratch_bytes = 0; a.counters = nullptr; a.n_counters = 0;
+        a.M = M; a.K = K; a.group = group;
+        if (gemm_small_w4a8_launch(a, status, (cudaStream_t)stream) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return MNNLLM_ERR_CUDA;
+        }
+        return MNNLLM_OK;
+    }
     // the GEMM multiplies the codes in their unsigned form (a_q + 128); the caller gets the signed
     // ones, written by a second run of the quantiser once the GEMM has consumed the buffer
     if (act_quant_launch(x, x_dtype, M, K, group, a_q, a_scale, A, nullptr, true, nullptr, 0, (cudaStream_t)stream) !=

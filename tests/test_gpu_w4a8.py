@@ -67,6 +67,58 @@ def test_w4a8_matches_oracle(M, N, K, group):
     assert_close(y, oracle.linear_w4a8(x.astype(np.float32), q, s, z, group))
 
 
+@pytest.mark.parametrize("M,N,K,group", [
+    (7, 48, 512, 64),          # short prompts take the GEMV-shaped kernel (M <= 64): one chunk
+    (8, 1000, 1536, 64),       # ragged last 16-row block
+    (9, 2048, 1536, 64),       # q+k+v rows, two token tiles (the second almost empty)
+    (33, 272, 8960, 64),       # partial last chunk, K cut into parts
+    (64, 8960, 1536, 64),      # gate/up projection at the longest short prompt
+    (64, 1536, 8960, 64),      # down projection: few rows, long K
+    (17, 130, 1024, 128),      # group 128
+    (64, 300, 3712, 128),      # group 128, K = 7.25 chunks
+    (50, 200, 576, 64),        # last chunk of a single group
+])
+def test_w4a8_short_prompt_kernel_matches_oracle(M, N, K, group):
+    W, packed, (q, s, z) = quantized(5 * M + N + K, N, K, group)
+    x = inputs.activations(M + 7 * N + K, M, K, outliers=True)
+    ref = oracle.linear_w4a8(x.astype(np.float32), q, s, z, group)
+    assert_close(run_w4a8(dev(x), packed, M, N, K, group, B.F32), ref, 2e-4)
+    assert_close(run_w4a8(dev(x), packed, M, N, K, group, B.F16), ref)
+    # and every int32 group partial through the same kernel, bit for bit
+    G = K // group
+    P = torch.full((M, N, G), -7777, dtype=torch.int32, device="cuda")
+    a_q = torch.empty((M, K), dtype=torch.int8, device="cuda")
+    a_scale = torch.empty((M,), dtype=torch.float32, device="cuda")
+    A = torch.empty((M, G), dtype=torch.int32, device="cuda")
+    B.debug_w4a8_partials(dev(x), dev(packed), P, a_q, a_scale, A, M, N, K, group)
+    assert B.read_status() == 0
+    aq0, _, _ = oracle.act_quant(x.astype(np.float32), group)
+    assert (a_q.cpu().numpy() == aq0).all()
+    assert (P.cpu().numpy() == oracle.group_partials(aq0, q, group)).all()
+
+
+def test_w4a8_short_prompt_batch_and_bf16_input():
+    M, K, group = 40, 1536, 64
+    shapes = [1536, 256, 250]
+    xb = inputs.activations(71, M, K, outliers=True, dtype="bf16")
+    xd = dev(inputs.bf16_bits(xb)).view(torch.bfloat16)
+    probs, refs, ys, keep = [], [], [], []
+    for i, N in enumerate(shapes):
+        W, packed, (q, s, z) = quantized(72 + i, N, K, group)
+        pd = dev(packed)
+        y = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
+        keep.append(pd)
+        probs.append(dict(packed=pd, y=y, N=N, y_dtype=B.F32))
+        refs.append(oracle.linear_w4a8(xb, q, s, z, group))
+        ys.append(y)
+    nbytes = B.workspace_size_w4a8(M, max(shapes), K, group)
+    ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    B.linear_w4a8_batch(probs, xd, M, K, group, ws, nbytes, x_dtype=B.BF16)
+    assert B.read_status() == 0
+    for y, ref in zip(ys, refs):
+        assert_close(y.cpu().numpy(), ref, 2e-4)
+
+
 def test_w4a8_output_and_input_dtypes():
     M, N, K, group = 70, 272, 1536, 64
     W, packed, (q, s, z) = quantized(11, N, K, group)
