@@ -186,6 +186,8 @@ int mnnllm_linear_w8a16(const void* x, const void* packed, void* y, int M, int N
  *
  *   x          device [M, K] of x_dtype (MNNLLM_F16 or MNNLLM_BF16)
  *   y          device [M, N] of y_dtype, overwritten
+ *   M          prompts of up to 32 tokens are memory-bound (Section 2) and run on a GEMV-shaped kernel
+ *              (warp-level u8 x s8 MMAs on the streamed weights), longer ones on the tensor-memory GEMM
  *   weights    the zero-point term sum_g scale*zero*A is evaluated on the tensor cores from a two-term
  *              fp16 split of scale*zero (about the group's |w_min|): every group needs |w_min| < 256,
  *              and the term is carried to 2^-33 absolute, i.e. without loss for weights whose typical
@@ -262,6 +264,13 @@ int mnnllm_debug_w4a8_partials(const void* x, int x_dtype, const void* packed, i
  * instead of spinning.  This call synchronises `stream`, reads the word, clears it and returns
  * MNNLLM_OK or MNNLLM_ERR_TIMEOUT (detail, if not null, receives the raw word). */
 int mnnllm_read_status(void* stream, uint32_t* detail);
+
+/* mnnllm_linear_w4a8 has two kernels: prompts of up to 32 tokens go to a GEMV-shaped kernel that
+ * streams the weights once (such prompts are bound by memory, Section 2), longer ones to the
+ * tensor-memory GEMM.  This call moves the boundary for the whole process (0..64 tokens; anything
+ * else restores the default) and returns the value in force before: a tuning and test knob.  Both
+ * kernels compute the same int32 group partials; their fp32 sums differ in order only. */
+int mnnllm_debug_set_w4a8_small_max(int max_tokens);
 
 /* Exercises the time-out path without any of the library's kernels having to fail: enqueues a
  * one-warp kernel that waits, with the kernels' own bounded wait, on a barrier nobody arrives at

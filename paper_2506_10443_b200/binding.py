@@ -87,6 +87,7 @@ _sig("mnnllm_linear_w4a8_static", _c.c_int,
 _sig("mnnllm_quantize_activations", _c.c_int, [_P, _c.c_int, _c.c_int, _c.c_int, _c.c_int, _P, _P, _P, _P])
 _sig("mnnllm_debug_w4a8_partials", _c.c_int,
      [_P, _c.c_int, _P, _P, _P, _P, _P, _c.c_int, _c.c_int, _c.c_int, _c.c_int, _P])
+_sig("mnnllm_debug_set_w4a8_small_max", _c.c_int, [_c.c_int])
 _sig("mnnllm_debug_wait_timeout", _c.c_int, [_c.c_int, _P])
 _sig("mnnllm_bench_mma_i8", _c.c_int, [_c.c_ulonglong, _P, _P])
 _sig("mnnllm_read_status", _c.c_int, [_P, _c.POINTER(_c.c_uint32)])
@@ -97,7 +98,7 @@ EXPORTS = [
     "mnnllm_packed_size_w8", "mnnllm_pack_w8", "mnnllm_unpack_w8", "mnnllm_linear_w4a16", "mnnllm_linear_w4a16_ex",
     "mnnllm_linear_w4a16_batch", "mnnllm_stack_plan_size", "mnnllm_stack_plan_w4a16", "mnnllm_stack_workspace_size",
     "mnnllm_stack_workspace_init", "mnnllm_linear_w4a16_stack", "mnnllm_linear_w8a16", "mnnllm_workspace_size_w4a8", "mnnllm_workspace_min_w4a8", "mnnllm_linear_w4a8", "mnnllm_linear_w4a8_batch", "mnnllm_linear_w4a8_static",
-    "mnnllm_quantize_activations", "mnnllm_debug_w4a8_partials", "mnnllm_debug_wait_timeout", "mnnllm_bench_mma_i8", "mnnllm_read_status", "mnnllm_device_supported",
+    "mnnllm_quantize_activations", "mnnllm_debug_w4a8_partials", "mnnllm_debug_set_w4a8_small_max", "mnnllm_debug_wait_timeout", "mnnllm_bench_mma_i8", "mnnllm_read_status", "mnnllm_device_supported",
 ]
 
 
@@ -303,6 +304,12 @@ def quantize_activations(x, M, K, group, a_q, a_scale, A, x_dtype=F16, stream=No
 def debug_w4a8_partials(x, packed, P, a_q, a_scale, A, M, N, K, group, x_dtype=F16, stream=None) -> None:
     _check(lib.mnnllm_debug_w4a8_partials(_ptr(x), x_dtype, _ptr(packed), _ptr(P), _ptr(a_q), _ptr(a_scale), _ptr(A),
                                           M, N, K, group, _stream(stream)), "debug_w4a8_partials")
+
+
+def debug_set_w4a8_small_max(max_tokens: int) -> int:
+    """Moves the token count up to which ``linear_w4a8`` uses its short-prompt kernel (0..64; -1 restores
+    the default); returns the value in force before."""
+    return int(lib.mnnllm_debug_set_w4a8_small_max(max_tokens))
 
 
 DEBUG_TIMEOUT_DETAIL = 0x2000

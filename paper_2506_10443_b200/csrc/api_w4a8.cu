@@ -1,5 +1,7 @@
 // C-ABI entry points of the W4A8 prefill path: argument checks, workspace carve-up, and the two
 // launches (activation quantiser, then the tensor-core GEMM).
+#include <cstdlib>
+
 #include "act_quant.h"
 #include "common.h"
 #include "gemm_small_w4a8.h"
@@ -10,6 +12,11 @@ using namespace mnnllm;
 
 namespace {
 
+// Measured on B200 (Qwen2-1.5B shapes, graph replay): at 16 tokens the GEMV-shaped kernel takes 9-15 us per
+// call against 14-26 us of the tensor-memory GEMM, at 32 tokens 11-21 against 15-26; at 64 tokens the two are
+// level (17-32 against 15-27), its mma.sync main loop being latency-bound by then.
+constexpr int kSmallPathDefaultMax = 32;
+
 int check_xq(const void* x, int x_dtype, int M, int K, int group) {
     if (!x || M < 1 || K < 1) return MNNLLM_ERR_INVALID_ARG;
     if (x_dtype != MNNLLM_F16 && x_dtype != MNNLLM_BF16) return MNNLLM_ERR_UNSUPPORTED;
@@ -19,6 +26,23 @@ int check_xq(const void* x, int x_dtype, int M, int K, int group) {
 }
 
 size_t round256(size_t v) { return (v + 255) & ~(size_t)255; }
+
+// Prompts of up to this many tokens take the GEMV-shaped kernel, longer ones the tensor-memory GEMM.
+// The default can be overridden by the environment (MNNLLM_W4A8_SMALL_MAX = 0..64, read once) or by
+// mnnllm_debug_set_w4a8_small_max: tuning and test knobs.
+int g_small_max_override = -1;
+int small_path_max_tokens() {
+    if (g_small_max_override >= 0) return g_small_max_override;
+    static int from_env = -2;
+    if (from_env == -2) {
+        from_env = -1;
+        if (const char* env = std::getenv("MNNLLM_W4A8_SMALL_MAX")) {
+            const int e = std::atoi(env);
+            if (e >= 0 && e <= kGemmSmallMaxTokens) from_env = e;
+        }
+    }
+    return from_env >= 0 ? from_env : kSmallPathDefaultMax;
+}
 
 // workspace: a_q int8 [M, K] | a_scale fp32 [M] | group sums: fp16 quadruples [M, G4] x 8 bytes for the
 //            tensor-memory GEMM, fp32 [G][64] for the short-prompt kernel (M <= 64)
@@ -114,7 +138,7 @@ int mnnllm_linear_w4a8_batch(const mnnllm_w4a8_problem* problems, int count, con
     float* a_scale = (float*)(ws + w.a_scale);
     void* ac = ws + w.ac;
     uint32_t* counters = split ? (uint32_t*)(ws + w.counters) : nullptr;
-    if (M <= kGemmSmallMaxTokens) {
+    if (M <= small_path_max_tokens()) {
         // short prompts: bound by HBM, not by the tensor cores; the GEMV-shaped kernel streams the weights once
         if (act_quant_launch(x, x_dtype, M, K, group, a_q, a_scale, nullptr, nullptr, false, counters, kGemmCounters,
                              (cudaStream_t)stream, (float*)ac) != cudaSuccess) {
@@ -179,7 +203,7 @@ int mnnllm_debug_w4a8_partials(const void* x, int x_dtype, const void* packed, i
     if (!device_is_supported()) return MNNLLM_ERR_UNSUPPORTED;
     uint32_t* status = status_word_ptr();
     if (!status) return MNNLLM_ERR_CUDA;
-    if (M <= kGemmSmallMaxTokens) {   // the short-prompt kernel multiplies the signed codes as they are
+    if (M <= small_path_max_tokens()) {   // the short-prompt kernel multiplies the signed codes as they are
         if (act_quant_launch(x, x_dtype, M, K, group, a_q, a_scale, A, nullptr, false, nullptr, 0, (cudaStream_t)stream) !=
             cudaSuccess) {
             (void)cudaGetLastError();
@@ -221,6 +245,12 @@ int mnnllm_debug_w4a8_partials(const void* x, int x_dtype, const void* packed, i
         return MNNLLM_ERR_CUDA;
     }
     return MNNLLM_OK;
+}
+
+int mnnllm_debug_set_w4a8_small_max(int max_tokens) {
+    const int before = small_path_max_tokens();
+    g_small_max_override = (max_tokens >= 0 && max_tokens <= kGemmSmallMaxTokens) ? max_tokens : -1;
+    return before;
 }
 
 int mnnllm_linear_w4a8_static(const void* x, const void* packed, void* y, int M, int N, int K, int group, int x_dtype,

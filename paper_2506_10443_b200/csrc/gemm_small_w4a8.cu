@@ -84,7 +84,9 @@ struct Params {
     int parts, chunks_per_part;
 };
 
-template <int GROUP, bool PARTIALS>
+// MT = token tiles of 8 (1, 2, 4 or 8): a compile-time bound, so that the loops over the tiles are
+// straight-line code and the loads and MMAs of different tiles overlap.
+template <int GROUP, bool PARTIALS, int MT>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_small_w4a8_kernel(const __grid_constant__ Params p, uint32_t* __restrict__ status) {
     using C = Geo<GROUP>;
@@ -105,7 +107,6 @@ gemm_small_w4a8_kernel(const __grid_constant__ Params p, uint32_t* __restrict__ 
     const int nj = j1 - j0;
     const int n_active = p.NB - tile * kWarps < kWarps ? p.NB - tile * kWarps : kWarps;
     const int last_ns = p.NS - 8 * (p.NC - 1);
-    const int mt = (p.M + 7) >> 3;                     // token tiles of 8
 
     // token rows beyond M are never copied: they must read as zero codes and zero sums
     for (int i = threadIdx.x; i < (2 * kActBytes + 2 * kAcBytes) / 16; i += kThreads)
@@ -166,9 +167,11 @@ gemm_small_w4a8_kernel(const __grid_constant__ Params p, uint32_t* __restrict__ 
         if (lane == 0)
             for (int jj = 0; jj < kSlots && jj < nj; ++jj) issue(jj);   // weights do not depend on the quantiser
 
-        float acc[8][4];
+        // fp32 accumulators as packed pairs: acc2[tt][0] = (row r; tokens 2c, 2c+1 of tile tt), acc2[tt][1] = row r + 8
+        uint64_t acc2[MT][2];
 #pragma unroll
-        for (int tt = 0; tt < 8; ++tt) acc[tt][0] = acc[tt][1] = acc[tt][2] = acc[tt][3] = 0.f;
+        for (int tt = 0; tt < MT; ++tt) acc2[tt][0] = acc2[tt][1] = 0ull;
+        const uint64_t kMagic2 = f32x2_pack(0x4B400000u, 0x4B400000u);   // (1.5 * 2^23, 1.5 * 2^23)
         constexpr uint32_t NIB = 0x0F0F0F0Fu;
 
         for (int jj = 0; jj < nj; ++jj) {
@@ -193,11 +196,19 @@ gemm_small_w4a8_kernel(const __grid_constant__ Params p, uint32_t* __restrict__ 
                     a[sp][1][0] = w.y & NIB; a[sp][1][1] = w.w & NIB; a[sp][1][2] = (w.y >> 4) & NIB; a[sp][1][3] = (w.w >> 4) & NIB;
                 }
                 const float2 sz0 = h2f2(table[r * ng + gi]), sz1 = h2f2(table[(r + 8) * ng + gi]);
-                const float s0 = sz0.x, s1 = sz1.x, nz0 = -sz0.x * sz0.y, nz1 = -sz1.x * sz1.y;   // s z: exact in fp32
+                // (s, s) and (-s z, -s z) for the two rows; s z is exact in fp32
+                const uint64_t s0 = f32x2_pack(__float_as_uint(sz0.x), __float_as_uint(sz0.x));
+                const uint64_t s1 = f32x2_pack(__float_as_uint(sz1.x), __float_as_uint(sz1.x));
+                const uint32_t nz0b = __float_as_uint(-sz0.x * sz0.y), nz1b = __float_as_uint(-sz1.x * sz1.y);
+                const uint64_t nz0 = f32x2_pack(nz0b, nz0b), nz1 = f32x2_pack(nz1b, nz1b);
 #pragma unroll
-                for (int tt = 0; tt < 8; ++tt) {
-                    if (tt < mt) {
-                        int d[4] = {0, 0, 0, 0};
+                for (int tt = 0; tt < MT; ++tt) {
+                    {
+                        // The accumulator starts at the bit pattern of 1.5 * 2^23: the int32 sum P then IS
+                        // the float 1.5 * 2^23 + P (|P| < 2^22), and one subtraction converts it exactly:
+                        // no conversion instruction, no integer add.
+                        int d[4] = {PARTIALS ? 0 : 0x4B400000, PARTIALS ? 0 : 0x4B400000, PARTIALS ? 0 : 0x4B400000,
+                                    PARTIALS ? 0 : 0x4B400000};
 #pragma unroll
                         for (int sp = 0; sp < C::SPG; ++sp) {
                             const uint4 bq = *reinterpret_cast<const uint4*>(at + (size_t)tt * 8 * kPitch + (gi * C::SPG + sp) * kSlabK4);
@@ -213,16 +224,11 @@ gemm_small_w4a8_kernel(const __grid_constant__ Params p, uint32_t* __restrict__ 
                                 if (m < p.M && n < p.N[sub]) p.P[((size_t)m * p.N[sub] + n) * p.G + g] = d[i];
                             }
                         } else {
-                            const float2 A = *reinterpret_cast<const float2*>(st + gi * kTok + tt * 8);
-                            // int -> float without the conversion pipe: |d| < 2^22, so 1.5 * 2^23 + d is exact
-                            const float f0 = __int_as_float(d[0] + 0x4B400000) - 12582912.f;
-                            const float f1 = __int_as_float(d[1] + 0x4B400000) - 12582912.f;
-                            const float f2 = __int_as_float(d[2] + 0x4B400000) - 12582912.f;
-                            const float f3 = __int_as_float(d[3] + 0x4B400000) - 12582912.f;
-                            acc[tt][0] = fmaf(nz0, A.x, fmaf(s0, f0, acc[tt][0]));
-                            acc[tt][1] = fmaf(nz0, A.y, fmaf(s0, f1, acc[tt][1]));
-                            acc[tt][2] = fmaf(nz1, A.x, fmaf(s1, f2, acc[tt][2]));
-                            acc[tt][3] = fmaf(nz1, A.y, fmaf(s1, f3, acc[tt][3]));
+                            const uint64_t A = *reinterpret_cast<const uint64_t*>(st + gi * kTok + tt * 8);   // sums of tokens 2c, 2c+1
+                            const uint64_t f01 = f32x2_sub(f32x2_pack((uint32_t)d[0], (uint32_t)d[1]), kMagic2);
+                            const uint64_t f23 = f32x2_sub(f32x2_pack((uint32_t)d[2], (uint32_t)d[3]), kMagic2);
+                            acc2[tt][0] = f32x2_fma(nz0, A, f32x2_fma(s0, f01, acc2[tt][0]));
+                            acc2[tt][1] = f32x2_fma(nz1, A, f32x2_fma(s1, f23, acc2[tt][1]));
                         }
                     }
                 }
@@ -235,6 +241,12 @@ gemm_small_w4a8_kernel(const __grid_constant__ Params p, uint32_t* __restrict__ 
             }
         }
 
+        float acc[MT][4];
+#pragma unroll
+        for (int tt = 0; tt < MT; ++tt) {
+            f32x2_unpack(acc2[tt][0], acc[tt][0], acc[tt][1]);
+            f32x2_unpack(acc2[tt][1], acc[tt][2], acc[tt][3]);
+        }
         // a_scale and the cleared counters come from the quantiser, like the tiles already consumed
         pdl_wait();
         if (!PARTIALS) {
@@ -245,7 +257,7 @@ gemm_small_w4a8_kernel(const __grid_constant__ Params p, uint32_t* __restrict__ 
                 // in the order of the k ranges, whoever it is
                 float* mine = p.scratch + ((size_t)(tile * p.parts + part) * kWarps + warp) * (kTok * 16);
 #pragma unroll
-                for (int tt = 0; tt < 8; ++tt)
+                for (int tt = 0; tt < MT; ++tt)
 #pragma unroll
                     for (int i = 0; i < 4; ++i) __stcg(mine + (tt * 4 + i) * 32 + lane, acc[tt][i]);
                 __threadfence();
@@ -258,21 +270,21 @@ gemm_small_w4a8_kernel(const __grid_constant__ Params p, uint32_t* __restrict__ 
                     __threadfence();
                     const float* parts0 = p.scratch + ((size_t)(tile * p.parts) * kWarps + warp) * (kTok * 16);
 #pragma unroll
-                    for (int tt = 0; tt < 8; ++tt)
+                    for (int tt = 0; tt < MT; ++tt)
 #pragma unroll
                         for (int i = 0; i < 4; ++i) acc[tt][i] = 0.f;
                     for (int ks = 0; ks < p.parts; ++ks) {
                         const float* src_p = parts0 + (size_t)ks * kWarps * (kTok * 16);
 #pragma unroll
-                        for (int tt = 0; tt < 8; ++tt)
+                        for (int tt = 0; tt < MT; ++tt)
 #pragma unroll
                             for (int i = 0; i < 4; ++i) acc[tt][i] += __ldcg(src_p + (tt * 4 + i) * 32 + lane);
                     }
                 }
             }
 #pragma unroll
-            for (int tt = 0; tt < 8; ++tt) {
-                if (finish && tt < mt) {
+            for (int tt = 0; tt < MT; ++tt) {
+                if (finish) {
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
                         const int m = tt * 8 + 2 * c + (i & 1), n = n0 + 8 * (i >> 1);
@@ -287,9 +299,9 @@ gemm_small_w4a8_kernel(const __grid_constant__ Params p, uint32_t* __restrict__ 
         for (int i = 0; i < 50; ++i) __nanosleep(1000);
 }
 
-template <int GROUP, bool PARTIALS>
+template <int GROUP, bool PARTIALS, int MT>
 cudaError_t launch(const Params& p, int grid, uint32_t* status, cudaStream_t stream) {
-    auto kern = gemm_small_w4a8_kernel<GROUP, PARTIALS>;
+    auto kern = gemm_small_w4a8_kernel<GROUP, PARTIALS, MT>;
     constexpr size_t smem = smem_bytes<GROUP>();
     static PerDevice<bool> configured;   // per instantiation and device
     if (cudaError_t e = configured.with([&](bool& done) {
@@ -338,24 +350,39 @@ cudaError_t gemm_small_w4a8_launch(const GemmSmallArgs& a, uint32_t* status, cud
     p.row_block_bytes = g0.row_block_bytes;
     p.M = a.M; p.K = a.K; p.G = g0.G; p.NB = nb; p.NC = g0.n_chunks; p.NS = g0.n_slabs;
     const int tiles = (nb + kWarps - 1) / kWarps;
-    // K is cut into parts (whole 512-k chunks) while the launch has fewer CTAs than about one and a
-    // half per SM, as far as the scratch slots (64 KiB per tile and part) and the counters reach.
+    // K may be cut into parts (whole 512-k chunks) that run as separate CTAs and meet through scratch
+    // memory (64 KiB per tile and part).  The number of parts is the one with the shortest critical
+    // path in units of one quantum's time per warp:
+    //     waves of CTAs x (chunks per part + 1.5)  +  (parts > 1 ? 1 + 0.2 x parts : 0)
+    // 1.5 standing for a CTA's prologue and epilogue, the last term for the scratch round trip and the
+    // sum over the parts (fitted to graph-replay timings of the Qwen2-1.5B shapes at 16 to 64 tokens).
     p.parts = 1;
     p.chunks_per_part = p.NC;
     const int n_sm = device_sm_count();
     if (!partials && a.scratch && a.counters && tiles * kWarps <= a.n_counters && n_sm > 0) {
         const long long max_slots = (long long)(a.scratch_bytes / ((size_t)kWarps * kTok * 16 * 4));
-        int want = (3 * n_sm / 2 + tiles - 1) / tiles;
-        if (want > p.NC) want = p.NC;
-        while (want > 1 && (long long)tiles * want > max_slots) --want;
-        if (want > 1) {
-            p.chunks_per_part = (p.NC + want - 1) / want;
-            p.parts = (p.NC + p.chunks_per_part - 1) / p.chunks_per_part;   // no empty part
+        double best = (double)((tiles + n_sm - 1) / n_sm) * (p.NC + 1.5);
+        for (int want = 2; want <= p.NC && (long long)tiles * want <= max_slots; ++want) {
+            const int cpp = (p.NC + want - 1) / want;
+            const int parts = (p.NC + cpp - 1) / cpp;   // no empty part
+            if (parts != want) continue;
+            const double cost = (double)(((long long)tiles * parts + n_sm - 1) / n_sm) * (cpp + 1.5) + 1.0 + 0.2 * parts;
+            if (cost < best) {
+                best = cost;
+                p.parts = parts;
+                p.chunks_per_part = cpp;
+            }
         }
     }
     const int grid = tiles * p.parts;
-    if (a.group == 64) return partials ? launch<64, true>(p, grid, status, stream) : launch<64, false>(p, grid, status, stream);
-    return partials ? launch<128, true>(p, grid, status, stream) : launch<128, false>(p, grid, status, stream);
+    const int mt = a.M <= 8 ? 1 : (a.M <= 16 ? 2 : (a.M <= 32 ? 4 : 8));
+#define MNN_CASE(G, PT, T) if (a.group == G && partials == PT && mt == T) return launch<G, PT, T>(p, grid, status, stream);
+    MNN_CASE(64, false, 1) MNN_CASE(64, false, 2) MNN_CASE(64, false, 4) MNN_CASE(64, false, 8)
+    MNN_CASE(128, false, 1) MNN_CASE(128, false, 2) MNN_CASE(128, false, 4) MNN_CASE(128, false, 8)
+    MNN_CASE(64, true, 1) MNN_CASE(64, true, 2) MNN_CASE(64, true, 4) MNN_CASE(64, true, 8)
+    MNN_CASE(128, true, 1) MNN_CASE(128, true, 2) MNN_CASE(128, true, 4) MNN_CASE(128, true, 8)
+#undef MNN_CASE
+    return cudaErrorInvalidValue;
 }
 
 }  // namespace mnnllm

@@ -67,6 +67,16 @@ def test_w4a8_matches_oracle(M, N, K, group):
     assert_close(y, oracle.linear_w4a8(x.astype(np.float32), q, s, z, group))
 
 
+@pytest.fixture
+def short_prompt_kernel_up_to_64():
+    """By default prompts of up to 32 tokens take the GEMV-shaped kernel; these tests drive it to its
+    limit of 64 tokens (eight token tiles) and put the default back afterwards."""
+    before = B.debug_set_w4a8_small_max(64)
+    yield
+    B.debug_set_w4a8_small_max(-1)
+    assert before == 32
+
+
 @pytest.mark.parametrize("M,N,K,group", [
     (7, 48, 512, 64),          # short prompts take the GEMV-shaped kernel (M <= 64): one chunk
     (8, 1000, 1536, 64),       # ragged last 16-row block
@@ -78,7 +88,7 @@ def test_w4a8_matches_oracle(M, N, K, group):
     (64, 300, 3712, 128),      # group 128, K = 7.25 chunks
     (50, 200, 576, 64),        # last chunk of a single group
 ])
-def test_w4a8_short_prompt_kernel_matches_oracle(M, N, K, group):
+def test_w4a8_short_prompt_kernel_matches_oracle(M, N, K, group, short_prompt_kernel_up_to_64):
     W, packed, (q, s, z) = quantized(5 * M + N + K, N, K, group)
     x = inputs.activations(M + 7 * N + K, M, K, outliers=True)
     ref = oracle.linear_w4a8(x.astype(np.float32), q, s, z, group)
@@ -97,7 +107,7 @@ def test_w4a8_short_prompt_kernel_matches_oracle(M, N, K, group):
     assert (P.cpu().numpy() == oracle.group_partials(aq0, q, group)).all()
 
 
-def test_w4a8_short_prompt_batch_and_bf16_input():
+def test_w4a8_short_prompt_batch_and_bf16_input(short_prompt_kernel_up_to_64):
     M, K, group = 40, 1536, 64
     shapes = [1536, 256, 250]
     xb = inputs.activations(71, M, K, outliers=True, dtype="bf16")
