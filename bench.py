@@ -374,33 +374,24 @@ def int8_mma_ceiling(device_index):
             "clocks": clk}
 
 
-def secondary_measurements(stack, model, peaks, device_index):
-    """The other rows of the hot path on the same GPU, reported beside the headline, each with its
-    own roofline: the one-launch form of the same decode step, the single-GEMV workload (cold L2), the
-    W4A8 prefill of 64 / 256 / 1024-token prompts over the same packed weights, the Qwen2-7B decode
-    and prefill stacks, the LM-head GEMVs, and the measured int8 tensor-core ceiling."""
+def _sec_decode_one_launch(ctx):
+    """The same decode step through the one-launch entry point (mnnllm_linear_w4a16_stack)."""
+    stack = ctx["stack"]()
+    g = _graph_of(stack.run_w4a16_stack)
+    ms = _time_steps(g.replay, 300, 20)
+    return {"decode_one_launch_qwen2_1p5b": _hbm_entry(
+        "stack_w4a16_kernel", stack.algorithmic_bytes_w4a16, ms, ctx["hbm"], launches_per_step=1,
+        note="whole stack as one persistent cooperative launch with device-side dependency counters")}
+
+
+def _sec_single_gemv(ctx):
+    """The single-GEMV workload: x [1, 1536], W [1536, 1536]; L2 flushed before every launch."""
     import torch
 
     from paper_2506_10443_b200 import binding as B
     from paper_2506_10443_b200 import inputs
-    from paper_2506_10443_b200.workloads import LinearStack, w4_bytes
 
-    out = {}
-    hbm = float(peaks["hbm_gbs"])
-    int8_peak = float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])) * INT8_OVER_BF16
-
-    out["int8_mma_ceiling"] = ceil = int8_mma_ceiling(device_index)
-    ceiling = ceil["value"]
-
-    # the same decode step through the one-launch entry point (mnnllm_linear_w4a16_stack)
-    g = _graph_of(stack.run_w4a16_stack)
-    ms = _time_steps(g.replay, 300, 20)
-    out["decode_one_launch_qwen2_1p5b"] = _hbm_entry(
-        "stack_w4a16_kernel", stack.algorithmic_bytes_w4a16, ms, hbm, launches_per_step=1,
-        note="whole stack as one persistent cooperative launch with device-side dependency counters")
-    del g
-
-    # the single-GEMV workload: x [1, 1536], W [1536, 1536]; L2 flushed before every launch
+    stack = ctx["stack"]()
     lin = stack.linears[0]
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
     xq, pq, yq = stack.x_view(0, "q"), stack.layers[0].packed["q"], stack.y_view(0, "q")
@@ -414,31 +405,50 @@ def secondary_measurements(stack, model, peaks, device_index):
         torch.cuda.synchronize()
         times.append(e0.elapsed_time(e1))
     ms = float(np.median(times[10:]))
-    out["single_gemv_1536x1536_m1"] = _hbm_entry(
-        "gemv_w4a16_kernel", inputs.linear_bytes(lin.N, lin.K, GROUP, 1), ms, hbm,
+    return {"single_gemv_1536x1536_m1": _hbm_entry(
+        "gemv_w4a16_kernel", inputs.linear_bytes(lin.N, lin.K, GROUP, 1), ms, ctx["hbm"],
         note="latency-bound: 1.3 MB is 0.2 us of HBM time; one launch timed alone with events, L2 flushed "
-             "(256 MB written) before each; median of 50")
-    del flush
+             "(256 MB written) before each; median of 50")}
 
+
+def _sec_prefill_1p5b(ctx):
+    """W4A8 prefill of 64 / 256 / 1024-token prompts over the stack's packed weights."""
+    import torch
+
+    from paper_2506_10443_b200 import binding as B
+    from paper_2506_10443_b200.workloads import LinearStack
+
+    stack, out = ctx["stack"](), {}
     for M, reps in ((64, 50), (256, 30), (1024, 20)):
-        pre = LinearStack(model, 3, M, GROUP, outliers=True, weights_from=stack, distinct=4)
+        pre = LinearStack(ctx["model"], 3, M, GROUP, outliers=True, weights_from=stack, distinct=4)
         g = _graph_of(pre.run_w4a8)
         assert B.read_status() == 0
         ms = _time_steps(g.replay, reps, 3)
-        e = _tensor_entry(pre.ops, ms, M, int8_peak, ceiling,
+        e = _tensor_entry(pre.ops, ms, M, ctx["int8_peak"], ctx["ceiling"],
                           note="activations of 4 distinct layers, reused by the others")
         if M == 64:   # 4 M = 256 int8 operations per weight byte: below the ridge, graded on bytes
             nbytes = pre.weight_bytes + sum(2 * M * (t.K + t.N) for t in pre.linears) * pre.n_layers
             gbs = nbytes / (ms * 1e-3) / 1e9
-            e["roofline_hbm"] = {"bound": "hbm", "achieved": gbs, "peak": hbm, "unit": "GB/s", "frac": gbs / hbm}
+            e["roofline_hbm"] = {"bound": "hbm", "achieved": gbs, "peak": ctx["hbm"], "unit": "GB/s", "frac": gbs / ctx["hbm"]}
+        e["traffic"] = traffic_from_profile("prefill_qwen2_1p5b_w4a8_g64_m%d" % M)
         out["prefill_w4a8_m%d" % M] = e
         del g, pre
     torch.cuda.empty_cache()
+    return out
 
-    # Qwen2-7B: decode and a 512-token prefill.  Four layers of distinct weights (524 MB, four times
-    # L2), reused in turn by the 28 layers: every pass streams its weights from DRAM.
-    m7 = inputs.QWEN2_7B
-    s7 = LinearStack(m7, 4, 1, GROUP, distinct=4)
+
+def _sec_qwen2_7b(ctx):
+    """Qwen2-7B: decode (launch per group of linears, and one launch) and a 512-token prefill.  Four
+    layers of distinct weights (524 MB, four times L2), reused in turn by the 28 layers: every pass
+    streams its weights from DRAM."""
+    import torch
+
+    from paper_2506_10443_b200 import binding as B
+    from paper_2506_10443_b200 import inputs
+    from paper_2506_10443_b200.workloads import LinearStack
+
+    out, hbm = {}, ctx["hbm"]
+    s7 = LinearStack(inputs.QWEN2_7B, 4, 1, GROUP, distinct=4)
     g = _graph_of(s7.run_w4a16)
     ms = _time_steps(g.replay, 100, 10)
     out["decode_qwen2_7b"] = _hbm_entry(
@@ -451,16 +461,26 @@ def secondary_measurements(stack, model, peaks, device_index):
     out["decode_one_launch_qwen2_7b"] = _hbm_entry("stack_w4a16_kernel", s7.algorithmic_bytes_w4a16, ms, hbm,
                                                    launches_per_step=1)
     del g
-    p7 = LinearStack(m7, 4, 512, GROUP, outliers=True, weights_from=s7, distinct=4)
+    p7 = LinearStack(inputs.QWEN2_7B, 4, 512, GROUP, outliers=True, weights_from=s7, distinct=4)
     g = _graph_of(p7.run_w4a8)
     ms = _time_steps(g.replay, 10, 3)
-    out["prefill_qwen2_7b_w4a8_m512"] = _tensor_entry(p7.ops, ms, 512, int8_peak, ceiling,
+    out["prefill_qwen2_7b_w4a8_m512"] = _tensor_entry(p7.ops, ms, 512, ctx["int8_peak"], ctx["ceiling"],
+                                                      traffic=traffic_from_profile("prefill_qwen2_7b_w4a8_g64_m512"),
                                                       note="28 layers over 4 layers of distinct weights and inputs")
     assert B.read_status() == 0
     del g, p7, s7
     torch.cuda.empty_cache()
+    return out
 
-    # LM head: int4 group 128 and int8 per channel, fp32 logits
+
+def _sec_lm_head(ctx):
+    """LM head 151936 x 3584: int4 group 128 (1 and 4 tokens) and int8 per channel, fp32 logits."""
+    import torch
+
+    from paper_2506_10443_b200 import binding as B
+    from paper_2506_10443_b200 import inputs
+
+    out, hbm = {}, ctx["hbm"]
     N, K, grp = inputs.LM_HEAD["N"], inputs.LM_HEAD["K"], inputs.LM_HEAD["group"]
     W = inputs.weights(inputs.seed_for(5, 0, 0, 0), N, K)
     x = torch.from_numpy(inputs.activations(inputs.seed_for(5, 0, 0, 1), 4, K)).cuda()
@@ -468,8 +488,8 @@ def secondary_measurements(stack, model, peaks, device_index):
     p4 = torch.from_numpy(B.pack_w4(W, grp)).cuda()
     for Mh in (1, 4):
         ms = _time_steps(lambda: B.linear_w4a16_ex(x, p4, y, Mh, N, K, grp, B.F16, B.F32), 50, 5)
-        out["lm_head_w4a16_g128_m%d" % Mh] = _hbm_entry("gemv_w4a16_kernel", w4_bytes(N, K, grp) + 2 * Mh * K + 4 * Mh * N,
-                                                        ms, hbm)
+        out["lm_head_w4a16_g128_m%d" % Mh] = _hbm_entry(
+            "gemv_w4a16_kernel", inputs.w4_bytes(N, K, grp) + 2 * Mh * K + 4 * Mh * N, ms, hbm)
     del p4
     p8 = torch.from_numpy(B.pack_w8(W)).cuda()
     del W
@@ -478,6 +498,33 @@ def secondary_measurements(stack, model, peaks, device_index):
     e["metric"] = "decode W8 GEMV GB/s"
     out["lm_head_w8a16_m1"] = e
     assert B.read_status() == 0
+    return out
+
+
+SECONDARY = {   # name -> function; also runnable alone: python bench.py --secondary-only NAME
+    "decode_one_launch": _sec_decode_one_launch,
+    "single_gemv": _sec_single_gemv,
+    "prefill_1p5b": _sec_prefill_1p5b,
+    "qwen2_7b": _sec_qwen2_7b,
+    "lm_head": _sec_lm_head,
+}
+
+
+def secondary_measurements(stack_fn, model, peaks, device_index, only=None):
+    """The other rows of the hot path on the same GPU, reported beside the headline, each with its
+    own roofline: the measured int8 tensor-core ceiling, the one-launch form of the same decode step,
+    the single-GEMV workload (cold L2), the W4A8 prefill of 64 / 256 / 1024-token prompts over the same
+    packed weights, the Qwen2-7B decode and prefill stacks, the LM-head GEMVs."""
+    out = {}
+    ceil = None
+    if only is None or only.startswith("prefill") or only == "qwen2_7b" or only == "int8_mma_ceiling":
+        out["int8_mma_ceiling"] = ceil = int8_mma_ceiling(device_index)
+    ctx = {"stack": stack_fn, "model": model, "hbm": float(peaks["hbm_gbs"]),
+           "int8_peak": float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])) * INT8_OVER_BF16,
+           "ceiling": ceil["value"] if ceil else None}
+    for name, fn in SECONDARY.items():
+        if only is None or only == name:
+            out.update(fn(ctx))
     return out
 
 
@@ -507,8 +554,23 @@ def run_ours(args):
     kind, M = wl["kind"], wl["M"]
     model = getattr(inputs, wl["model"])
     metric, unit, dtype = metric_of(kind)
-    # every rank: an independent replica of the workload
-    stack = LinearStack(model, wl["config"], M, GROUP, outliers=kind == "prefill")
+    if args.secondary_only:   # one group of the secondary measurements alone (used for profiling)
+        peaks, _ = measured_peaks()
+        made = {}
+
+        def lazy_stack():
+            if "s" not in made:
+                made["s"] = LinearStack(inputs.QWEN2_1P5B, 2, 1, GROUP, distinct=8)   # 210 MB of weights: above L2
+            return made["s"]
+
+        print(json.dumps({"secondary": secondary_measurements(lazy_stack, inputs.QWEN2_1P5B, peaks, local_rank,
+                                                              only=args.secondary_only)}), flush=True)
+        return
+    # every rank: an independent replica of the workload.  The 7B stack draws four layers of distinct
+    # weights (524 MB, four times L2) and reuses them in turn: the host time to draw 6.5 G random
+    # numbers is not part of what is measured, and every pass still streams its weights from DRAM.
+    distinct = 4 if wl["model"] == "QWEN2_7B" else None
+    stack = LinearStack(model, wl["config"], M, GROUP, outliers=kind == "prefill", distinct=distinct)
     run = stack.run_w4a16 if kind == "decode" else stack.run_w4a8
     launches = stack.launches_per_step_w4a16 if kind == "decode" else stack.launches_per_step_w4a8
     step_units = stack.algorithmic_bytes_w4a16 if kind == "decode" else stack.ops
@@ -607,6 +669,7 @@ def run_ours(args):
                 "workload": args.workload, "tokens_per_step": M, "group": GROUP, "layers": stack.n_layers,
                 "linears_per_layer": 7, "weight_bytes": stack.weight_bytes, "algorithmic_units_per_step": step_units,
                 "l2": l2, "cuda_graph": graph is not None,
+                "distinct_layers": stack.distinct,
                 "parallelism": "replicas only" if world > 1 else "single GPU",
             },
             "tokens_per_s": M * world / (ms_per_step * 1e-3),
@@ -618,7 +681,7 @@ def run_ours(args):
             "roofline": roof,
         }
         if world == 1 and kind == "decode" and not args.no_secondary:
-            line["secondary"] = secondary_measurements(stack, model, peaks, local_rank)
+            line["secondary"] = secondary_measurements(lambda: stack, model, peaks, local_rank)
         if world == 1 and not args.no_cpu_baseline:
             sample, what, threads = oracle_sample(wl, model, args.cpu_seconds)
             t = time.perf_counter()
@@ -648,6 +711,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-secondary", action="store_true",
                     help="skip the extra measurements (prefill on the same weights, LM-head GEMVs) added to the line")
+    ap.add_argument("--secondary-only", default=None, choices=sorted(SECONDARY) + ["int8_mma_ceiling"],
+                    help="run one group of the secondary measurements alone and print it")
     ap.add_argument("--cpu-seconds", type=float, default=10.0, help="oracle time budget of the cpu_baseline leg")
     args = ap.parse_args()
     decode = WORKLOADS[args.workload]["kind"] == "decode"
