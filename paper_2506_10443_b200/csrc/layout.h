@@ -12,6 +12,11 @@
 //                    ((w >> 4) & 0x0F0F0F0F) is k 4..7: the int8 expansion needs no shuffle, and
 //                    (w & 0x000F000F), (w & 0x00F000F0) are (k0,k2), (k4,k6) as fp16 mantissa bits.
 //   scale/zero     = [row 0..15][group 0..ng-1] pairs of fp16 (scale, zero), 4 B each.
+//   trailer        (after the last row block, 128-byte aligned) = 16 bytes {uint32 limb_ok, reserved} followed by
+//                    one {int64 row_sum, int32 row_exp, int32 0} per padded row.  It serves the integer-limb form
+//                    of the prefill GEMM: every scale of row n is S[n,g] * 2^row_exp[n] with an integer S;
+//                    limb_ok = 1 when 15 * S < 2^24 for every group of every row (the product q * S fits three
+//                    bytes: the scales of a row may span nine binades) and row_sum[n] = sum_k q[n,k] * S[n,g(k)].
 //
 // W8 (bits = 8), per channel: same blocking with slabs of 16 rows x 32 k (lane L = 4r + c holds
 //   bytes k = 8c .. 8c+7 of row r in w0 w1 and of row r + 8 in w2 w3, natural byte order), 16 slabs
@@ -59,8 +64,19 @@ struct W4Geometry {
     int G;                 // K / group
     size_t chunk_bytes;      // full chunk: 8 slabs + 16 * groups_per_chunk * 4
     size_t row_block_bytes;  // n_slabs * 512 + 16 * G * 4
+    size_t trailer_offset;   // header + n_row_blocks * row_block_bytes, rounded up to 128
     size_t total_bytes;
 };
+constexpr int kTrailerHeadBytes = 16;
+struct W4RowInfo { long long row_sum; int32_t row_exp, pad; };
+constexpr int kLimbMaxShift = 9;   // S = M << shift with M < 2048: 15 * S < 2^24
+
+// A scale's fp16 bit pattern as integer significand M and exponent x: value = M * 2^x (M = 0 for zero).
+MNN_HD void w4_scale_parts(uint32_t bits, int& M, int& x) {
+    const int e = (int)((bits >> 10) & 31u), m = (int)(bits & 1023u);
+    M = e ? 1024 + m : m;
+    x = e ? e - 25 : -24;
+}
 
 MNN_HD W4Geometry w4_geometry(int N, int K, int group) {
     W4Geometry g;
@@ -72,7 +88,9 @@ MNN_HD W4Geometry w4_geometry(int N, int K, int group) {
     g.G = K / group;
     g.chunk_bytes = (size_t)8 * kSlabBytes + (size_t)16 * g.groups_per_chunk * 4;
     g.row_block_bytes = (size_t)g.n_slabs * kSlabBytes + (size_t)16 * g.G * 4;
-    g.total_bytes = kHeaderBytes + (size_t)g.n_row_blocks * g.row_block_bytes;
+    g.trailer_offset = (kHeaderBytes + (size_t)g.n_row_blocks * g.row_block_bytes + 127) & ~(size_t)127;
+    g.total_bytes = g.trailer_offset +
+                    (((size_t)kTrailerHeadBytes + (size_t)g.n_row_blocks * kRowsPerBlock * sizeof(W4RowInfo) + 127) & ~(size_t)127);
     return g;
 }
 

@@ -121,8 +121,13 @@ int mnnllm_pack_w4(const float* W, int N, int K, int group, void* packed_out) {
     h.row_block_bytes = geo.row_block_bytes; h.chunk_bytes = geo.chunk_bytes;
     h.body_bytes = geo.total_bytes - kHeaderBytes;
     std::memcpy(out, &h, sizeof(h));
+    // padding between the last row block and the trailer, and the trailer's head
+    std::memset(out + kHeaderBytes + (size_t)geo.n_row_blocks * geo.row_block_bytes, 0,
+                geo.total_bytes - (kHeaderBytes + (size_t)geo.n_row_blocks * geo.row_block_bytes));
+    W4RowInfo* info = (W4RowInfo*)(out + geo.trailer_offset + kTrailerHeadBytes);
+    int limb_ok = 1;
 
-#pragma omp parallel
+#pragma omp parallel reduction(&& : limb_ok)
     {
         std::vector<uint8_t> q((size_t)16 * K);        // codes of the 16 rows of this block
         std::vector<uint16_t> sb((size_t)16 * geo.G), zb((size_t)16 * geo.G);
@@ -139,6 +144,30 @@ int mnnllm_pack_w4(const float* W, int N, int K, int group, void* packed_out) {
                     std::memset(&q[(size_t)r * K], 0, K);
                     for (int g = 0; g < geo.G; ++g) sb[(size_t)r * geo.G + g] = zb[(size_t)r * geo.G + g] = 0;
                 }
+            }
+            // trailer: the row's scales as integers S * 2^row_exp, and sum_k q * S (integer-limb GEMM)
+            for (int r = 0; r < 16; ++r) {
+                int emin = 1 << 20;
+                for (int g = 0; g < geo.G; ++g) {
+                    int M, x;
+                    w4_scale_parts(sb[(size_t)r * geo.G + g], M, x);
+                    if (M && x < emin) emin = x;
+                }
+                if (emin == (1 << 20)) emin = 0;   // a row of zero scales (padding)
+                long long sum = 0;
+                for (int g = 0; g < geo.G; ++g) {
+                    int M, x;
+                    w4_scale_parts(sb[(size_t)r * geo.G + g], M, x);
+                    const int sh = x - emin;
+                    if (M && sh > kLimbMaxShift) { limb_ok = 0; continue; }
+                    const long long S = M ? ((long long)M << sh) : 0;
+                    long long qs = 0;
+                    for (int k = 0; k < group; ++k) qs += q[(size_t)r * K + (size_t)g * group + k];
+                    sum += qs * S;
+                }
+                info[rb * 16 + r].row_sum = sum;
+                info[rb * 16 + r].row_exp = emin;
+                info[rb * 16 + r].pad = 0;
             }
             for (int j = 0; j < geo.n_chunks; ++j) {
                 uint8_t* chunk = out + w4_chunk_offset(geo, rb, j);
@@ -167,6 +196,7 @@ int mnnllm_pack_w4(const float* W, int N, int K, int group, void* packed_out) {
             }
         }
     }
+    *(uint32_t*)(out + geo.trailer_offset) = (uint32_t)limb_ok;
     return MNNLLM_OK;
 }
 

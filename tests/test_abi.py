@@ -33,9 +33,15 @@ def test_status_strings():
 
 
 def test_packed_size_rejects_bad_arguments():
-    assert B.packed_size_w4(16, 64, 64) == 128 + 512 + 16 * 4
-    assert B.packed_size_w4(17, 64, 64) == 128 + 2 * (512 + 64)
-    assert B.packed_size_w4(16, 128, 128) == 128 + 1024 + 64
+    def trailer(n_row_blocks):   # 16-byte head + 16 bytes per padded row, 128-byte granules
+        return -(-(16 + n_row_blocks * 16 * 16) // 128) * 128
+
+    def up128(v):
+        return -(-v // 128) * 128
+
+    assert B.packed_size_w4(16, 64, 64) == up128(128 + 512 + 16 * 4) + trailer(1)
+    assert B.packed_size_w4(17, 64, 64) == up128(128 + 2 * (512 + 64)) + trailer(2)
+    assert B.packed_size_w4(16, 128, 128) == up128(128 + 1024 + 64) + trailer(1)
     for bad in [(0, 64, 64), (16, 0, 64), (16, 64, 32), (16, 96, 64), (16, 192, 128), (-1, 64, 64)]:
         assert B.packed_size_w4(*bad) == 0
     assert B.packed_size_w8(16, 32) == 128 + 512 + 64

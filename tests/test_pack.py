@@ -45,7 +45,21 @@ def test_documented_layout_nibbles_and_padding():
     q, s, z = oracle.quantize_w4(W, group)
     body = packed[128:]
     row_block = 9 * 512 + 16 * 9 * 4
-    assert len(body) == 2 * row_block
+    trailer_at = -(-(128 + 2 * row_block) // 128) * 128
+    assert len(packed) == trailer_at + -(-(16 + 32 * 16) // 128) * 128
+    # trailer: every scale of a row is an integer S times 2^row_exp, row_sum = sum_k q S (from the oracle's codes)
+    assert packed[trailer_at:trailer_at + 4].view(np.uint32)[0] == 1
+    info = packed[trailer_at + 16: trailer_at + 16 + 32 * 16].view(np.int64).reshape(32, 2)
+    sv = s.view(np.float16).astype(np.float64)
+    for n in range(32):
+        row_sum, row_exp = int(info[n, 0]), int(info[n, 1] & 0xFFFFFFFF)
+        row_exp -= (1 << 32) if row_exp >= (1 << 31) else 0
+        if n >= N:
+            assert row_sum == 0
+            continue
+        S = sv[n] / 2.0 ** row_exp
+        assert (S == np.round(S)).all() and S.min() >= 1 and 15 * S.max() < 2 ** 24
+        assert row_sum == int((q[n].reshape(-1, group).sum(1).astype(np.int64) * S.astype(np.int64)).sum())
     full_chunk = 8 * 512 + 16 * 8 * 4
     nib = [0, 4, 1, 5, 2, 6, 3, 7]
     for rb in range(2):
