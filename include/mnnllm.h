@@ -272,6 +272,18 @@ int mnnllm_read_status(void* stream, uint32_t* detail);
  * kernels compute the same int32 group partials; their fp32 sums differ in order only. */
 int mnnllm_debug_set_w4a8_small_max(int max_tokens);
 
+/* Long prompts have a second tensor-core kernel, off by default.  It folds every group scale into
+ * the integer weight operand (three byte "limbs" of code x integer scale, one int32 accumulator each
+ * over all of K: no per-group rescale; Section 4.2's W4A8 evaluated exactly in integers) and needs
+ * every row's scales within five binades of each other, which the packer records; where that does
+ * not hold the kernel that rescales every group's partial does the work.  Its unpack
+ * costs what the rescale saved, and it measured slower than the default kernel (250 against 390
+ * TOP/s on a Qwen2-1.5B layer at 1024 tokens); it is kept as a checked alternative.  This
+ * call switches it off (0), on for launches with at least 0.6 tiles per SM (1) or on whatever the
+ * number of tiles (2); anything else restores the default (off, or on with MNNLLM_W4A8_LIMB=1 in the
+ * environment); returns 1 if it was on before, else 0: a tuning and test knob. */
+int mnnllm_debug_set_w4a8_limb(int enabled);
+
 /* Exercises the time-out path without any of the library's kernels having to fail: enqueues a
  * one-warp kernel that waits, with the kernels' own bounded wait, on a barrier nobody arrives at
  * (max_polls tries of at most 20 microseconds each, 1..1000), records MNNLLM_DEBUG_TIMEOUT_DETAIL in

@@ -18,6 +18,9 @@
 //   orc_linear_w4a8        the per-group identity  sum_k a*s*(q-z) = s*(sum a*q - z*sum a)  in
 //                          exact rational arithmetic; equality with orc_linear_wa16 when the
 //                          activations are exactly representable in int8.
+//   orc_linear_w8a8        Python-integer brute force of its one dot product per output; equality
+//                          with orc_linear_wa16 on int8-exact activations; the closed form for
+//                          constant codes (y = a_scale s (c - z) sum_k a_q).
 //   fp16 conversions       exhaustive round trip over all 65536 bit patterns and comparison with
 //                          numpy's float16 on random and boundary values.
 //
@@ -247,6 +250,31 @@ void orc_linear_w4a8(const float* x, const uint8_t* q, const uint16_t* scale_bit
     delete[] a_q;
     delete[] a_scale;
     delete[] A_g;
+}
+
+// W8A8 (Section 4.2), per-channel int8 weights (one scale and zero point per weight row, codes
+// 0..255) and per-token int8 activations:
+//   y[m, n] = a_scale[m] * s[n] * (sum_k a_q[m, k] q[n, k]  -  z[n] * sum_k a_q[m, k]), fp64.
+void orc_linear_w8a8(const float* x, const uint8_t* q, const uint16_t* scale_bits,
+                     const uint16_t* zero_bits, int M, int N, int K, double* y) {
+    int8_t* a_q = new int8_t[(size_t)M * K];
+    float* a_scale = new float[M];
+    int32_t* A = new int32_t[M];
+    orc_act_quant(x, M, K, K, a_q, a_scale, A);   // one group = the whole row: A[m] = sum_k a_q[m, k]
+#pragma omp parallel for schedule(static)
+    for (int n = 0; n < N; ++n) {
+        const double s = (double)orc_f16_to_f32(scale_bits[n]);
+        const double z = (double)orc_f16_to_f32(zero_bits[n]);
+        for (int m = 0; m < M; ++m) {
+            int64_t P = 0;
+            for (int k = 0; k < K; ++k)
+                P += (int64_t)a_q[(size_t)m * K + k] * (int64_t)q[(size_t)n * K + k];
+            y[(size_t)m * N + n] = (double)a_scale[m] * (s * ((double)P - z * (double)A[m]));
+        }
+    }
+    delete[] a_q;
+    delete[] a_scale;
+    delete[] A;
 }
 
 int orc_num_threads(void) {

@@ -20,7 +20,7 @@ _LIB = os.path.join(_HERE, "libmnnllm_oracle.so")
 
 __all__ = [
     "build", "num_threads", "f16_to_f32", "f32_to_f16", "quantize_w4", "quantize_w8", "dequant",
-    "linear_wa16", "act_quant", "group_partials", "linear_w4a8",
+    "linear_wa16", "act_quant", "group_partials", "linear_w4a8", "linear_w8a8",
 ]
 
 
@@ -56,6 +56,8 @@ def _l():
         lib.orc_act_quant.argtypes = [P, c.c_int, c.c_int, c.c_int, P, P, P]
         lib.orc_group_partials.argtypes = [P, P, c.c_int, c.c_int, c.c_int, c.c_int, P]
         lib.orc_linear_w4a8.argtypes = [P, P, P, P, c.c_int, c.c_int, c.c_int, c.c_int, P]
+        lib.orc_linear_w8a8.argtypes = [P, P, P, P, c.c_int, c.c_int, c.c_int, P]
+        lib.orc_linear_w8a8.restype = None
         lib.orc_num_threads.restype = c.c_int
         for f in ("orc_quantize_w4", "orc_quantize_w8", "orc_dequant", "orc_linear_wa16",
                   "orc_act_quant", "orc_group_partials", "orc_linear_w4a8"):
@@ -70,6 +72,19 @@ def _p(a: np.ndarray):
 
 def _c(a, dtype) -> np.ndarray:
     return np.ascontiguousarray(a, dtype=dtype)
+
+
+def linear_w8a8(x, q, s_bits, z_bits) -> np.ndarray:
+    """y[M,N] fp64 of the per-channel W8A8 path (activations quantised per token inside)."""
+    x = _c(x, np.float32)
+    q = _c(q, np.uint8)
+    M, K = x.shape
+    N = q.shape[0]
+    s_bits = _c(s_bits, np.uint16)
+    z_bits = _c(z_bits, np.uint16)
+    y = np.empty((M, N), np.float64)
+    _l().orc_linear_w8a8(_p(x), _p(q), _p(s_bits), _p(z_bits), M, N, K, _p(y))
+    return y
 
 
 def num_threads() -> int:

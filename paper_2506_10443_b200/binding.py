@@ -88,6 +88,7 @@ _sig("mnnllm_quantize_activations", _c.c_int, [_P, _c.c_int, _c.c_int, _c.c_int,
 _sig("mnnllm_debug_w4a8_partials", _c.c_int,
      [_P, _c.c_int, _P, _P, _P, _P, _P, _c.c_int, _c.c_int, _c.c_int, _c.c_int, _P])
 _sig("mnnllm_debug_set_w4a8_small_max", _c.c_int, [_c.c_int])
+_sig("mnnllm_debug_set_w4a8_limb", _c.c_int, [_c.c_int])
 _sig("mnnllm_debug_wait_timeout", _c.c_int, [_c.c_int, _P])
 _sig("mnnllm_bench_mma_i8", _c.c_int, [_c.c_ulonglong, _P, _P])
 _sig("mnnllm_read_status", _c.c_int, [_P, _c.POINTER(_c.c_uint32)])
@@ -98,7 +99,7 @@ EXPORTS = [
     "mnnllm_packed_size_w8", "mnnllm_pack_w8", "mnnllm_unpack_w8", "mnnllm_linear_w4a16", "mnnllm_linear_w4a16_ex",
     "mnnllm_linear_w4a16_batch", "mnnllm_stack_plan_size", "mnnllm_stack_plan_w4a16", "mnnllm_stack_workspace_size",
     "mnnllm_stack_workspace_init", "mnnllm_linear_w4a16_stack", "mnnllm_linear_w8a16", "mnnllm_workspace_size_w4a8", "mnnllm_workspace_min_w4a8", "mnnllm_linear_w4a8", "mnnllm_linear_w4a8_batch", "mnnllm_linear_w4a8_static",
-    "mnnllm_quantize_activations", "mnnllm_debug_w4a8_partials", "mnnllm_debug_set_w4a8_small_max", "mnnllm_debug_wait_timeout", "mnnllm_bench_mma_i8", "mnnllm_read_status", "mnnllm_device_supported",
+    "mnnllm_quantize_activations", "mnnllm_debug_w4a8_partials", "mnnllm_debug_set_w4a8_small_max", "mnnllm_debug_set_w4a8_limb", "mnnllm_debug_wait_timeout", "mnnllm_bench_mma_i8", "mnnllm_read_status", "mnnllm_device_supported",
 ]
 
 
@@ -310,6 +311,12 @@ def debug_set_w4a8_small_max(max_tokens: int) -> int:
     """Moves the token count up to which ``linear_w4a8`` uses its short-prompt kernel (0..64; -1 restores
     the default); returns the value in force before."""
     return int(lib.mnnllm_debug_set_w4a8_small_max(max_tokens))
+
+
+def debug_set_w4a8_limb(enabled: int) -> int:
+    """Switches the integer-limb prefill GEMM (an alternative, off by default) off (0), on (1) or on
+    whatever the number of tiles (2); -1 restores the default.  Returns 1 if it was on before."""
+    return int(lib.mnnllm_debug_set_w4a8_limb(enabled))
 
 
 DEBUG_TIMEOUT_DETAIL = 0x2000

@@ -25,6 +25,7 @@ SOURCES = [
     "act_quant.cu",
     "gemm_w4a8.cu",
     "gemm_small_w4a8.cu",
+    "gemm_limb_w4a8.cu",
     "api_w4a8.cu",
     "bench_mma_i8.cu",
 ]

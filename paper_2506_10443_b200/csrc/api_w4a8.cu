@@ -4,6 +4,7 @@
 
 #include "act_quant.h"
 #include "common.h"
+#include "gemm_limb_w4a8.h"
 #include "gemm_small_w4a8.h"
 #include "gemm_w4a8.h"
 #include "layout.h"
@@ -42,6 +43,20 @@ int small_path_max_tokens() {
         }
     }
     return from_env >= 0 ? from_env : kSmallPathDefaultMax;
+}
+
+// The integer-limb GEMM is an alternative that measured slower than the per-group kernel: off unless MNNLLM_W4A8_LIMB=1 (read once) or
+// the debug call switches it on.
+int g_limb_override = -1;
+bool limb_path_forced() { return g_limb_override == 2; }   // whatever the number of tiles (tests)
+bool limb_path_enabled() {
+    if (g_limb_override >= 0) return g_limb_override != 0;
+    static int from_env = -1;
+    if (from_env < 0) {
+        const char* env = std::getenv("MNNLLM_W4A8_LIMB");
+        from_env = (env && env[0] == '1') ? 1 : 0;
+    }
+    return from_env != 0;
 }
 
 // workspace: a_q int8 [M, K] | a_scale fp32 [M] | group sums: fp16 quadruples [M, G4] x 8 bytes for the
@@ -168,8 +183,30 @@ int mnnllm_linear_w4a8_batch(const mnnllm_w4a8_problem* problems, int count, con
         (void)cudaGetLastError();
         return MNNLLM_ERR_CUDA;
     }
+    // When the integer-limb kernel (no per-group drain) is switched on, launches with enough 128 x 128
+    // tiles for the GPU try it first; the tensor-memory GEMM launched behind it returns at once unless
+    // a matrix's scales do not fit the limbs (the packer's flag), in which case the limb kernel has
+    // returned at once.
+    bool limb = false;
+    if (limb_path_enabled()) {
+        GemmLimbArgs l;
+        l.count = count;
+        for (int i = 0; i < count; ++i) {
+            l.packed[i] = problems[i].packed; l.y[i] = problems[i].y; l.N[i] = problems[i].N; l.y_dtype[i] = problems[i].y_dtype;
+        }
+        l.a_q = a_q; l.a_scale = a_scale; l.AC = ac; l.M = M; l.K = K; l.group = group;
+        if (limb_path_forced() || gemm_limb_w4a8_tiles(l) * 5 >= device_sm_count() * 3) {   // at least 0.6 tiles per SM
+            const cudaError_t e = gemm_limb_w4a8_launch(l, status, (cudaStream_t)stream);
+            if (e != cudaSuccess) {
+                (void)cudaGetLastError();
+                return e == cudaErrorNotSupported ? MNNLLM_ERR_UNSUPPORTED : MNNLLM_ERR_CUDA;
+            }
+            limb = true;
+        }
+    }
     GemmW4A8Args a;
     a.count = count;
+    a.skip_if_limb_ok = limb;
     for (int i = 0; i < count; ++i) {
         a.packed[i] = problems[i].packed; a.y[i] = problems[i].y; a.N[i] = problems[i].N; a.y_dtype[i] = problems[i].y_dtype;
     }
@@ -230,6 +267,7 @@ int mnnllm_debug_w4a8_partials(const void* x, int x_dtype, const void* packed, i
     }
     GemmW4A8Args a;
     a.count = 1;
+    a.skip_if_limb_ok = false;
     a.packed[0] = packed; a.y[0] = nullptr; a.N[0] = N; a.y_dtype[0] = MNNLLM_F32;
     a.a_q = a_q; a.a_scale = a_scale; a.AC = nullptr; a.P = P;
     a.scratch = nullptr; a.counters = nullptr;
@@ -245,6 +283,12 @@ int mnnllm_debug_w4a8_partials(const void* x, int x_dtype, const void* packed, i
         return MNNLLM_ERR_CUDA;
     }
     return MNNLLM_OK;
+}
+
+int mnnllm_debug_set_w4a8_limb(int enabled) {
+    const int before = limb_path_enabled() ? 1 : 0;
+    g_limb_override = (enabled >= 0 && enabled <= 2) ? enabled : -1;
+    return before;
 }
 
 int mnnllm_debug_set_w4a8_small_max(int max_tokens) {

@@ -109,6 +109,7 @@ struct Params {
     float* scratch;             // split > 1: [total_tiles * split][kTileT][kTileN] fp32 parts of the tiles
     uint32_t* counters;         // split > 1: [total_tiles][kDrainWarps], zero when the kernel starts
     unsigned long long chunk_bytes;
+    const uint32_t* limb_ok[kGemmMaxBatch];   // null, or the packed buffers' limb flags: return at once if all are set
     Problem prob[kGemmMaxBatch];
 };
 struct WeightMaps {   // the packed bodies as 2-D tensors: codes box and table box per weight matrix
@@ -205,10 +206,21 @@ cudaError_t gemm_w4a8_launch(const GemmW4A8Args& a, uint32_t* status, cudaStream
     p.n_stages = (a.K + kStageK - 1) / kStageK;
     p.count = a.count;
     p.chunk_bytes = geo0.chunk_bytes;
+    for (int i = 0; i < kGemmMaxBatch; ++i) {
+        const int src = i < a.count ? i : 0;
+        p.limb_ok[i] = a.skip_if_limb_ok
+            ? (const uint32_t*)((const uint8_t*)a.packed[src] + w4_geometry(a.N[src], a.K, a.group).trailer_offset) : nullptr;
+    }
     int tiles = 0;
     for (int i = 0; i < kGemmMaxBatch; ++i) {
         const int src = i < a.count ? i : 0;   // unused slots repeat the first matrix
         const W4Geometry geo = w4_geometry(a.N[src], a.K, a.group);
+        if (i >= a.count) {   // ... without encoding its tensor maps again
+            wmaps.pk[i] = wmaps.pk[0];
+            wmaps.tab[i] = wmaps.tab[0];
+            p.prob[i] = p.prob[0];
+            continue;
+        }
         // the packed body as [row block][32-bit words]: codes box 8 x 1 KiB, table box 8 x 512 B
         const cuuint64_t dims[2] = {(cuuint64_t)(geo.row_block_bytes / 4), (cuuint64_t)geo.n_row_blocks};
         const cuuint64_t strides[1] = {(cuuint64_t)geo.row_block_bytes};

@@ -30,6 +30,7 @@ struct GemmW4A8Args {
     float* scratch;        // device, kGemmScratchBytes (null: tiles are never split along K)
     uint32_t* counters;    // device, kGemmCounters words, zero when the kernel starts (null with scratch)
     int M, K, group;
+    bool skip_if_limb_ok;  // the integer-limb kernel was launched ahead: do nothing if every matrix allowed it
 };
 
 // Enqueues the GEMM on `stream`.  With args.P set the kernel stores every int32 group partial and

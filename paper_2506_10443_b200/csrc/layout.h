@@ -13,10 +13,12 @@
 //                    (w & 0x000F000F), (w & 0x00F000F0) are (k0,k2), (k4,k6) as fp16 mantissa bits.
 //   scale/zero     = [row 0..15][group 0..ng-1] pairs of fp16 (scale, zero), 4 B each.
 //   trailer        (after the last row block, 128-byte aligned) = 16 bytes {uint32 limb_ok, reserved} followed by
-//                    one {int64 row_sum, int32 row_exp, int32 0} per padded row.  It serves the integer-limb form
-//                    of the prefill GEMM: every scale of row n is S[n,g] * 2^row_exp[n] with an integer S;
-//                    limb_ok = 1 when 15 * S < 2^24 for every group of every row (the product q * S fits three
-//                    bytes: the scales of a row may span nine binades) and row_sum[n] = sum_k q[n,k] * S[n,g(k)].
+//                    one {int32 limb_sum[3], int32 row_exp} per padded row.  It serves the integer-limb form of
+//                    the prefill GEMM: every scale of row n is S[n,g] * 2^row_exp[n] with an integer S; the product
+//                    q * S = b0 + 256 b1 + 4096 c0 with the byte limbs b0 = (q (S & 4095)) & 255,
+//                    b1 = (q (S & 4095)) >> 8, c0 = q (S >> 12); limb_sum[i] = sum_k limb_i[n,k];
+//                    limb_ok = 1 when S < 2^16 for every group of every row (a row's scales span at most five
+//                    binades beyond the 11 bits of their significands).
 //
 // W8 (bits = 8), per channel: same blocking with slabs of 16 rows x 32 k (lane L = 4r + c holds
 //   bytes k = 8c .. 8c+7 of row r in w0 w1 and of row r + 8 in w2 w3, natural byte order), 16 slabs
@@ -68,8 +70,8 @@ struct W4Geometry {
     size_t total_bytes;
 };
 constexpr int kTrailerHeadBytes = 16;
-struct W4RowInfo { long long row_sum; int32_t row_exp, pad; };
-constexpr int kLimbMaxShift = 9;   // S = M << shift with M < 2048: 15 * S < 2^24
+struct W4RowInfo { int32_t limb_sum[3]; int32_t row_exp; };
+constexpr int kLimbMaxShift = 5;   // S = M << shift with M < 2048: S < 2^16
 
 // A scale's fp16 bit pattern as integer significand M and exponent x: value = M * 2^x (M = 0 for zero).
 MNN_HD void w4_scale_parts(uint32_t bits, int& M, int& x) {

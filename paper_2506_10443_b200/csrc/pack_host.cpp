@@ -154,20 +154,23 @@ int mnnllm_pack_w4(const float* W, int N, int K, int group, void* packed_out) {
                     if (M && x < emin) emin = x;
                 }
                 if (emin == (1 << 20)) emin = 0;   // a row of zero scales (padding)
-                long long sum = 0;
+                long long sums[3] = {0, 0, 0};
                 for (int g = 0; g < geo.G; ++g) {
                     int M, x;
                     w4_scale_parts(sb[(size_t)r * geo.G + g], M, x);
                     const int sh = x - emin;
                     if (M && sh > kLimbMaxShift) { limb_ok = 0; continue; }
                     const long long S = M ? ((long long)M << sh) : 0;
-                    long long qs = 0;
-                    for (int k = 0; k < group; ++k) qs += q[(size_t)r * K + (size_t)g * group + k];
-                    sum += qs * S;
+                    for (int k = 0; k < group; ++k) {
+                        const long long qq = q[(size_t)r * K + (size_t)g * group + k];
+                        const long long lo = qq * (S & 4095);
+                        sums[0] += lo & 255;
+                        sums[1] += lo >> 8;
+                        sums[2] += qq * (S >> 12);
+                    }
                 }
-                info[rb * 16 + r].row_sum = sum;
+                for (int i = 0; i < 3; ++i) info[rb * 16 + r].limb_sum[i] = (int32_t)sums[i];   // < 255 K
                 info[rb * 16 + r].row_exp = emin;
-                info[rb * 16 + r].pad = 0;
             }
             for (int j = 0; j < geo.n_chunks; ++j) {
                 uint8_t* chunk = out + w4_chunk_offset(geo, rb, j);

@@ -129,6 +129,73 @@ def test_w4a8_short_prompt_batch_and_bf16_input(short_prompt_kernel_up_to_64):
         assert_close(y.cpu().numpy(), ref, 2e-4)
 
 
+@pytest.fixture
+def limb_kernel_forced():
+    """The integer-limb GEMM normally takes launches with at least 0.6 tiles per SM; these tests force it
+    onto small shapes too and put the default back afterwards."""
+    B.debug_set_w4a8_limb(2)
+    yield
+    B.debug_set_w4a8_limb(-1)
+
+
+@pytest.mark.parametrize("M,N,K,group", [
+    (65, 16, 64, 64),          # one group
+    (130, 200, 320, 64),       # ragged in M, N and K against the 128 x 128 x 128 tiles
+    (128, 128, 1024, 64),      # one full tile, two chunks
+    (256, 512, 8960, 64),      # long K, partial last chunk
+    (300, 1000, 448, 64),      # G = 7: the last zero-point block holds three groups
+    (77, 130, 1024, 128),      # group 128
+    (512, 384, 3584, 128),
+    (1024, 1536, 1536, 64),    # q projection at the longest prompt
+])
+def test_w4a8_limb_kernel_matches_oracle(M, N, K, group, limb_kernel_forced):
+    W, packed, (q, s, z) = quantized(2 * M + N + K + 1, N, K, group)
+    x = inputs.activations(M + 2 * N + K + 1, M, K, outliers=True)
+    ref = oracle.linear_w4a8(x.astype(np.float32), q, s, z, group)
+    y = run_w4a8(dev(x), packed, M, N, K, group, B.F32)
+    assert_close(y, ref, 2e-4)
+    B.debug_set_w4a8_limb(0)      # and the per-group kernel on the same call, for comparison
+    y_old = run_w4a8(dev(x), packed, M, N, K, group, B.F32)
+    assert_close(y_old, ref, 2e-4)
+    assert_close(y, y_old.astype(np.float64), 1e-5)
+
+
+def test_w4a8_limb_kernel_falls_back_when_a_row_spans_too_many_binades(limb_kernel_forced):
+    # one group of one row is constant (scale 1 against ~0.005 elsewhere: eight binades): the packer
+    # clears the flag, the limb kernel returns at once and the per-group kernel does the work
+    M, N, K, group = 140, 144, 1536, 64
+    W = inputs.weights(31, N, K)
+    W[5, 128:192] = 0.25
+    packed, (q, s, z) = B.pack_w4(W, group), oracle.quantize_w4(W, group)
+    off = -(-(128 + (N // 16) * ((K // 64) * 512 + 16 * (K // group) * 4)) // 128) * 128
+    assert packed[off:off + 4].view(np.uint32)[0] == 0
+    x = inputs.activations(32, M, K, outliers=True)
+    y = run_w4a8(dev(x), packed, M, N, K, group, B.F32)
+    assert_close(y, oracle.linear_w4a8(x.astype(np.float32), q, s, z, group), 2e-4)
+
+
+def test_w4a8_limb_kernel_batch_and_weight_range(limb_kernel_forced):
+    M, K, group = 200, 1536, 64
+    x = (inputs.activations(41, M, K).astype(np.float32) + 1.0).astype(np.float16)
+    for std in (1e-5, 3.0):
+        probs, refs, ys, keep = [], [], [], []
+        for i, N in enumerate((272, 130)):
+            W = inputs.weights(42 + i, N, K, std=std)
+            pd = dev(B.pack_w4(W, group))
+            q, s, z = oracle.quantize_w4(W, group)
+            y = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
+            keep.append(pd)
+            probs.append(dict(packed=pd, y=y, N=N, y_dtype=B.F32))
+            refs.append(oracle.linear_w4a8(x.astype(np.float32), q, s, z, group))
+            ys.append(y)
+        nbytes = B.workspace_size_w4a8(M, 272, K, group)
+        ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+        B.linear_w4a8_batch(probs, dev(x), M, K, group, ws, nbytes)
+        assert B.read_status() == 0
+        for y, ref in zip(ys, refs):
+            assert_close(y.cpu().numpy(), ref)
+
+
 def test_w4a8_output_and_input_dtypes():
     M, N, K, group = 70, 272, 1536, 64
     W, packed, (q, s, z) = quantized(11, N, K, group)

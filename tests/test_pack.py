@@ -49,17 +49,20 @@ def test_documented_layout_nibbles_and_padding():
     assert len(packed) == trailer_at + -(-(16 + 32 * 16) // 128) * 128
     # trailer: every scale of a row is an integer S times 2^row_exp, row_sum = sum_k q S (from the oracle's codes)
     assert packed[trailer_at:trailer_at + 4].view(np.uint32)[0] == 1
-    info = packed[trailer_at + 16: trailer_at + 16 + 32 * 16].view(np.int64).reshape(32, 2)
+    info = packed[trailer_at + 16: trailer_at + 16 + 32 * 16].view(np.int32).reshape(32, 4)
     sv = s.view(np.float16).astype(np.float64)
     for n in range(32):
-        row_sum, row_exp = int(info[n, 0]), int(info[n, 1] & 0xFFFFFFFF)
-        row_exp -= (1 << 32) if row_exp >= (1 << 31) else 0
         if n >= N:
-            assert row_sum == 0
+            assert (info[n, :3] == 0).all()
             continue
-        S = sv[n] / 2.0 ** row_exp
-        assert (S == np.round(S)).all() and S.min() >= 1 and 15 * S.max() < 2 ** 24
-        assert row_sum == int((q[n].reshape(-1, group).sum(1).astype(np.int64) * S.astype(np.int64)).sum())
+        S = sv[n] / 2.0 ** int(info[n, 3])
+        assert (S == np.round(S)).all() and S.min() >= 1 and S.max() < 2 ** 16
+        Sk = np.repeat(S.astype(np.int64), group)             # per k
+        qk = q[n].astype(np.int64)
+        lo = qk * (Sk & 4095)
+        limbs = [lo & 255, lo >> 8, qk * (Sk >> 12)]
+        assert (limbs[0] + 256 * limbs[1] + 4096 * limbs[2] == qk * Sk).all() and max(l.max() for l in limbs) <= 255
+        assert [int(l.sum()) for l in limbs] == [int(v) for v in info[n, :3]]
     full_chunk = 8 * 512 + 16 * 8 * 4
     nib = [0, 4, 1, 5, 2, 6, 3, 7]
     for rb in range(2):
