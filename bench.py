@@ -330,9 +330,9 @@ def _hbm_entry(kernel, nbytes, ms, hbm, **extra):
     return e
 
 
-def _tensor_entry(ops, ms, M, int8_peak, ceiling, **extra):
+def _tensor_entry(ops, ms, M, int8_peak, ceiling, kernel="gemm_w4a8_kernel", **extra):
     tops = ops / (ms * 1e-3) / 1e12
-    roof = {"bound": "tensor", "kernel": "gemm_w4a8_kernel", "achieved": tops, "peak": int8_peak, "unit": "TOP/s",
+    roof = {"bound": "tensor", "kernel": kernel, "achieved": tops, "peak": int8_peak, "unit": "TOP/s",
             "frac": tops / int8_peak, "frac_of_nominal_4500": tops / 4500.0,
             "frac_of_measured_int8_mma_ceiling": (tops / ceiling) if ceiling else None}
     e = {"metric": "prefill W4A8 TOPS", "value": tops, "unit": "TOPS", "ms_per_step": ms,
@@ -501,10 +501,67 @@ def _sec_lm_head(ctx):
     return out
 
 
+def _sec_prefill_w8a8(ctx):
+    """Per-channel W8A8 prefill (no per-group rescale) on Qwen2-1.5B shapes at 1024 tokens: the seven
+    linears of a layer over four layers of distinct int8 weights (188 MB, more than L2), 28 layers per
+    step like the W4A8 rows; and the gate+up shape alone (17920 x 1536), where 560 tiles keep every
+    SM busy."""
+    import torch
+
+    from paper_2506_10443_b200 import binding as B
+    from paper_2506_10443_b200 import inputs
+
+    M, out = 1024, {}
+    lins = inputs.decoder_layer(ctx["model"]["hidden"], ctx["model"]["kv_dim"], ctx["model"]["inter"])
+    ws_bytes = max(B.workspace_size_w8a8(M, t.K) for t in lins)
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+    layers = []
+    for layer in range(4):
+        calls = []
+        for t in lins:
+            W = inputs.weights(inputs.seed_for(6, layer, t.matrix_id, 0), t.N, t.K)
+            x = inputs.activations(inputs.seed_for(6, layer, t.matrix_id, 1), M, t.K, outliers=True)
+            calls.append((torch.from_numpy(x).cuda(), torch.from_numpy(B.pack_w8(W)).cuda(),
+                          torch.empty((M, t.N), dtype=torch.float16, device="cuda"), t.N, t.K))
+        layers.append(calls)
+
+    def run(stream=None):
+        for i in range(ctx["model"]["layers"]):
+            for x, pk, y, N, K in layers[i % 4]:
+                B.linear_w8a8(x, pk, y, M, N, K, ws, ws_bytes, B.F16, B.F16, stream)
+
+    g = _graph_of(run)
+    assert B.read_status() == 0
+    ms = _time_steps(g.replay, 10, 3)
+    ops = 2.0 * M * sum(t.N * t.K for t in lins) * ctx["model"]["layers"]
+    e = _tensor_entry(ops, ms, M, ctx["int8_peak"], ctx["ceiling"], kernel="gemm_w8a8_kernel",
+                      note="seven calls per layer (quantiser + GEMM each), 4 layers of distinct weights and inputs")
+    e["metric"] = "prefill W8A8 TOPS"
+    out["prefill_w8a8_m1024"] = e
+    del g
+    # gate and up stacked: one [17920, 1536] matrix
+    t = lins[4]
+    N2 = 2 * t.N
+    W = inputs.weights(inputs.seed_for(6, 9, 0, 0), N2, t.K)
+    pk = torch.from_numpy(B.pack_w8(W)).cuda()
+    x = layers[0][4][0]
+    y = torch.empty((M, N2), dtype=torch.float16, device="cuda")
+    ms = _time_steps(lambda: B.linear_w8a8(x, pk, y, M, N2, t.K, ws, ws_bytes), 50, 5)
+    e = _tensor_entry(2.0 * M * N2 * t.K, ms, M, ctx["int8_peak"], ctx["ceiling"], kernel="gemm_w8a8_kernel",
+                      note="one call (quantiser + GEMM), M=1024 N=17920 K=1536, weights 27.5 MB (L2-resident)")
+    e["metric"] = "prefill W8A8 TOPS"
+    out["prefill_w8a8_gate_up_m1024"] = e
+    assert B.read_status() == 0
+    del layers, pk, x, y, ws
+    torch.cuda.empty_cache()
+    return out
+
+
 SECONDARY = {   # name -> function; also runnable alone: python bench.py --secondary-only NAME
     "decode_one_launch": _sec_decode_one_launch,
     "single_gemv": _sec_single_gemv,
     "prefill_1p5b": _sec_prefill_1p5b,
+    "prefill_w8a8": _sec_prefill_w8a8,
     "qwen2_7b": _sec_qwen2_7b,
     "lm_head": _sec_lm_head,
 }

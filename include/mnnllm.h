@@ -250,6 +250,24 @@ int mnnllm_linear_w4a8_batch(const mnnllm_w4a8_problem* problems, int count, con
 int mnnllm_linear_w4a8_static(const void* x, const void* packed, void* y, int M, int N, int K, int group,
                               int x_dtype, int y_dtype, void* stream);
 
+/* ------------------------------------------------------------------------------------------------
+ * W8A8 (Section 4.2 names W4A8 and W8A8 as the integer paths): per-channel int8 weights packed by
+ * mnnllm_pack_w8 (one fp16 scale s[n] and zero point z[n] per weight row, codes 0..255) and the
+ * per-token int8 activations defined above:
+ *   y[m, n] = a_scale[m] * s[n] * ( sum_k a_q[m, k] q[n, k]  -  z[n] * sum_k a_q[m, k] )
+ * The integer sum runs over all of K in one int32 tensor-memory accumulator (|sum| <= 127 * 255 * K:
+ * K <= 66048) and is rescaled once, in fp32.  x device [M, K] fp16/bf16 (16-byte aligned), packed
+ * device (128-byte aligned), y device [M, N] fp16/bf16/fp32, K a multiple of 32.  workspace: device,
+ * 256-byte aligned, at least mnnllm_workspace_size_w8a8(M, K) bytes (0 for invalid arguments), owned
+ * by the caller, free for reuse when the stream has passed the call; it holds a_q, a_scale and the
+ * row sums of a_q.  Two launches (quantiser, GEMM) on `stream`; nothing is allocated or synchronised.
+ * Built for prompts (hundreds of tokens); any M >= 1 is computed correctly.
+ * Errors: INVALID_ARG (null pointer, size < 1), UNSUPPORTED (dtype, K % 32 != 0, device),
+ * ALIGNMENT, WORKSPACE (null or too small), CUDA (launch failure; the sticky error is cleared). */
+size_t mnnllm_workspace_size_w8a8(int M, int K);
+int mnnllm_linear_w8a8(const void* x, const void* packed, void* y, int M, int N, int K, int x_dtype, int y_dtype,
+                       void* workspace, size_t workspace_bytes, void* stream);
+
 /* The activation quantiser alone (first kernel of the W4A8 path), writing caller-owned outputs:
  * a_q int8 [M, K], a_scale fp32 [M], A int32 [M, G]. */
 int mnnllm_quantize_activations(const void* x, int x_dtype, int M, int K, int group, int8_t* a_q,

@@ -24,6 +24,8 @@ SOURCES = [
     "api_stack.cu",
     "act_quant.cu",
     "gemm_w4a8.cu",
+    "gemm_w8a8.cu",
+    "api_w8a8.cu",
     "gemm_small_w4a8.cu",
     "gemm_limb_w4a8.cu",
     "api_w4a8.cu",

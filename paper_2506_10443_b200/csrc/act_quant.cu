@@ -48,8 +48,9 @@ __global__ void __launch_bounds__(kThreads) act_quant_kernel(const T* __restrict
                                                              int8_t* __restrict__ a_q, float* __restrict__ a_scale,
                                                              int32_t* __restrict__ A, uint2* __restrict__ AC, int G4,
                                                              uint32_t code_xor, uint32_t* __restrict__ clear, int n_clear,
-                                                             float* __restrict__ sums_t) {
+                                                             float* __restrict__ sums_t, int32_t* __restrict__ row_sum) {
     __shared__ float warp_max[kThreads / 32];
+    __shared__ int warp_tot[kThreads / 32];
     ptx::pdl_launch_dependents();
     ptx::pdl_wait();
     const int m = blockIdx.x;
@@ -80,6 +81,7 @@ __global__ void __launch_bounds__(kThreads) act_quant_kernel(const T* __restrict
     const int G = K / group;
     if (AC != nullptr)  // groups that only pad the row to a multiple of four
         for (int g = G + threadIdx.x; g < G4; g += kThreads) AC[(size_t)m * G4 + g] = make_uint2(0u, 0u);
+    int total = 0;   // this thread's share of the row's sum of codes
     for (int v0 = 0; v0 < nvec; v0 += kThreads) {
         const int v = v0 + threadIdx.x;
         int sum = 0;
@@ -103,6 +105,7 @@ __global__ void __launch_bounds__(kThreads) act_quant_kernel(const T* __restrict
             pk.x ^= code_xor;
             pk.y ^= code_xor;
             out[v] = pk;
+            total += sum;
         }
         // group sums: a group is 8 (or 16) consecutive vectors, i.e. consecutive lanes of one warp
         sum += __shfl_xor_sync(0xffffffffu, sum, 1);
@@ -124,13 +127,25 @@ __global__ void __launch_bounds__(kThreads) act_quant_kernel(const T* __restrict
             }
         }
     }
+    if (row_sum != nullptr) {   // sum_k a_q[m, k]: the zero-point factor of a per-channel weight matrix
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
+        if ((threadIdx.x & 31) == 0) warp_tot[threadIdx.x >> 5] = total;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            int t = 0;
+#pragma unroll
+            for (int w = 0; w < kThreads / 32; ++w) t += warp_tot[w];
+            row_sum[m] = t;
+        }
+    }
 }
 
 }  // namespace
 
 cudaError_t act_quant_launch(const void* x, int x_dtype, int M, int K, int group, int8_t* a_q, float* a_scale,
                              int32_t* A, void* AC, bool offset128, uint32_t* clear, int n_clear, cudaStream_t stream,
-                             float* sums_t) {
+                             float* sums_t, int32_t* row_sum) {
     if (sums_t && M > 64) return cudaErrorInvalidValue;
     if (!clear) n_clear = 0;
     static PerDevice<bool> carveout_set;
@@ -161,9 +176,9 @@ cudaError_t act_quant_launch(const void* x, int x_dtype, int M, int K, int group
     cfg.numAttrs = 1;
     if (x_dtype == MNNLLM_F16)
         return cudaLaunchKernelEx(&cfg, act_quant_kernel<__half>, (const __half*)x, K, group, a_q, a_scale, A, ac,
-                                  G4, code_xor, clear, n_clear, sums_t);
+                                  G4, code_xor, clear, n_clear, sums_t, row_sum);
     return cudaLaunchKernelEx(&cfg, act_quant_kernel<__nv_bfloat16>, (const __nv_bfloat16*)x, K, group, a_q, a_scale,
-                              A, ac, G4, code_xor, clear, n_clear, sums_t);
+                              A, ac, G4, code_xor, clear, n_clear, sums_t, row_sum);
 }
 
 }  // namespace mnnllm

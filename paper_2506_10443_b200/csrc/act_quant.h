@@ -14,9 +14,9 @@ namespace mnnllm {
 // sums A and AC are those of the signed codes either way.  `clear` (may be null) is an array of
 // n_clear words that the kernel sets to zero: the counters of the GEMM that follows.  `sums_t` (may be
 // null; M <= 64 only) receives the group sums as fp32, transposed: [K / group][64], token fastest
-// (entries of tokens >= M are left as they are).
+// (entries of tokens >= M are left as they are).  `row_sum` (may be null) receives sum_k a_q[m, k], int32 [M].
 cudaError_t act_quant_launch(const void* x, int x_dtype, int M, int K, int group, int8_t* a_q, float* a_scale,
                              int32_t* A, void* AC, bool offset128, uint32_t* clear, int n_clear, cudaStream_t stream,
-                             float* sums_t = nullptr);
+                             float* sums_t = nullptr, int32_t* row_sum = nullptr);
 
 }  // namespace mnnllm
