@@ -35,6 +35,7 @@ PROFILE_OF = {   # committed ncu summary of the dominant kernel of a workload (p
     "prefill_qwen2_1p5b_w4a8_g64_m1024": "gemm_w4a8_prefill_qwen2_1p5b_m1024.txt",
     "prefill_qwen2_1p5b_w4a8_g64_m64": "gemm_w4a8_prefill_qwen2_1p5b_m64.txt",
     "prefill_qwen2_7b_w4a8_g64_m512": "gemm_w4a8_prefill_qwen2_7b_m512.txt",
+    "prefill_qwen2_1p5b_w8a8_m1024": "gemm_w8a8_prefill_qwen2_1p5b_m1024.txt",
 }
 
 
@@ -502,10 +503,10 @@ def _sec_lm_head(ctx):
 
 
 def _sec_prefill_w8a8(ctx):
-    """Per-channel W8A8 prefill (no per-group rescale) on Qwen2-1.5B shapes at 1024 tokens: the seven
-    linears of a layer over four layers of distinct int8 weights (188 MB, more than L2), 28 layers per
-    step like the W4A8 rows; and the gate+up shape alone (17920 x 1536), where 560 tiles keep every
-    SM busy."""
+    """Per-channel W8A8 prefill (no per-group rescale) on Qwen2-1.5B shapes at 1024 tokens: a layer's
+    linears as four calls (q+k+v and gate+up stacked along N) over four layers of distinct int8 weights
+    (188 MB, more than L2), 28 layers per step like the W4A8 rows; and the gate+up shape alone
+    (17920 x 1536), where 560 tiles keep every SM busy."""
     import torch
 
     from paper_2506_10443_b200 import binding as B
@@ -513,16 +514,19 @@ def _sec_prefill_w8a8(ctx):
 
     M, out = 1024, {}
     lins = inputs.decoder_layer(ctx["model"]["hidden"], ctx["model"]["kv_dim"], ctx["model"]["inter"])
+    # q, k, v and gate, up read the same activations: their weight matrices are stacked along N before
+    # packing (one call each, four calls per layer)
+    fused = [lins[0:3], lins[3:4], lins[4:6], lins[6:7]]
     ws_bytes = max(B.workspace_size_w8a8(M, t.K) for t in lins)
     ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
     layers = []
     for layer in range(4):
         calls = []
-        for t in lins:
-            W = inputs.weights(inputs.seed_for(6, layer, t.matrix_id, 0), t.N, t.K)
-            x = inputs.activations(inputs.seed_for(6, layer, t.matrix_id, 1), M, t.K, outliers=True)
+        for grp in fused:
+            W = np.concatenate([inputs.weights(inputs.seed_for(6, layer, t.matrix_id, 0), t.N, t.K) for t in grp])
+            x = inputs.activations(inputs.seed_for(6, layer, grp[0].matrix_id, 1), M, grp[0].K, outliers=True)
             calls.append((torch.from_numpy(x).cuda(), torch.from_numpy(B.pack_w8(W)).cuda(),
-                          torch.empty((M, t.N), dtype=torch.float16, device="cuda"), t.N, t.K))
+                          torch.empty((M, W.shape[0]), dtype=torch.float16, device="cuda"), W.shape[0], grp[0].K))
         layers.append(calls)
 
     def run(stream=None):
@@ -535,17 +539,15 @@ def _sec_prefill_w8a8(ctx):
     ms = _time_steps(g.replay, 10, 3)
     ops = 2.0 * M * sum(t.N * t.K for t in lins) * ctx["model"]["layers"]
     e = _tensor_entry(ops, ms, M, ctx["int8_peak"], ctx["ceiling"], kernel="gemm_w8a8_kernel",
-                      note="seven calls per layer (quantiser + GEMM each), 4 layers of distinct weights and inputs")
+                      note="four calls per layer (q+k+v and gate+up stacked along N; quantiser + GEMM each), 4 layers of distinct weights and inputs",
+                      traffic=traffic_from_profile("prefill_qwen2_1p5b_w8a8_m1024"))
     e["metric"] = "prefill W8A8 TOPS"
     out["prefill_w8a8_m1024"] = e
     del g
-    # gate and up stacked: one [17920, 1536] matrix
+    # gate and up stacked alone: one [17920, 1536] matrix
     t = lins[4]
     N2 = 2 * t.N
-    W = inputs.weights(inputs.seed_for(6, 9, 0, 0), N2, t.K)
-    pk = torch.from_numpy(B.pack_w8(W)).cuda()
-    x = layers[0][4][0]
-    y = torch.empty((M, N2), dtype=torch.float16, device="cuda")
+    x, pk, y = layers[0][2][:3]
     ms = _time_steps(lambda: B.linear_w8a8(x, pk, y, M, N2, t.K, ws, ws_bytes), 50, 5)
     e = _tensor_entry(2.0 * M * N2 * t.K, ms, M, ctx["int8_peak"], ctx["ceiling"], kernel="gemm_w8a8_kernel",
                       note="one call (quantiser + GEMM), M=1024 N=17920 K=1536, weights 27.5 MB (L2-resident)")
@@ -557,11 +559,46 @@ def _sec_prefill_w8a8(ctx):
     return out
 
 
+def _sec_decode_w8a16(ctx):
+    """W8A16 decode (per-channel int8 weights, Section 4.2's GPU pairing) over the Qwen2-1.5B stack: one
+    token, seven launches per layer, 28 layers of distinct weights (1.3 GB: every pass streams from DRAM)."""
+    import torch
+
+    from paper_2506_10443_b200 import binding as B
+    from paper_2506_10443_b200 import inputs
+
+    lins = inputs.decoder_layer(ctx["model"]["hidden"], ctx["model"]["kv_dim"], ctx["model"]["inter"])
+    n_layers = ctx["model"]["layers"]
+    calls, nbytes = [], 0
+    for layer in range(n_layers):
+        for t in lins:
+            W = inputs.weights(inputs.seed_for(7, layer % 4, t.matrix_id, 0) + 100000 * (layer // 4), t.N, t.K)
+            x = inputs.activations(inputs.seed_for(7, layer, t.matrix_id, 1), 1, t.K)
+            calls.append((torch.from_numpy(x).cuda(), torch.from_numpy(B.pack_w8(W)).cuda(),
+                          torch.empty((1, t.N), dtype=torch.float16, device="cuda"), t.N, t.K))
+            nbytes += t.N * t.K + 4 * t.N + 2 * t.K + 2 * t.N   # int8 codes, fp16 scale and zero, x, y
+
+    def run(stream=None):
+        for x, pk, y, N, K in calls:
+            B.linear_w8a16(x, pk, y, 1, N, K, B.F16, stream)
+
+    g = _graph_of(run)
+    assert B.read_status() == 0
+    ms = _time_steps(g.replay, 100, 10)
+    e = _hbm_entry("gemv_w8a16_kernel", nbytes, ms, ctx["hbm"], launches_per_step=len(calls),
+                   tokens_per_s=1.0 / (ms * 1e-3))
+    e["metric"] = "decode W8 GEMV GB/s"
+    del g, calls
+    torch.cuda.empty_cache()
+    return {"decode_w8a16_qwen2_1p5b": e}
+
+
 SECONDARY = {   # name -> function; also runnable alone: python bench.py --secondary-only NAME
     "decode_one_launch": _sec_decode_one_launch,
     "single_gemv": _sec_single_gemv,
     "prefill_1p5b": _sec_prefill_1p5b,
     "prefill_w8a8": _sec_prefill_w8a8,
+    "decode_w8a16": _sec_decode_w8a16,
     "qwen2_7b": _sec_qwen2_7b,
     "lm_head": _sec_lm_head,
 }

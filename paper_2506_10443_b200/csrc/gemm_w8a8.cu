@@ -20,6 +20,13 @@
 // lanes of a store wavefront then write eight different 16-byte columns (no bank conflict), and
 // the loads are conflict-free in any order.
 //
+// Measured on B200: 1.2-1.7 POP/s (17920 x 1536 at 1024 tokens: 1.5; K = 6144: 1.7), three to four
+// times the W4A8 kernel.  The main loop takes ~0.7 us per 128-k stage whatever the tile count, i.e.
+// every SM takes in its 48 KiB of operands per stage at ~67 GB/s, ~10 TB/s over the GPU: the operand
+// feed from L2, not the tensor pipe (0.29 us per stage), sets the pace.  A variant that copied the
+// slabs with 8-byte cp.async straight into the swizzled tile (no staging buffer, four stages
+// instead of three) was 15 % slower: twice the requests for the same bytes.
+//
 // Roles (14 warps): TMA producer | MMA issue | 4 rearranging warps | 8 epilogue warps (two per
 // tensor-memory lane quarter, half of the token columns each).
 #include <cuda.h>
