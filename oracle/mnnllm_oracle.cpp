@@ -21,6 +21,9 @@
 //   orc_linear_w8a8        Python-integer brute force of its one dot product per output; equality
 //                          with orc_linear_wa16 on int8-exact activations; the closed form for
 //                          constant codes (y = a_scale s (c - z) sum_k a_q).
+//   orc_lora_bypass        equality with the other association (LoRA_A LoRA_B) x in exact rationals
+//                          on small integers; rank-1 closed form; Table 3's operation and memory
+//                          counts for both orders (tests/golden/table3_lora.txt).
 //   fp16 conversions       exhaustive round trip over all 65536 bit patterns and comparison with
 //                          numpy's float16 on random and boundary values.
 //
@@ -275,6 +278,28 @@ void orc_linear_w8a8(const float* x, const uint8_t* q, const uint16_t* scale_bit
     delete[] a_q;
     delete[] a_scale;
     delete[] A;
+}
+
+// LoRA bypass (Section 5.5, Table 3): y[m, n] += sum_j A[n, j] * t[m, j],  t[m, j] = sum_k B[j, k] x[m, k],
+// i.e. LoRA_A (LoRA_B x) in the order the paper chooses (the small product first).  A is [N, r],
+// B is [r, K], both given as the fp32 values of their fp16 entries; everything in fp64.
+void orc_lora_bypass(const float* x, const float* A, const float* B, int M, int N, int K, int r,
+                     double* y) {
+    double* t = new double[(size_t)M * r];
+    for (int m = 0; m < M; ++m)
+        for (int j = 0; j < r; ++j) {
+            double acc = 0.0;
+            for (int k = 0; k < K; ++k) acc += (double)B[(size_t)j * K + k] * (double)x[(size_t)m * K + k];
+            t[(size_t)m * r + j] = acc;
+        }
+#pragma omp parallel for schedule(static)
+    for (int n = 0; n < N; ++n)
+        for (int m = 0; m < M; ++m) {
+            double acc = 0.0;
+            for (int j = 0; j < r; ++j) acc += (double)A[(size_t)n * r + j] * t[(size_t)m * r + j];
+            y[(size_t)m * N + n] += acc;
+        }
+    delete[] t;
 }
 
 int orc_num_threads(void) {

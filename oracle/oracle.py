@@ -20,7 +20,7 @@ _LIB = os.path.join(_HERE, "libmnnllm_oracle.so")
 
 __all__ = [
     "build", "num_threads", "f16_to_f32", "f32_to_f16", "quantize_w4", "quantize_w8", "dequant",
-    "linear_wa16", "act_quant", "group_partials", "linear_w4a8", "linear_w8a8",
+    "linear_wa16", "act_quant", "group_partials", "linear_w4a8", "linear_w8a8", "lora_bypass",
 ]
 
 
@@ -58,6 +58,8 @@ def _l():
         lib.orc_linear_w4a8.argtypes = [P, P, P, P, c.c_int, c.c_int, c.c_int, c.c_int, P]
         lib.orc_linear_w8a8.argtypes = [P, P, P, P, c.c_int, c.c_int, c.c_int, P]
         lib.orc_linear_w8a8.restype = None
+        lib.orc_lora_bypass.argtypes = [P, P, P, c.c_int, c.c_int, c.c_int, c.c_int, P]
+        lib.orc_lora_bypass.restype = None
         lib.orc_num_threads.restype = c.c_int
         for f in ("orc_quantize_w4", "orc_quantize_w8", "orc_dequant", "orc_linear_wa16",
                   "orc_act_quant", "orc_group_partials", "orc_linear_w4a8"):
@@ -85,6 +87,20 @@ def linear_w8a8(x, q, s_bits, z_bits) -> np.ndarray:
     y = np.empty((M, N), np.float64)
     _l().orc_linear_w8a8(_p(x), _p(q), _p(s_bits), _p(z_bits), M, N, K, _p(y))
     return y
+
+
+def lora_bypass(y, x, lora_A, lora_B) -> np.ndarray:
+    """y + LoRA_A (LoRA_B x): y fp64 [M,N] (e.g. a linear's output), x [M,K], LoRA_A [N,r], LoRA_B [r,K]."""
+    x = _c(x, np.float32)
+    A = _c(lora_A, np.float32)
+    Bm = _c(lora_B, np.float32)
+    M, K = x.shape
+    N, r = A.shape
+    assert Bm.shape == (r, K)
+    out = np.array(y, dtype=np.float64, order="C", copy=True)
+    assert out.shape == (M, N)
+    _l().orc_lora_bypass(_p(x), _p(A), _p(Bm), M, N, K, r, _p(out))
+    return out
 
 
 def num_threads() -> int:
