@@ -593,12 +593,60 @@ def _sec_decode_w8a16(ctx):
     return {"decode_w8a16_qwen2_1p5b": e}
 
 
+def _sec_decode_lora(ctx):
+    """W4A16 decode with a rank-8 LoRA bypass on every linear (Section 5.5), Qwen2-1.5B stack, one token:
+    one launch per linear (the GEMV's CTAs compute LoRA_B x between them and add LoRA_A (LoRA_B x) where
+    they store).  Timed
+    beside the same seven launches per layer without the bypass (the batched q+k+v / gate+up form of
+    the headline has no LoRA entry)."""
+    import torch
+
+    from paper_2506_10443_b200 import binding as B
+    from paper_2506_10443_b200 import inputs
+
+    stack, r = ctx["stack"](), 8
+    rng = np.random.default_rng(8)
+    ws_bytes = B.workspace_size_lora(1, r)
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")   # one workspace: the calls are on one stream
+    B.lora_workspace_init(ws, ws_bytes)
+    calls, extra = [], 0
+    for li in range(stack.n_layers):
+        for t in stack.linears:
+            A = torch.from_numpy((rng.standard_normal((t.N, r)) * 0.05).astype(np.float16)).cuda()
+            Bm = torch.from_numpy((rng.standard_normal((r, t.K)) * 0.05).astype(np.float16)).cuda()
+            calls.append((stack.x_view(li, t.name), stack.layers[li].packed[t.name], A, Bm, stack.y_view(li, t.name), t.N, t.K, ws))
+            extra += 2 * r * (t.N + t.K)
+
+    def run_lora(stream=None):
+        for x, pk, A, Bm, y, N, K, ws in calls:
+            B.linear_w4a16_lora(x, pk, A, Bm, y, 1, N, K, GROUP, r, ws, ws_bytes, B.F16, B.F16, stream)
+
+    def run_plain(stream=None):
+        for x, pk, A, Bm, y, N, K, ws in calls:
+            B.linear_w4a16_ex(x, pk, y, 1, N, K, GROUP, B.F16, B.F16, stream)
+
+    g = _graph_of(run_lora)
+    ms = _time_steps(g.replay, 100, 10)
+    del g
+    g = _graph_of(run_plain)
+    ms0 = _time_steps(g.replay, 100, 10)
+    del g
+    assert B.read_status() == 0
+    e = _hbm_entry("gemv_w4a16_kernel", stack.algorithmic_bytes_w4a16 + extra, ms, ctx["hbm"],
+                   launches_per_step=len(calls), tokens_per_s=1.0 / (ms * 1e-3), rank=r,
+                   ms_per_step_without_bypass=ms0, launches_without_bypass=len(calls),
+                   lora_bytes_fraction=extra / stack.algorithmic_bytes_w4a16)
+    e["metric"] = "decode W4 GEMV + LoRA GB/s"
+    return {"decode_lora_r8_qwen2_1p5b": e}
+
+
 SECONDARY = {   # name -> function; also runnable alone: python bench.py --secondary-only NAME
     "decode_one_launch": _sec_decode_one_launch,
     "single_gemv": _sec_single_gemv,
     "prefill_1p5b": _sec_prefill_1p5b,
     "prefill_w8a8": _sec_prefill_w8a8,
     "decode_w8a16": _sec_decode_w8a16,
+    "decode_lora": _sec_decode_lora,
     "qwen2_7b": _sec_qwen2_7b,
     "lm_head": _sec_lm_head,
 }

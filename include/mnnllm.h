@@ -125,6 +125,33 @@ typedef struct {
 } mnnllm_w4a16_problem;
 int mnnllm_linear_w4a16_batch(const mnnllm_w4a16_problem* problems, int count, int M, void* stream);
 
+/* W4A16 linear with a LoRA bypass (Section 5.5, Table 3):
+ *   y[m, n] = (W4A16 linear of x)[m, n] + sum_j lora_A[n, j] * t[m, j],   t[m, j] = sum_k lora_B[j, k] * x[m, k]
+ * i.e. A' = W A + LoRA_A (LoRA_B A) in the order the paper chooses: the rank-r product first, so that
+ * the bypass costs 2 r (N + K) operations and r (N + K) fp16 values per token instead of an N x K
+ * matrix.  lora_A device fp16 [N, rank] (row n contiguous), lora_B device fp16 [rank, K] (16-byte
+ * aligned), 1 <= rank <= MNNLLM_LORA_MAX_RANK; the other arguments as for mnnllm_linear_w4a16_ex.
+ * workspace: device, 16-byte aligned, at least mnnllm_workspace_size_lora(M, rank) bytes (0 for
+ * invalid arguments), owned by the caller and cleared ONCE with mnnllm_lora_workspace_init before
+ * its first use; calls on one stream may share it (it is free for reuse when the stream has passed
+ * the call), calls that can overlap on the GPU may not.  It holds an epoch, a counter and the entries
+ * of t as {fp32 value, epoch tag} words.  ONE launch on `stream`: the GEMV's own CTAs compute the
+ * entries of t between them once the activations are complete (while their weights are already
+ * streaming in) and publish each as one tagged word; every CTA waits (bounded) for the words of this
+ * launch before it stores its first outputs, to which it adds the second product; y is written
+ * once, both products accumulate in fp32.  A
+ * separate launch for t would put another dependent stage in front of every linear, which costs
+ * more than the whole bypass.
+ * Errors: as mnnllm_linear_w4a16_ex, plus INVALID_ARG (null LoRA pointer, rank out of range),
+ * WORKSPACE (null or too small); a wait that ran out shows as MNNLLM_ERR_TIMEOUT (detail 0x700 |
+ * problem) in mnnllm_read_status. */
+#define MNNLLM_LORA_MAX_RANK 64
+size_t mnnllm_workspace_size_lora(int M, int rank);
+int mnnllm_lora_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
+int mnnllm_linear_w4a16_lora(const void* x, const void* packed, const void* lora_A, const void* lora_B, void* y,
+                             int M, int N, int K, int group, int rank, int x_dtype, int y_dtype, void* workspace,
+                             size_t workspace_bytes, void* stream);
+
 /* ------------------------------------------------------------------------------------------------
  * A whole decoder stack of W4A16 linears in ONE launch (decode, M <= 8 tokens).
  *

@@ -76,6 +76,9 @@ _sig("mnnllm_stack_workspace_size", _c.c_size_t, [_P])
 _sig("mnnllm_stack_workspace_init", _c.c_int, [_P, _c.c_size_t, _P])
 _sig("mnnllm_linear_w4a16_stack", _c.c_int, [_P, _P, _P, _c.c_size_t, _P])
 _sig("mnnllm_linear_w8a16", _c.c_int, [_P, _P, _P, _c.c_int, _c.c_int, _c.c_int, _c.c_int, _P])
+_sig("mnnllm_workspace_size_lora", _c.c_size_t, [_c.c_int, _c.c_int])
+_sig("mnnllm_lora_workspace_init", _c.c_int, [_P, _c.c_size_t, _P])
+_sig("mnnllm_linear_w4a16_lora", _c.c_int, [_P, _P, _P, _P, _P] + [_c.c_int] * 7 + [_P, _c.c_size_t, _P])
 _sig("mnnllm_workspace_size_w8a8", _c.c_size_t, [_c.c_int, _c.c_int])
 _sig("mnnllm_linear_w8a8", _c.c_int, [_P, _P, _P, _c.c_int, _c.c_int, _c.c_int, _c.c_int, _c.c_int, _P, _c.c_size_t, _P])
 _sig("mnnllm_workspace_size_w4a8", _c.c_size_t, [_c.c_int, _c.c_int, _c.c_int, _c.c_int])
@@ -100,7 +103,7 @@ EXPORTS = [
     "mnnllm_status_string", "mnnllm_packed_size_w4", "mnnllm_pack_w4", "mnnllm_unpack_w4", "mnnllm_packed_info",
     "mnnllm_packed_size_w8", "mnnllm_pack_w8", "mnnllm_unpack_w8", "mnnllm_linear_w4a16", "mnnllm_linear_w4a16_ex",
     "mnnllm_linear_w4a16_batch", "mnnllm_stack_plan_size", "mnnllm_stack_plan_w4a16", "mnnllm_stack_workspace_size",
-    "mnnllm_stack_workspace_init", "mnnllm_linear_w4a16_stack", "mnnllm_linear_w8a16", "mnnllm_workspace_size_w8a8", "mnnllm_linear_w8a8", "mnnllm_workspace_size_w4a8", "mnnllm_workspace_min_w4a8", "mnnllm_linear_w4a8", "mnnllm_linear_w4a8_batch", "mnnllm_linear_w4a8_static",
+    "mnnllm_stack_workspace_init", "mnnllm_linear_w4a16_stack", "mnnllm_linear_w8a16", "mnnllm_workspace_size_lora", "mnnllm_lora_workspace_init", "mnnllm_linear_w4a16_lora", "mnnllm_workspace_size_w8a8", "mnnllm_linear_w8a8", "mnnllm_workspace_size_w4a8", "mnnllm_workspace_min_w4a8", "mnnllm_linear_w4a8", "mnnllm_linear_w4a8_batch", "mnnllm_linear_w4a8_static",
     "mnnllm_quantize_activations", "mnnllm_debug_w4a8_partials", "mnnllm_debug_set_w4a8_small_max", "mnnllm_debug_set_w4a8_limb", "mnnllm_debug_wait_timeout", "mnnllm_bench_mma_i8", "mnnllm_read_status", "mnnllm_device_supported",
 ]
 
@@ -270,6 +273,23 @@ def linear_w4a8(x, packed, y, M, N, K, group, workspace, workspace_bytes, x_dtyp
                 stream=None) -> None:
     _check(lib.mnnllm_linear_w4a8(_ptr(x), _ptr(packed), _ptr(y), M, N, K, group, x_dtype, y_dtype, _ptr(workspace),
                                   workspace_bytes, _stream(stream)), "linear_w4a8")
+
+
+def workspace_size_lora(M: int, rank: int) -> int:
+    return int(lib.mnnllm_workspace_size_lora(M, rank))
+
+
+def lora_workspace_init(workspace, workspace_bytes, stream=None) -> None:
+    """Clears the counters of a LoRA workspace: once, before its first use."""
+    _check(lib.mnnllm_lora_workspace_init(_ptr(workspace), workspace_bytes, _stream(stream)), "lora_workspace_init")
+
+
+def linear_w4a16_lora(x, packed, lora_A, lora_B, y, M, N, K, group, rank, workspace, workspace_bytes, x_dtype=F16,
+                      y_dtype=F16, stream=None) -> None:
+    """W4A16 linear plus the LoRA bypass ``lora_A (lora_B x)``; lora_A fp16 [N, rank], lora_B fp16 [rank, K]."""
+    _check(lib.mnnllm_linear_w4a16_lora(_ptr(x), _ptr(packed), _ptr(lora_A), _ptr(lora_B), _ptr(y), M, N, K, group, rank,
+                                        x_dtype, y_dtype, _ptr(workspace), workspace_bytes, _stream(stream)),
+           "linear_w4a16_lora")
 
 
 def workspace_size_w8a8(M: int, K: int) -> int:

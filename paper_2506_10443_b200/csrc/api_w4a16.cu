@@ -182,7 +182,16 @@ int check_problem(const mnnllm_w4a16_problem& q, int M) {
     return MNNLLM_OK;
 }
 
-int run_batch(const mnnllm_w4a16_problem* problems, int count, int M, int x_dtype, cudaStream_t stream) {
+struct LoraArgs {   // bypass of one problem of a batch (r == 0: none)
+    const __half* A;     // [N, r]
+    const __half* B;     // [r, K]
+    float* t;            // [M, r] scratch
+    unsigned int* sync;  // two counters, zero between launches
+    int r;
+};
+
+int run_batch(const mnnllm_w4a16_problem* problems, int count, int M, int x_dtype, cudaStream_t stream,
+              const LoraArgs* lora = nullptr) {
     if (!problems || count < 1 || count > MNNLLM_MAX_BATCH) return MNNLLM_ERR_INVALID_ARG;
     const int group = problems[0].group;
     for (int i = 0; i < count; ++i) {
@@ -226,6 +235,13 @@ int run_batch(const mnnllm_w4a16_problem* problems, int count, int M, int x_dtyp
             P.y_dtype = q.y_dtype;
             P.x_dtype = x_dtype;
             P.row_block_bytes = g.row_block_bytes;
+            if (lora && lora[i].r > 0) {
+                P.lora_A = lora[i].A;
+                P.lora_B = lora[i].B;
+                P.lora_t = lora[i].t;   // every pass of eight tokens reuses the scratch from its start
+                P.lora_sync = lora[i].sync;
+                P.lora_r = lora[i].r;
+            }
             clusters += ncl[i];
         }
         if (gemv_w4a16_launch(L, group, MP, clusters, plan.CS, status, stream) != cudaSuccess) {
@@ -268,6 +284,40 @@ int mnnllm_debug_wait_timeout(int max_polls, void* stream) {
 
 int mnnllm_linear_w4a16_batch(const mnnllm_w4a16_problem* problems, int count, int M, void* stream) {
     return run_batch(problems, count, M, MNNLLM_F16, (cudaStream_t)stream);
+}
+
+size_t mnnllm_workspace_size_lora(int M, int rank) {
+    if (M < 1 || rank < 1 || rank > MNNLLM_LORA_MAX_RANK) return 0;
+    return 256 + 8 * (size_t)rank * 8;   // epoch and counter | tagged t of one pass of at most eight tokens
+}
+
+int mnnllm_lora_workspace_init(void* workspace, size_t workspace_bytes, void* stream) {
+    if (!workspace || workspace_bytes < 256) return MNNLLM_ERR_INVALID_ARG;
+    if (cudaMemsetAsync(workspace, 0, workspace_bytes, (cudaStream_t)stream) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return MNNLLM_ERR_CUDA;
+    }
+    return MNNLLM_OK;
+}
+
+int mnnllm_linear_w4a16_lora(const void* x, const void* packed, const void* lora_A, const void* lora_B, void* y, int M,
+                             int N, int K, int group, int rank, int x_dtype, int y_dtype, void* workspace,
+                             size_t workspace_bytes, void* stream) {
+    if (!lora_A || !lora_B || rank < 1 || rank > MNNLLM_LORA_MAX_RANK) return MNNLLM_ERR_INVALID_ARG;
+    if (x_dtype != MNNLLM_F16 && x_dtype != MNNLLM_BF16) return MNNLLM_ERR_UNSUPPORTED;
+    mnnllm_w4a16_problem q;
+    q.x = x; q.packed = packed; q.y = y; q.N = N; q.K = K; q.group = group; q.y_dtype = y_dtype;
+    const int st = check_problem(q, M);
+    if (st != MNNLLM_OK) return st;
+    if (((uintptr_t)lora_B & 15) || ((uintptr_t)lora_A & 1)) return MNNLLM_ERR_ALIGNMENT;
+    if (!workspace || workspace_bytes < mnnllm_workspace_size_lora(M, rank)) return MNNLLM_ERR_WORKSPACE;
+    if ((uintptr_t)workspace & 15) return MNNLLM_ERR_ALIGNMENT;
+    LoraArgs l;
+    l.A = (const __half*)lora_A; l.B = (const __half*)lora_B;
+    l.sync = (unsigned int*)workspace;
+    l.t = (float*)((uint8_t*)workspace + 256);
+    l.r = rank;
+    return run_batch(&q, 1, M, x_dtype, (cudaStream_t)stream, &l);
 }
 
 int mnnllm_linear_w8a16(const void* x, const void* packed, void* y, int M, int N, int K, int y_dtype, void* stream) {

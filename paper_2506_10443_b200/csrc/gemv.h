@@ -24,6 +24,15 @@ struct GemvProblem {
     int x_dtype;            // MNNLLM_F16, or MNNLLM_BF16 (converted to fp16 as the fragments are built)
     unsigned long long row_block_bytes;
     unsigned long long table_offset;  // W8: per-row (scale, zero) table, from the buffer start
+    // LoRA bypass (W4 kernel, instantiations with LORA; lora_r == 0: none):
+    // y[m, n] += sum_j lora_A[n, j] * t[m, j], t[m, j] = sum_k lora_B[j, k] x[m, k].  The launch's own CTAs
+    // compute t into lora_t as 8-byte {value, tag} words, tag = lora_sync[0] + 1 (the epoch); lora_sync[1]
+    // counts the CTAs that are through, the last one moves the epoch on.
+    const __half* lora_A;   // [N, lora_r]
+    const __half* lora_B;   // [lora_r, K]
+    float* lora_t;          // [M, lora_r] x 8 bytes
+    unsigned int* lora_sync;
+    int lora_r;
 };
 
 struct GemvLaunch {

@@ -33,7 +33,99 @@ namespace {
 
 constexpr uint32_t kMaxPolls = 1u << 15;  // x 20 us per try: gives up after ~0.65 s
 
-template <int GROUP, int MP, bool XBF>   // XBF: activations are bf16 (converted to fp16 as the fragments are built)
+constexpr unsigned int kLoraMaxPolls = 1u << 20;   // ~1 s of L2 round trips
+constexpr int kLoraMaxEntries = 8 * MNNLLM_LORA_MAX_RANK;   // (token, j) pairs of a launch
+
+// Eight consecutive fp16 (or bf16) values as floats.
+__device__ __forceinline__ void widen8(const uint4& v, bool bf16, float (&f)[8]) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        if (bf16) {   // a bf16 is the upper half of the fp32 of the same value
+            f[2 * i] = __uint_as_float(w[i] << 16);
+            f[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+        } else {
+            const float2 p = __half22float2(*reinterpret_cast<const __half2*>(&w[i]));
+            f[2 * i] = p.x;
+            f[2 * i + 1] = p.y;
+        }
+    }
+}
+
+// LoRA bypass (Section 5.5): y += LoRA_A (LoRA_B x), the small product first.  The CTAs of the problem
+// compute t = x . LoRA_B^T between them: entry o = (token, j) falls to CTA o mod n_ctas, whose threads
+// split K.  An entry is published as one 8-byte word {value, tag}, tag = the workspace's epoch + 1:
+// a reader needs no flag and no fence, it sees a whole word of this launch or an older one.
+struct LoraCtx {
+    unsigned long long* t2;   // [M * r] tagged entries
+    unsigned int tag;
+};
+
+// before the activations are complete: bring this CTA's rows of LoRA_B (static data) into L2
+__device__ __forceinline__ void lora_prefetch(const GemvProblem& P, int M, int cta, int n_ctas) {
+    const int n_t = M * P.lora_r;
+    for (int o = cta; o < n_t; o += n_ctas) {
+        const char* row = reinterpret_cast<const char*>(P.lora_B + (size_t)(o % P.lora_r) * P.K);
+        for (int b = threadIdx.x * 128; b < P.K * 2; b += blockDim.x * 128)
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(row + b));
+    }
+}
+
+__device__ __forceinline__ void lora_produce(const GemvProblem& P, const LoraCtx& lc, int M, bool x_bf16, int cta,
+                                             int n_ctas, float* red) {
+    const int n_t = M * P.lora_r;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, n_warps = blockDim.x >> 5;
+    for (int o = cta; o < n_t; o += n_ctas) {
+        const int m = o / P.lora_r, j = o - m * P.lora_r;
+        const uint4* xr = reinterpret_cast<const uint4*>(reinterpret_cast<const uint16_t*>(P.x) + (size_t)m * P.K);
+        const uint4* br = reinterpret_cast<const uint4*>(P.lora_B + (size_t)j * P.K);
+        float acc = 0.f;
+        for (int v = threadIdx.x; v < P.K / 8; v += blockDim.x) {
+            float a[8], b[8];
+            widen8(xr[v], x_bf16, a);
+            widen8(__ldg(br + v), false, b);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) acc = fmaf(a[i], b[i], acc);
+        }
+#pragma unroll
+        for (int s = 16; s > 0; s >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, s);
+        __syncthreads();   // red free (the previous entry has been summed)
+        if (lane == 0) red[warp] = acc;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            float sum = 0.f;
+            for (int w = 0; w < n_warps; ++w) sum += red[w];   // fixed order: the same t whoever runs first
+            __stcg(lc.t2 + o, ((unsigned long long)lc.tag << 32) | (unsigned long long)__float_as_uint(sum));
+        }
+    }
+}
+
+// Before the first output is stored: every entry of t into shared memory, each waited for (bounded)
+// until it carries this launch's tag.  Returns false when a wait ran out.
+__device__ __forceinline__ bool lora_collect(const LoraCtx& lc, int n_t, float* ts) {
+    bool ok = true;
+    for (int o = threadIdx.x; o < n_t; o += blockDim.x) {
+        unsigned long long w = 0;
+        unsigned int polls = 0;
+        for (;;) {
+            w = *reinterpret_cast<volatile unsigned long long*>(lc.t2 + o);
+            if ((unsigned int)(w >> 32) == lc.tag) break;
+            if (++polls > kLoraMaxPolls) { ok = false; break; }
+        }
+        ts[o] = __uint_as_float((unsigned int)w);
+    }
+    return ok;
+}
+
+__device__ __forceinline__ float lora_term(const GemvProblem& P, const float* ts, int n, int tok) {
+    const __half* a = P.lora_A + (size_t)n * P.lora_r;
+    const float* t = ts + tok * P.lora_r;
+    float acc = 0.f;
+    for (int j = 0; j < P.lora_r; ++j) acc = fmaf(__half2float(__ldg(a + j)), t[j], acc);
+    return acc;
+}
+
+template <int GROUP, int MP, bool XBF, bool LORA>   // XBF: activations are bf16; LORA: outputs take the bypass term (converted to fp16 as the fragments are built)
 __global__ void __launch_bounds__(kGemvMaxWarps * 32, (MP <= 2 ? 2 : 1))
 gemv_w4a16_kernel(const __grid_constant__ GemvLaunch L, uint32_t* __restrict__ status) {
     using C = Cfg<GROUP, MP>;
@@ -127,8 +219,20 @@ gemv_w4a16_kernel(const __grid_constant__ GemvLaunch L, uint32_t* __restrict__ s
 
     pdl_launch_dependents();
     for (int s = 0; s < S; ++s) issue_next();
+    __shared__ float lora_ts[LORA ? kLoraMaxEntries : 1];
+    __shared__ float lora_red[LORA ? kGemvMaxWarps : 1];
+    const bool has_lora = LORA && P.lora_r > 0;
+    if (has_lora) lora_prefetch(P, L.M, cl * CS + rank, P.n_clusters * CS);
     // everything above touched only weights; the activations may come from the previous kernel
     pdl_wait();
+    LoraCtx lc = {nullptr, 0u};
+    if (has_lora) {
+        // the epoch is stable here: the launch that last used the workspace has completed
+        lc.t2 = reinterpret_cast<unsigned long long*>(P.lora_t);
+        lc.tag = __ldcg(P.lora_sync) + 1u;
+        lora_produce(P, lc, L.M, XBF, cl * CS + rank, P.n_clusters * CS, lora_red);
+    }
+    bool lora_ready = !has_lora;
 
     const int tokB = r % MP, gsB = r / MP;  // B-operand role of this lane: column r of the MMA
     constexpr bool x_bf16 = XBF;
@@ -276,6 +380,10 @@ gemv_w4a16_kernel(const __grid_constant__ GemvLaunch L, uint32_t* __restrict__ s
             }
 
         // ---- end of round: sum over the warps (k-chunks) of this CTA, then over the cluster ----
+        if (LORA && !lora_ready) {
+            if (!lora_collect(lc, L.M * P.lora_r, lora_ts)) atomicOr(status, 0x700u | (unsigned)pi);
+            lora_ready = true;
+        }
         __syncthreads();
         const int n_out = per_round * MP * 16;
         float* red_rd = red + (rd & 1) * SR * C::PART_FLOATS;
@@ -288,7 +396,8 @@ gemv_w4a16_kernel(const __grid_constant__ GemvLaunch L, uint32_t* __restrict__ s
                     acc += part_all[((s_r * L.WC + w) * 2 + (rd & 1)) * C::PART_FLOATS + (it * MP + tok) * 16 + row];
             if (CS == 1) {
                 const int n = rb * 16 + row;
-                if (rb < rb_end && n < P.N && tok < L.M) store_out(P.y, P.y_dtype, (size_t)tok * P.N + n, acc);
+                if (rb < rb_end && n < P.N && tok < L.M)
+                    store_out(P.y, P.y_dtype, (size_t)tok * P.N + n, LORA ? acc + lora_term(P, lora_ts, n, tok) : acc);
             } else {
                 red_rd[o] = acc;
             }
@@ -302,9 +411,18 @@ gemv_w4a16_kernel(const __grid_constant__ GemvLaunch L, uint32_t* __restrict__ s
                 if (rb < rb_end && n < P.N && tok < L.M) {
                     float acc = 0.f;
                     for (int cr = 0; cr < CS; ++cr) acc += ld_dsmem_f32(red_rd + o, (uint32_t)cr);
-                    store_out(P.y, P.y_dtype, (size_t)tok * P.N + n, acc);
+                    store_out(P.y, P.y_dtype, (size_t)tok * P.N + n, LORA ? acc + lora_term(P, lora_ts, n, tok) : acc);
                 }
             }
+        }
+    }
+    if (has_lora) {
+        // this CTA has read t for the last time; the last CTA of the problem moves the epoch on (the
+        // next launch that uses the workspace reads it only after this grid has completed)
+        __syncthreads();
+        if (threadIdx.x == 0 && atomicAdd(P.lora_sync + 1, 1u) == (unsigned int)(P.n_clusters * CS) - 1u) {
+            P.lora_sync[0] = lc.tag;
+            P.lora_sync[1] = 0u;
         }
     }
     if (dead)   // copies issued before the give-up may still be in flight into this CTA's shared memory
@@ -320,7 +438,7 @@ size_t smem_bytes(int W, int SR, int S) {
 }
 
 // Raises the kernel's dynamic shared memory limit when a launch needs more than any before it.
-template <int GROUP, int MP, bool XBF>
+template <int GROUP, int MP, bool XBF, bool LORA>
 cudaError_t ensure_smem(size_t smem) {
     struct State { size_t configured; bool carveout_set; };
     static PerDevice<State> state;   // per instantiation and device
@@ -328,14 +446,14 @@ cudaError_t ensure_smem(size_t smem) {
         if (!st.carveout_set) {
             // every launch of the library asks for the same (largest) shared-memory carve-out, so that
             // an SM does not have to re-partition its L1 between consecutive dependent launches
-            cudaError_t e = cudaFuncSetAttribute(gemv_w4a16_kernel<GROUP, MP, XBF>,
+            cudaError_t e = cudaFuncSetAttribute(gemv_w4a16_kernel<GROUP, MP, XBF, LORA>,
                                                  cudaFuncAttributePreferredSharedMemoryCarveout,
                                                  (int)cudaSharedmemCarveoutMaxShared);
             if (e != cudaSuccess) return e;
             st.carveout_set = true;
         }
         if (smem > st.configured) {
-            cudaError_t e = cudaFuncSetAttribute(gemv_w4a16_kernel<GROUP, MP, XBF>,
+            cudaError_t e = cudaFuncSetAttribute(gemv_w4a16_kernel<GROUP, MP, XBF, LORA>,
                                                  cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
             if (e != cudaSuccess) return e;
             st.configured = smem;
@@ -344,12 +462,12 @@ cudaError_t ensure_smem(size_t smem) {
     });
 }
 
-template <int GROUP, int MP, bool XBF>
+template <int GROUP, int MP, bool XBF, bool LORA>
 cudaError_t launch_one(const GemvLaunch& L, int n_clusters, int CS, uint32_t* status, cudaStream_t stream) {
     const int W = L.WC * L.SR;
     const size_t smem = smem_bytes<GROUP, MP>(W, L.SR, L.stages);
-    auto kern = gemv_w4a16_kernel<GROUP, MP, XBF>;
-    if (cudaError_t e = ensure_smem<GROUP, MP, XBF>(smem); e != cudaSuccess) return e;
+    auto kern = gemv_w4a16_kernel<GROUP, MP, XBF, LORA>;
+    if (cudaError_t e = ensure_smem<GROUP, MP, XBF, LORA>(smem); e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(n_clusters * CS));
     cfg.blockDim = dim3((unsigned)(W * 32));
@@ -367,12 +485,24 @@ cudaError_t launch_one(const GemvLaunch& L, int n_clusters, int CS, uint32_t* st
     return cudaLaunchKernelEx(&cfg, kern, L, status);
 }
 
-template <int GROUP, int MP, bool XBF = false>
+// the instantiation by activation type and bypass (a launch has the bypass when one of its problems has)
+template <int GROUP, int MP>
+cudaError_t dispatch(const GemvLaunch& L, int n_clusters, int CS, uint32_t* status, cudaStream_t stream) {
+    bool lora = false;
+    for (int i = 0; i < L.count; ++i) lora |= L.prob[i].lora_r > 0;
+    const bool xbf = L.prob[0].x_dtype == MNNLLM_BF16;
+    if (lora) return xbf ? launch_one<GROUP, MP, true, true>(L, n_clusters, CS, status, stream)
+                         : launch_one<GROUP, MP, false, true>(L, n_clusters, CS, status, stream);
+    return xbf ? launch_one<GROUP, MP, true, false>(L, n_clusters, CS, status, stream)
+               : launch_one<GROUP, MP, false, false>(L, n_clusters, CS, status, stream);
+}
+
+template <int GROUP, int MP, bool XBF = false, bool LORA = false>
 int occupancy_of(int W, int SR, int S) {
     int n = 0;
     const size_t smem = smem_bytes<GROUP, MP>(W, SR, S);
-    auto kern = gemv_w4a16_kernel<GROUP, MP, XBF>;
-    if (ensure_smem<GROUP, MP, XBF>(smem) != cudaSuccess) return 0;
+    auto kern = gemv_w4a16_kernel<GROUP, MP, XBF, LORA>;
+    if (ensure_smem<GROUP, MP, XBF, LORA>(smem) != cudaSuccess) return 0;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kern, W * 32, smem) != cudaSuccess) return 0;
     return n;
 }
@@ -400,8 +530,7 @@ cudaError_t gemv_w4a16_launch(const GemvLaunch& L, int group, int MP, int n_clus
                               cudaStream_t stream) {
 #define MNN_CASE(G, P)                                                                                   \
     if (group == G && MP == P)                                                                          \
-        return L.prob[0].x_dtype == MNNLLM_BF16 ? launch_one<G, P, true>(L, n_clusters, CS, status, stream) \
-                                                : launch_one<G, P, false>(L, n_clusters, CS, status, stream);
+        return dispatch<G, P>(L, n_clusters, CS, status, stream);
     MNN_CASE(64, 1) MNN_CASE(64, 2) MNN_CASE(64, 4) MNN_CASE(64, 8)
     MNN_CASE(128, 1) MNN_CASE(128, 2) MNN_CASE(128, 4) MNN_CASE(128, 8)
 #undef MNN_CASE
