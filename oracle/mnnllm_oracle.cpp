@@ -24,6 +24,10 @@
 //   orc_lora_bypass        equality with the other association (LoRA_A LoRA_B) x in exact rationals
 //                          on small integers; rank-1 closed form; Table 3's operation and memory
 //                          counts for both orders (tests/golden/table3_lora.txt).
+//   orc_f32_to_e4m3 / back the 256 bit patterns written out from the format's definition in the test,
+//                          round trip, ties to even, saturation at 448.
+//   orc_attention_decode   equal keys -> mean of the values; one key far ahead -> its value; softmax
+//                          shift invariance; Python brute force of a tiny case; group-query mapping.
 //   fp16 conversions       exhaustive round trip over all 65536 bit patterns and comparison with
 //                          numpy's float16 on random and boundary values.
 //
@@ -300,6 +304,78 @@ void orc_lora_bypass(const float* x, const float* A, const float* B, int M, int 
             y[(size_t)m * N + n] += acc;
         }
     delete[] t;
+}
+
+// ---- fp8 E4M3 (1 sign, 4 exponent bits with bias 7, 3 fraction bits; no infinities, S.1111.111 is
+// NaN, largest finite value 448; subnormals 2^-9 .. 7 * 2^-9) -------------------------------------
+float orc_e4m3_to_f32(uint8_t b) {
+    const int sign = b >> 7, e = (b >> 3) & 15, f = b & 7;
+    double v;
+    if (e == 15 && f == 7) return std::nanf("");
+    if (e == 0) v = std::ldexp((double)f, -9);
+    else v = std::ldexp(1.0 + (double)f / 8.0, e - 7);
+    return (float)(sign ? -v : v);
+}
+
+// Round to nearest, ties to the even code; magnitudes above 448 (and infinities) saturate at 448.
+uint8_t orc_f32_to_e4m3(float x) {
+    if (std::isnan(x)) return 0x7F;
+    const uint8_t sign = std::signbit(x) ? 0x80 : 0;
+    const double a = std::fabs((double)x);
+    if (a >= 448.0) return sign | 0x7E;
+    // the codes 0 .. 0x7E are increasing in value: find the two neighbours and take the nearer one
+    int lo = 0;
+    for (int c = 0; c <= 0x7E; ++c)
+        if ((double)orc_e4m3_to_f32((uint8_t)c) <= a) lo = c;
+    if (lo == 0x7E) return sign | 0x7E;
+    const double vlo = (double)orc_e4m3_to_f32((uint8_t)lo), vhi = (double)orc_e4m3_to_f32((uint8_t)(lo + 1));
+    int pick;
+    if (a - vlo < vhi - a) pick = lo;
+    else if (a - vlo > vhi - a) pick = lo + 1;
+    else pick = (lo & 1) ? lo + 1 : lo;   // tie: the code with an even fraction
+    return sign | (uint8_t)pick;
+}
+
+// Attention for one decoded token over a quantised KV cache (Section 4.2: keys int8, quantised per
+// key vector along head_dim with Eq. 1; values fp8; Section 5.4: softmax in full precision, the
+// query divided by sqrt(head_dim) before the product with the keys).
+//   q        [H, D]       query values (fp16 widened to fp32)
+//   k_codes  [Hk, S, D]   uint8 codes, k_scale / k_zero [Hk, S] fp16 bits: k_hat = s * (c - z)
+//   v        [Hk, S, D]   E4M3 bytes
+//   out      [H, D]       fp64;   query head h reads kv head h / (H / Hk)
+//   score[h, t] = sum_d (q[h, d] / sqrt(D)) * k_hat[t, d];  p = softmax_t(score);  out[h, :] = sum_t p[t] * v[t, :]
+void orc_attention_decode(const float* q, const uint8_t* k_codes, const uint16_t* k_scale,
+                          const uint16_t* k_zero, const uint8_t* v, int H, int Hk, int S, int D,
+                          double* out) {
+    const int rep = H / Hk;
+    const double inv = 1.0 / std::sqrt((double)D);
+#pragma omp parallel for schedule(static)
+    for (int h = 0; h < H; ++h) {
+        const int hk = h / rep;
+        double* score = new double[S];
+        double mx = -INFINITY;
+        for (int t = 0; t < S; ++t) {
+            const size_t row = (size_t)hk * S + t;
+            const double s = (double)orc_f16_to_f32(k_scale[row]), z = (double)orc_f16_to_f32(k_zero[row]);
+            double acc = 0.0;
+            for (int d = 0; d < D; ++d)
+                acc += ((double)q[(size_t)h * D + d] * inv) * (s * ((double)k_codes[row * D + d] - z));
+            score[t] = acc;
+            if (acc > mx) mx = acc;
+        }
+        double denom = 0.0;
+        for (int t = 0; t < S; ++t) {
+            score[t] = std::exp(score[t] - mx);
+            denom += score[t];
+        }
+        for (int d = 0; d < D; ++d) {
+            double acc = 0.0;
+            for (int t = 0; t < S; ++t)
+                acc += (score[t] / denom) * (double)orc_e4m3_to_f32(v[((size_t)hk * S + t) * D + d]);
+            out[(size_t)h * D + d] = acc;
+        }
+        delete[] score;
+    }
 }
 
 int orc_num_threads(void) {

@@ -20,7 +20,8 @@ _LIB = os.path.join(_HERE, "libmnnllm_oracle.so")
 
 __all__ = [
     "build", "num_threads", "f16_to_f32", "f32_to_f16", "quantize_w4", "quantize_w8", "dequant",
-    "linear_wa16", "act_quant", "group_partials", "linear_w4a8", "linear_w8a8", "lora_bypass",
+    "linear_wa16", "act_quant", "group_partials", "linear_w4a8", "linear_w8a8", "lora_bypass", "e4m3_to_f32", "f32_to_e4m3", "quantize_keys",
+    "quantize_values", "attention_decode",
 ]
 
 
@@ -60,6 +61,12 @@ def _l():
         lib.orc_linear_w8a8.restype = None
         lib.orc_lora_bypass.argtypes = [P, P, P, c.c_int, c.c_int, c.c_int, c.c_int, P]
         lib.orc_lora_bypass.restype = None
+        lib.orc_e4m3_to_f32.restype = c.c_float
+        lib.orc_e4m3_to_f32.argtypes = [c.c_uint8]
+        lib.orc_f32_to_e4m3.restype = c.c_uint8
+        lib.orc_f32_to_e4m3.argtypes = [c.c_float]
+        lib.orc_attention_decode.argtypes = [P, P, P, P, P, c.c_int, c.c_int, c.c_int, c.c_int, P]
+        lib.orc_attention_decode.restype = None
         lib.orc_num_threads.restype = c.c_int
         for f in ("orc_quantize_w4", "orc_quantize_w8", "orc_dequant", "orc_linear_wa16",
                   "orc_act_quant", "orc_group_partials", "orc_linear_w4a8"):
@@ -100,6 +107,49 @@ def lora_bypass(y, x, lora_A, lora_B) -> np.ndarray:
     out = np.array(y, dtype=np.float64, order="C", copy=True)
     assert out.shape == (M, N)
     _l().orc_lora_bypass(_p(x), _p(A), _p(Bm), M, N, K, r, _p(out))
+    return out
+
+
+def e4m3_to_f32(bits: int) -> float:
+    return float(_l().orc_e4m3_to_f32(int(bits)))
+
+
+def f32_to_e4m3(x: float) -> int:
+    return int(_l().orc_f32_to_e4m3(float(x)))
+
+
+def quantize_keys(k: np.ndarray) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
+    """Keys [Hk, S, D] -> int8 codes per key vector (Eq. 1 along head_dim, codes 0..255): codes uint8
+    [Hk, S, D], scale and zero fp16 bits [Hk, S]."""
+    k = _c(k, np.float32)
+    Hk, S, D = k.shape
+    q, s, z = quantize_w8(k.reshape(Hk * S, D))
+    return q.reshape(Hk, S, D), s.reshape(Hk, S), z.reshape(Hk, S)
+
+
+def quantize_values(v: np.ndarray) -> np.ndarray:
+    """Values [Hk, S, D] -> E4M3 bytes, element by element (round to nearest even, saturating at 448)."""
+    v = _c(v, np.float32)
+    lib = _l()
+    flat = v.reshape(-1)
+    out = np.empty(flat.shape, np.uint8)
+    for i, x in enumerate(flat):
+        out[i] = lib.orc_f32_to_e4m3(float(x))
+    return out.reshape(v.shape)
+
+
+def attention_decode(q, k_codes, k_scale, k_zero, v_bytes) -> np.ndarray:
+    """out[H, D] fp64 of one decoded token over the quantised cache (see orc_attention_decode)."""
+    q = _c(q, np.float32)
+    k_codes = _c(k_codes, np.uint8)
+    k_scale = _c(k_scale, np.uint16)
+    k_zero = _c(k_zero, np.uint16)
+    v_bytes = _c(v_bytes, np.uint8)
+    H, D = q.shape
+    Hk, S, D2 = k_codes.shape
+    assert D2 == D and v_bytes.shape == (Hk, S, D) and H % Hk == 0
+    out = np.empty((H, D), np.float64)
+    _l().orc_attention_decode(_p(q), _p(k_codes), _p(k_scale), _p(k_zero), _p(v_bytes), H, Hk, S, D, _p(out))
     return out
 
 
