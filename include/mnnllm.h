@@ -295,6 +295,34 @@ size_t mnnllm_workspace_size_w8a8(int M, int K);
 int mnnllm_linear_w8a8(const void* x, const void* packed, void* y, int M, int N, int K, int x_dtype, int y_dtype,
                        void* workspace, size_t workspace_bytes, void* stream);
 
+/* ------------------------------------------------------------------------------------------------
+ * Attention of one decoded token over a quantised KV cache (Section 4.2: keys are quantised to int8
+ * along head_dim when they are stored, one Eq. 1 scale and zero point per key vector; values are
+ * stored as fp8, entry by entry, so that nothing already in the cache changes when a token is added;
+ * Section 5.4: softmax in full precision, the query divided by sqrt(head_dim) before the product):
+ *   k_hat[t, :] = s[t] * (codes[t, :] - z[t]);  score[h, t] = (q[h, :] / sqrt(D)) . k_hat[t, :]
+ *   out[h, :] = sum_t softmax_t(score[h, .])[t] * v[t, :]         query head h reads kv head h / (H / Hk)
+ * Cache of one layer, device memory owned by the caller, head_dim = 128 only:
+ *   k_codes  uint8 [Hk, S_cap, 128]  (16-byte aligned)     k_meta  uint32 [Hk, S_cap]: fp16 scale | fp16 zero << 16
+ *   v        E4M3  [Hk, S_cap, 128]  (1 sign, 4 exponent bits with bias 7, 3 fraction bits, no infinities, max 448)
+ * mnnllm_kv_append quantises one new key and value per kv head (k_new, v_new: device fp16 [Hk, 128];
+ * round to nearest even; E4M3 saturates at +-448) and stores them at position pos < S_cap.
+ * mnnllm_attention_decode: q device fp16 [H, 128], out device fp16 or fp32 [H, 128], positions [0, S),
+ * 1 <= S <= S_cap, H a multiple of Hk with H / Hk <= 8, Hk <= 64.  workspace: device, 16-byte aligned,
+ * at least mnnllm_attention_workspace_size(H, Hk, S) bytes (0 for invalid arguments), cleared ONCE
+ * with mnnllm_attention_workspace_init before its first use (every call leaves it cleared); calls on
+ * one stream may share it.  One launch each; nothing is allocated or synchronised.  The sequence is
+ * split over the SMs; the last CTA of a kv head merges the parts in the order of the splits.
+ * Errors: INVALID_ARG (null pointer, size < 1, pos or S outside the cache), UNSUPPORTED (head_dim,
+ * head counts, dtype, device), ALIGNMENT, WORKSPACE, CUDA. */
+int mnnllm_kv_append(void* k_codes, void* k_meta, void* v, int Hk, int S_cap, int head_dim, int pos,
+                     const void* k_new, const void* v_new, void* stream);
+size_t mnnllm_attention_workspace_size(int H, int Hk, int S);
+int mnnllm_attention_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
+int mnnllm_attention_decode(const void* q, const void* k_codes, const void* k_meta, const void* v, void* out,
+                            int H, int Hk, int head_dim, int S, int S_cap, int out_dtype, void* workspace,
+                            size_t workspace_bytes, void* stream);
+
 /* The activation quantiser alone (first kernel of the W4A8 path), writing caller-owned outputs:
  * a_q int8 [M, K], a_scale fp32 [M], A int32 [M, G]. */
 int mnnllm_quantize_activations(const void* x, int x_dtype, int M, int K, int group, int8_t* a_q,

@@ -336,6 +336,12 @@ uint8_t orc_f32_to_e4m3(float x) {
     return sign | (uint8_t)pick;
 }
 
+// Values to E4M3, entry by entry (nothing in the cache depends on any other entry).
+void orc_quantize_values(const float* v, long long n, uint8_t* out) {
+#pragma omp parallel for schedule(static)
+    for (long long i = 0; i < n; ++i) out[i] = orc_f32_to_e4m3(v[i]);
+}
+
 // Attention for one decoded token over a quantised KV cache (Section 4.2: keys int8, quantised per
 // key vector along head_dim with Eq. 1; values fp8; Section 5.4: softmax in full precision, the
 // query divided by sqrt(head_dim) before the product with the keys).

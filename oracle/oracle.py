@@ -65,6 +65,8 @@ def _l():
         lib.orc_e4m3_to_f32.argtypes = [c.c_uint8]
         lib.orc_f32_to_e4m3.restype = c.c_uint8
         lib.orc_f32_to_e4m3.argtypes = [c.c_float]
+        lib.orc_quantize_values.argtypes = [P, c.c_longlong, P]
+        lib.orc_quantize_values.restype = None
         lib.orc_attention_decode.argtypes = [P, P, P, P, P, c.c_int, c.c_int, c.c_int, c.c_int, P]
         lib.orc_attention_decode.restype = None
         lib.orc_num_threads.restype = c.c_int
@@ -130,12 +132,9 @@ def quantize_keys(k: np.ndarray) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
 def quantize_values(v: np.ndarray) -> np.ndarray:
     """Values [Hk, S, D] -> E4M3 bytes, element by element (round to nearest even, saturating at 448)."""
     v = _c(v, np.float32)
-    lib = _l()
-    flat = v.reshape(-1)
-    out = np.empty(flat.shape, np.uint8)
-    for i, x in enumerate(flat):
-        out[i] = lib.orc_f32_to_e4m3(float(x))
-    return out.reshape(v.shape)
+    out = np.empty(v.shape, np.uint8)
+    _l().orc_quantize_values(_p(v), v.size, _p(out))
+    return out
 
 
 def attention_decode(q, k_codes, k_scale, k_zero, v_bytes) -> np.ndarray:

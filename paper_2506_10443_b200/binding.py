@@ -79,6 +79,10 @@ _sig("mnnllm_linear_w8a16", _c.c_int, [_P, _P, _P, _c.c_int, _c.c_int, _c.c_int,
 _sig("mnnllm_workspace_size_lora", _c.c_size_t, [_c.c_int, _c.c_int])
 _sig("mnnllm_lora_workspace_init", _c.c_int, [_P, _c.c_size_t, _P])
 _sig("mnnllm_linear_w4a16_lora", _c.c_int, [_P, _P, _P, _P, _P] + [_c.c_int] * 7 + [_P, _c.c_size_t, _P])
+_sig("mnnllm_kv_append", _c.c_int, [_P, _P, _P, _c.c_int, _c.c_int, _c.c_int, _c.c_int, _P, _P, _P])
+_sig("mnnllm_attention_workspace_size", _c.c_size_t, [_c.c_int, _c.c_int, _c.c_int])
+_sig("mnnllm_attention_workspace_init", _c.c_int, [_P, _c.c_size_t, _P])
+_sig("mnnllm_attention_decode", _c.c_int, [_P, _P, _P, _P, _P] + [_c.c_int] * 6 + [_P, _c.c_size_t, _P])
 _sig("mnnllm_workspace_size_w8a8", _c.c_size_t, [_c.c_int, _c.c_int])
 _sig("mnnllm_linear_w8a8", _c.c_int, [_P, _P, _P, _c.c_int, _c.c_int, _c.c_int, _c.c_int, _c.c_int, _P, _c.c_size_t, _P])
 _sig("mnnllm_workspace_size_w4a8", _c.c_size_t, [_c.c_int, _c.c_int, _c.c_int, _c.c_int])
@@ -103,7 +107,8 @@ EXPORTS = [
     "mnnllm_status_string", "mnnllm_packed_size_w4", "mnnllm_pack_w4", "mnnllm_unpack_w4", "mnnllm_packed_info",
     "mnnllm_packed_size_w8", "mnnllm_pack_w8", "mnnllm_unpack_w8", "mnnllm_linear_w4a16", "mnnllm_linear_w4a16_ex",
     "mnnllm_linear_w4a16_batch", "mnnllm_stack_plan_size", "mnnllm_stack_plan_w4a16", "mnnllm_stack_workspace_size",
-    "mnnllm_stack_workspace_init", "mnnllm_linear_w4a16_stack", "mnnllm_linear_w8a16", "mnnllm_workspace_size_lora", "mnnllm_lora_workspace_init", "mnnllm_linear_w4a16_lora", "mnnllm_workspace_size_w8a8", "mnnllm_linear_w8a8", "mnnllm_workspace_size_w4a8", "mnnllm_workspace_min_w4a8", "mnnllm_linear_w4a8", "mnnllm_linear_w4a8_batch", "mnnllm_linear_w4a8_static",
+    "mnnllm_stack_workspace_init", "mnnllm_linear_w4a16_stack", "mnnllm_linear_w8a16", "mnnllm_kv_append", "mnnllm_attention_workspace_size", "mnnllm_attention_workspace_init",
+    "mnnllm_attention_decode", "mnnllm_workspace_size_lora", "mnnllm_lora_workspace_init", "mnnllm_linear_w4a16_lora", "mnnllm_workspace_size_w8a8", "mnnllm_linear_w8a8", "mnnllm_workspace_size_w4a8", "mnnllm_workspace_min_w4a8", "mnnllm_linear_w4a8", "mnnllm_linear_w4a8_batch", "mnnllm_linear_w4a8_static",
     "mnnllm_quantize_activations", "mnnllm_debug_w4a8_partials", "mnnllm_debug_set_w4a8_small_max", "mnnllm_debug_set_w4a8_limb", "mnnllm_debug_wait_timeout", "mnnllm_bench_mma_i8", "mnnllm_read_status", "mnnllm_device_supported",
 ]
 
@@ -290,6 +295,27 @@ def linear_w4a16_lora(x, packed, lora_A, lora_B, y, M, N, K, group, rank, worksp
     _check(lib.mnnllm_linear_w4a16_lora(_ptr(x), _ptr(packed), _ptr(lora_A), _ptr(lora_B), _ptr(y), M, N, K, group, rank,
                                         x_dtype, y_dtype, _ptr(workspace), workspace_bytes, _stream(stream)),
            "linear_w4a16_lora")
+
+
+def kv_append(k_codes, k_meta, v, Hk, S_cap, pos, k_new, v_new, head_dim=128, stream=None) -> None:
+    """Quantises one new key (int8, Eq. 1 per key vector) and value (E4M3) per kv head into the cache at ``pos``."""
+    _check(lib.mnnllm_kv_append(_ptr(k_codes), _ptr(k_meta), _ptr(v), Hk, S_cap, head_dim, pos, _ptr(k_new), _ptr(v_new),
+                                _stream(stream)), "kv_append")
+
+
+def attention_workspace_size(H: int, Hk: int, S: int) -> int:
+    return int(lib.mnnllm_attention_workspace_size(H, Hk, S))
+
+
+def attention_workspace_init(workspace, workspace_bytes, stream=None) -> None:
+    _check(lib.mnnllm_attention_workspace_init(_ptr(workspace), workspace_bytes, _stream(stream)), "attention_workspace_init")
+
+
+def attention_decode(q, k_codes, k_meta, v, out, H, Hk, S, S_cap, workspace, workspace_bytes, out_dtype=F16, head_dim=128,
+                     stream=None) -> None:
+    """One decoded token's attention over the quantised cache: q fp16 [H, 128] -> out [H, 128]."""
+    _check(lib.mnnllm_attention_decode(_ptr(q), _ptr(k_codes), _ptr(k_meta), _ptr(v), _ptr(out), H, Hk, head_dim, S, S_cap,
+                                       out_dtype, _ptr(workspace), workspace_bytes, _stream(stream)), "attention_decode")
 
 
 def workspace_size_w8a8(M: int, K: int) -> int:

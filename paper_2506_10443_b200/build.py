@@ -25,6 +25,8 @@ SOURCES = [
     "act_quant.cu",
     "gemm_w4a8.cu",
     "gemm_w8a8.cu",
+    "attn_decode.cu",
+    "api_attn.cu",
     "api_w8a8.cu",
     "gemm_small_w4a8.cu",
     "gemm_limb_w4a8.cu",
