@@ -640,6 +640,47 @@ def _sec_decode_lora(ctx):
     return {"decode_lora_r8_qwen2_1p5b": e}
 
 
+def _sec_attention_decode(ctx):
+    """Decode attention over a quantised KV cache (int8 keys, E4M3 values; Section 4.2) with Qwen2-1.5B
+    heads (12 query, 2 kv, head_dim 128) and Qwen2-7B heads (28 / 4): 28 layers per step, each with its own
+    cache (every pass streams from DRAM), 4096 and 32768 tokens of context.  Bytes = codes + values +
+    4 bytes of scale/zero per key."""
+    import torch
+
+    from paper_2506_10443_b200 import binding as B
+
+    out = {}
+    for name, H, Hk, S in (("qwen2_1p5b_s4096", 12, 2, 4096), ("qwen2_1p5b_s32768", 12, 2, 32768),
+                           ("qwen2_7b_s32768", 28, 4, 32768)):
+        n_layers = 28
+        gen = torch.Generator(device="cuda").manual_seed(9)
+        kc = torch.randint(0, 256, (n_layers, Hk, S, 128), dtype=torch.uint8, device="cuda", generator=gen)
+        # values: random E4M3 bytes below the NaN pattern; keys: scale 2^-6 (fp16 0x2400), zero 128 (0x5800)
+        vb = torch.randint(0, 0x78, (n_layers, Hk, S, 128), dtype=torch.uint8, device="cuda", generator=gen)
+        meta = torch.full((n_layers, Hk, S), 0x58002400, dtype=torch.int32, device="cuda")
+        q = torch.randn((n_layers, H, 128), device="cuda", generator=gen).half()
+        o = torch.empty((n_layers, H, 128), dtype=torch.float16, device="cuda")
+        ws_bytes = B.attention_workspace_size(H, Hk, S)
+        ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+        B.attention_workspace_init(ws, ws_bytes)
+
+        def run(stream=None):
+            for l in range(n_layers):
+                B.attention_decode(q[l], kc[l], meta[l], vb[l], o[l], H, Hk, S, S, ws, ws_bytes, B.F16, stream=stream)
+
+        g = _graph_of(run)
+        assert B.read_status() == 0
+        ms = _time_steps(g.replay, 50, 5)
+        nbytes = n_layers * (Hk * S * (128 + 128 + 4) + 2 * 2 * H * 128)
+        e = _hbm_entry("attn_decode_kernel", nbytes, ms, ctx["hbm"], launches_per_step=n_layers, context_tokens=S,
+                       heads="%d query / %d kv" % (H, Hk))
+        e["metric"] = "decode attention (int8 K, fp8 V) GB/s"
+        out["attention_decode_" + name] = e
+        del g, kc, vb, meta
+        torch.cuda.empty_cache()
+    return out
+
+
 SECONDARY = {   # name -> function; also runnable alone: python bench.py --secondary-only NAME
     "decode_one_launch": _sec_decode_one_launch,
     "single_gemv": _sec_single_gemv,
@@ -647,6 +688,7 @@ SECONDARY = {   # name -> function; also runnable alone: python bench.py --secon
     "prefill_w8a8": _sec_prefill_w8a8,
     "decode_w8a16": _sec_decode_w8a16,
     "decode_lora": _sec_decode_lora,
+    "attention_decode": _sec_attention_decode,
     "qwen2_7b": _sec_qwen2_7b,
     "lm_head": _sec_lm_head,
 }

@@ -42,8 +42,8 @@ int mnnllm_kv_append(void* k_codes, void* k_meta, void* v, int Hk, int S_cap, in
 
 size_t mnnllm_attention_workspace_size(int H, int Hk, int S) {
     if (H < 1 || Hk < 1 || Hk > 64 || S < 1 || H % Hk != 0 || H / Hk > kAttnMaxRep) return 0;
-    // one part per 256-token chunk at most (the launch uses fewer when the GPU has fewer SMs to feed)
-    return kCounterBytes + (size_t)((S + kAttnChunk - 1) / kAttnChunk) * H * (kAttnHeadDim + 2) * 4;
+    // one part per 128 tokens at most (the launch uses fewer when the sequence is long)
+    return kCounterBytes + (size_t)((S + kAttnMinSplit - 1) / kAttnMinSplit) * H * (kAttnHeadDim + 2) * 4;
 }
 
 int mnnllm_attention_workspace_init(void* workspace, size_t workspace_bytes, void* stream) {

@@ -89,80 +89,129 @@ __global__ void __launch_bounds__(32) attn_append_kernel(AttnCache c, const __ha
 
 namespace {
 
-// an E4M3 byte as float: its bits placed in an fp16 give the value * 2^-8, exactly (subnormals too)
-__device__ __forceinline__ float e4m3_to_f32(uint32_t b) {
-    const uint16_t h = (uint16_t)(((b & 0x80u) << 8) | ((b & 0x7Fu) << 7));
-    return __half2float(__ushort_as_half(h)) * 256.f;
+// four E4M3 bytes of a word as floats TIMES 2^-8: a byte's bits placed in an fp16 give exactly that
+// (subnormals included); the factor 2^8 goes on once, where a CTA's part is written
+__device__ __forceinline__ void e4m3x4_to_f32_scaled(uint32_t w, float (&f)[4]) {
+    // bytes 0, 1 and 2, 3 as two half2: sign to bit 15, the other seven bits to bits 7..13
+    const uint32_t lo = __byte_perm(w, 0u, 0x1404), hi = __byte_perm(w, 0u, 0x3424);   // [0, b0, 0, b1], [0, b2, 0, b3]
+    const uint32_t hl = (lo & 0x80008000u) | ((lo & 0x7F007F00u) >> 1);
+    const uint32_t hh = (hi & 0x80008000u) | ((hi & 0x7F007F00u) >> 1);
+    const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&hl));
+    const float2 b = __half22float2(*reinterpret_cast<const __half2*>(&hh));
+    f[0] = a.x; f[1] = a.y; f[2] = b.x; f[3] = b.y;
 }
 
-struct Part {   // what a CTA leaves per query head: running maximum, sum of weights, weighted values
-    float m, l;
-};
-
-// grid (splits, Hk), 256 threads.  Tokens [t0, t1) of kv head hk in chunks of 256:
-//   1. thread t: scores of token t for the kv head's `rep` query heads (the key row is 8 x 16 bytes
-//      per thread, the scaled queries come from shared memory as broadcasts);
+// grid (splits, Hk), 256 threads = 8 warps.  Tokens [t0, t1) of kv head hk in chunks of up to 256:
+//   1. scores on the tensor cores: mma.sync m16n8k16 with the kv head's query heads as rows (fp16,
+//      unscaled: exact) and eight tokens as columns; the codes enter as the fp16 numbers 1024 + code
+//      (a byte permute), head_dim is walked in an order that lets a lane take its two 16-byte pieces
+//      of a key row as they are (the same order on the query side); the excess 1024 and the zero
+//      point come off with the row sum of the query, the scale and 1/sqrt(128) go on in fp32;
 //   2. warp h: the chunk's maximum for head h, the new running maximum and the factor that rescales
 //      what has been accumulated so far; then every score becomes its weight exp(score - max);
-//   3. thread (d, half): value entry d of the tokens of its half of the chunk, rep accumulators.
+//   3. weighted values: warp w takes tokens w, w + 8, ..., a lane four value entries of the row
+//      (one 128-byte row per load instruction), REP x 4 accumulators per thread.
 template <int REP>
 __global__ void __launch_bounds__(kThreads) attn_decode_kernel(AttnCache c, const __half* __restrict__ q, void* out,
                                                                int out_dtype, int S, int per_split, float* partials,
                                                                unsigned int* counters, uint32_t* status) {
-    __shared__ float qs[REP][kD];          // q / sqrt(128)
-    __shared__ float qsum[REP];            // sum_d of the scaled query (zero-point term)
-    __shared__ float sc[REP][kAttnChunk];  // scores, then weights
+    __shared__ float sc[REP][kAttnChunk];   // scores, then weights
+    __shared__ float qsum[REP];             // sum_d q[h, d]
     __shared__ float m_run[REP], l_run[REP], rescale[REP];
-    __shared__ float acc_half[REP][kD];    // second half's accumulators for the final sum
+    __shared__ float red[4][REP][kD];       // cross-warp sum of the accumulators
     __shared__ unsigned int last_flag;
+    __shared__ uint32_t meta_s[kAttnChunk];  // the chunk's (scale, zero) pairs
+    __shared__ __align__(8) uint64_t bar;   // the chunk's key and value rows have landed
+    extern __shared__ __align__(128) uint8_t dyn[];
+    uint8_t* kbuf = dyn;                            // [kAttnChunk][128] key codes
+    uint8_t* vbuf = dyn + kAttnChunk * kD;          // [kAttnChunk][128] values
 
     const int split = blockIdx.x, hk = blockIdx.y, n_splits = gridDim.x;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int g = lane >> 2, cq = lane & 3;
     const int t0 = split * per_split, t1 = min(S, t0 + per_split);
     ptx::pdl_launch_dependents();
     ptx::pdl_wait();   // q (and the newest cache row) come from kernels before
-    for (int i = tid; i < REP * kD; i += kThreads)
-        qs[i / kD][i % kD] = __half2float(q[(size_t)(hk * REP) * kD + i]) * 0.08838834764831845f;   // 1 / sqrt(128)
-    if (tid < REP) { m_run[tid] = -INFINITY; l_run[tid] = 0.f; }
-    __syncthreads();
-    if (warp < REP) {
-        float a = qs[warp][lane] + qs[warp][lane + 32] + qs[warp][lane + 64] + qs[warp][lane + 96];
+
+    // query fragments: k-step s covers head_dim entries 16 (cq + 4 (s >> 2)) + 4 (s & 3) + {0, 1 | 2, 3}
+    uint32_t qa0[8], qa2[8];
+    {
+        const __half* qr = q + (size_t)(hk * REP + (g < REP ? g : 0)) * kD;
+        float sum = 0.f;
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
-        if (lane == 0) qsum[warp] = a;
+        for (int s = 0; s < 8; ++s) {
+            const uint2 w = *reinterpret_cast<const uint2*>(qr + 16 * (cq + 4 * (s >> 2)) + 4 * (s & 3));
+            qa0[s] = g < REP ? w.x : 0u;
+            qa2[s] = g < REP ? w.y : 0u;
+            const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&w.x));
+            const float2 b = __half22float2(*reinterpret_cast<const __half2*>(&w.y));
+            sum += (a.x + a.y) + (b.x + b.y);
+        }
+        sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+        sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+        if (warp == 0 && cq == 0 && g < REP) qsum[g] = sum;
+    }
+    if (tid < REP) { m_run[tid] = -INFINITY; l_run[tid] = 0.f; }
+    if (tid == 0) {
+        ptx::mbar_init(&bar, 1);
+        ptx::fence_mbar_init();
     }
     __syncthreads();
+    uint32_t phase = 0;
+    bool dead = false;   // a bounded wait gave up
 
-    const int d = tid & (kD - 1), half = tid >> 7;
-    float acc[REP];
+    float acc[REP][4];
 #pragma unroll
-    for (int h = 0; h < REP; ++h) acc[h] = 0.f;
+    for (int h = 0; h < REP; ++h)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) acc[h][i] = 0.f;
 
     for (int c0 = t0; c0 < t1; c0 += kAttnChunk) {
         const int n = min(kAttnChunk, t1 - c0);
-        // ---- 1. scores
-        if (tid < n) {
-            const size_t row = (size_t)hk * c.S_cap + c0 + tid;
-            const uint4* kr = reinterpret_cast<const uint4*>(c.k_codes + row * kD);
-            const uint32_t meta = __ldg(c.k_meta + row);
-            const __half2 sz = *reinterpret_cast<const __half2*>(&meta);
-            const float s = __low2float(sz), z = __high2float(sz);
-            float dot[REP];
+        // the chunk's rows are contiguous in the cache: two bulk copies put all of a CTA's bytes in
+        // flight at once (with loads issued by the warps as they go, the kernel ran at a tenth of the
+        // memory rate: a handful of rows in flight per warp against a microsecond of latency)
+        if (tid == 0 && !dead) {
+            const size_t row0 = ((size_t)hk * c.S_cap + c0) * kD;
+            ptx::mbar_arrive_expect_tx(&bar, 2u * (uint32_t)n * kD);
+            ptx::bulk_g2s(kbuf, c.k_codes + row0, (uint32_t)n * kD, &bar);
+            ptx::bulk_g2s(vbuf, c.v + row0, (uint32_t)n * kD, &bar);
+        }
+        if (tid < n) meta_s[tid] = __ldg(c.k_meta + (size_t)hk * c.S_cap + c0 + tid);
+        if (!dead && !ptx::mbar_wait_bounded(&bar, phase, 1u << 22)) {
+            dead = true;
+            if (lane == 0) atomicOr(status, 0x800u);
+        }
+        phase ^= 1u;
+        dead = __syncthreads_or(dead);
+        if (dead) break;
+        // ---- 1. scores: token groups of eight, one group per warp and round
+        for (int g0 = warp * 8; g0 < n; g0 += 64) {
+            const int tok = g0 + g;   // this lane's B-operand column
+            uint4 u0 = make_uint4(0, 0, 0, 0), u1 = u0;
+            if (tok < n) {
+                const uint4* kr = reinterpret_cast<const uint4*>(kbuf + tok * kD);
+                u0 = kr[cq];
+                u1 = kr[cq + 4];
+            }
+            const uint32_t w[8] = {u0.x, u0.y, u0.z, u0.w, u1.x, u1.y, u1.z, u1.w};
+            float d[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-            for (int h = 0; h < REP; ++h) dot[h] = 0.f;
+            for (int s = 0; s < 8; ++s)
+                ptx::mma_m16n8k16_f16(d, qa0[s], 0u, qa2[s], 0u, __byte_perm(w[s], 0x64646464u, 0x4140),
+                                      __byte_perm(w[s], 0x64646464u, 0x4342));
+            // d[0], d[1]: query head g, tokens g0 + 2 cq and + 1
+            if (g < REP) {
 #pragma unroll
-            for (int v = 0; v < kD / 16; ++v) {
-                const uint4 w = __ldg(kr + v);
-                const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
-#pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    const float code = (float)((ww[j >> 2] >> (8 * (j & 3))) & 0xFFu);
-#pragma unroll
-                    for (int h = 0; h < REP; ++h) dot[h] = fmaf(qs[h][v * 16 + j], code, dot[h]);
+                for (int e = 0; e < 2; ++e) {
+                    const int t = g0 + 2 * cq + e;
+                    if (t < n) {
+                        const uint32_t meta = meta_s[t];
+                        const __half2 sz = *reinterpret_cast<const __half2*>(&meta);
+                        sc[g][t] = (__low2float(sz) * 0.08838834764831845f) * (d[e] - (1024.f + __high2float(sz)) * qsum[g]);
+                    }
                 }
             }
-#pragma unroll
-            for (int h = 0; h < REP; ++h) sc[h][tid] = s * (dot[h] - z * qsum[h]);
         }
         __syncthreads();
         // ---- 2. running maximum and weights
@@ -190,26 +239,52 @@ __global__ void __launch_bounds__(kThreads) attn_decode_kernel(AttnCache c, cons
         __syncthreads();
         // ---- 3. weighted values
 #pragma unroll
-        for (int h = 0; h < REP; ++h) acc[h] *= rescale[h];
-        const uint8_t* vr = c.v + ((size_t)hk * c.S_cap + c0) * kD + d;
-        for (int t = half; t < n; t += 2) {
-            const float val = e4m3_to_f32(__ldg(vr + (size_t)t * kD));
+        for (int h = 0; h < REP; ++h)
 #pragma unroll
-            for (int h = 0; h < REP; ++h) acc[h] = fmaf(sc[h][t], val, acc[h]);
+            for (int i = 0; i < 4; ++i) acc[h][i] *= rescale[h];
+        const uint32_t* vr = reinterpret_cast<const uint32_t*>(vbuf) + lane;
+#pragma unroll 4
+        for (int t = warp; t < n; t += 8) {
+            float val[4];
+            e4m3x4_to_f32_scaled(vr[t * (kD / 4)], val);
+#pragma unroll
+            for (int h = 0; h < REP; ++h) {
+                const float p = sc[h][t];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) acc[h][i] = fmaf(p, val[i], acc[h][i]);
+            }
         }
-        __syncthreads();   // sc and rescale are rewritten by the next chunk
+        __syncthreads();   // sc, rescale and the row buffers are rewritten by the next chunk
+    }
+    if (dead) {   // give copies in flight time to land before the CTA goes away; its part is not counted
+        for (int i = 0; i < 50; ++i) __nanosleep(1000);
+        return;
     }
 
-    // ---- this CTA's part: {m, l, acc[128]} per query head (the two halves of the threads summed)
-    if (half == 1)
+    // ---- the eight warps' accumulators summed in a fixed tree (4 + 4, 2 + 2, 1 + 1)
 #pragma unroll
-        for (int h = 0; h < REP; ++h) acc_half[h][d] = acc[h];
-    __syncthreads();
+    for (int stride = 4; stride >= 1; stride >>= 1) {
+        if (warp >= stride && warp < 2 * stride)
+#pragma unroll
+            for (int h = 0; h < REP; ++h)
+                *reinterpret_cast<float4*>(&red[warp - stride][h][lane * 4]) = make_float4(acc[h][0], acc[h][1], acc[h][2], acc[h][3]);
+        __syncthreads();
+        if (warp < stride)
+#pragma unroll
+            for (int h = 0; h < REP; ++h) {
+                const float4 o = *reinterpret_cast<const float4*>(&red[warp][h][lane * 4]);
+                acc[h][0] += o.x; acc[h][1] += o.y; acc[h][2] += o.z; acc[h][3] += o.w;
+            }
+        __syncthreads();
+    }
+    // ---- this CTA's part: {m, l, acc[128]} per query head
     constexpr int kPart = kD + 2;
     float* mine = partials + ((size_t)(hk * n_splits + split) * REP) * kPart;
-    if (half == 0)
+    if (warp == 0)
 #pragma unroll
-        for (int h = 0; h < REP; ++h) __stcg(mine + h * kPart + 2 + d, acc[h] + acc_half[h][d]);
+        for (int h = 0; h < REP; ++h)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) __stcg(mine + h * kPart + 2 + lane * 4 + i, acc[h][i] * 256.f);
     if (tid < REP) {
         __stcg(mine + tid * kPart, m_run[tid]);
         __stcg(mine + tid * kPart + 1, l_run[tid]);
@@ -224,20 +299,62 @@ __global__ void __launch_bounds__(kThreads) attn_decode_kernel(AttnCache c, cons
     __threadfence();
     if (tid == 0) counters[hk] = 0u;
     const float* parts = partials + ((size_t)hk * n_splits * REP) * kPart;
-    for (int o = tid; o < REP * kD; o += kThreads) {
-        const int h = o / kD, dd = o - h * kD;
-        float m = -INFINITY;
-        for (int s = 0; s < n_splits; ++s) m = fmaxf(m, __ldcg(parts + ((size_t)s * REP + h) * kPart));
-        float l = 0.f, a = 0.f;
-        for (int s = 0; s < n_splits; ++s) {
-            const float* ps = parts + ((size_t)s * REP + h) * kPart;
-            const float ms = __ldcg(ps);
-            const float w = ms == -INFINITY ? 0.f : expf(ms - m);   // a split without tokens carries nothing
-            l = fmaf(__ldcg(ps + 1), w, l);
-            a = fmaf(__ldcg(ps + 2 + dd), w, a);
+    // warp h: head h's {m, l} of every part in one pass of loads (n_splits <= 256: eight per lane), the
+    // overall maximum, every part's weight exp(m_s - m) (into sc) and the sum of the weighted l_s
+    if (warp < REP) {
+        float2 ml[kAttnChunk / 32];
+#pragma unroll
+        for (int i = 0; i < kAttnChunk / 32; ++i) {
+            const int s = lane + 32 * i;
+            ml[i] = s < n_splits ? __ldcg(reinterpret_cast<const float2*>(parts + ((size_t)s * REP + warp) * kPart))
+                                 : make_float2(-INFINITY, 0.f);
         }
-        const float r = a / l;
-        const size_t idx = (size_t)(hk * REP + h) * kD + dd;
+        float m = -INFINITY;
+#pragma unroll
+        for (int i = 0; i < kAttnChunk / 32; ++i) m = fmaxf(m, ml[i].x);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+        float l = 0.f;
+#pragma unroll
+        for (int i = 0; i < kAttnChunk / 32; ++i) {
+            const int s = lane + 32 * i;
+            const float w = ml[i].x == -INFINITY ? 0.f : expf(ml[i].x - m);   // a part without tokens carries nothing
+            if (s < n_splits) sc[warp][s] = w;
+            l = fmaf(ml[i].y, w, l);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
+        if (lane == 0) l_run[warp] = l;
+    }
+    __syncthreads();
+    // the weighted sum of the parts' accumulators: warp w takes parts w, w + 8, ... for all heads (a lane
+    // four entries: one 512-byte row of a part per pair of loads, REP rows per part in flight together);
+    // then the eight warps' sums are added in a fixed order through the row buffers, which are free now
+    float4 a[REP];
+#pragma unroll
+    for (int h = 0; h < REP; ++h) a[h] = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 2
+    for (int s = warp; s < n_splits; s += 8) {
+#pragma unroll
+        for (int h = 0; h < REP; ++h) {
+            const float* ps = parts + ((size_t)s * REP + h) * kPart + 2 + lane * 4;   // 8 bytes into a part
+            const float w = sc[h][s];
+            const float2 lo = __ldcg(reinterpret_cast<const float2*>(ps)), hi = __ldcg(reinterpret_cast<const float2*>(ps + 2));
+            a[h].x = fmaf(lo.x, w, a[h].x); a[h].y = fmaf(lo.y, w, a[h].y);
+            a[h].z = fmaf(hi.x, w, a[h].z); a[h].w = fmaf(hi.y, w, a[h].w);
+        }
+    }
+    float* mrg = reinterpret_cast<float*>(dyn);   // [8 warps][REP][128]
+#pragma unroll
+    for (int h = 0; h < REP; ++h) *reinterpret_cast<float4*>(mrg + ((warp * REP + h) * kD) + lane * 4) = a[h];
+    __syncthreads();
+    for (int o = tid; o < REP * kD; o += kThreads) {
+        const int h = o / kD;
+        float sum = 0.f;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) sum += mrg[w * REP * kD + o];
+        const float r = sum / l_run[h];
+        const size_t idx = (size_t)(hk * REP) * kD + o;
         if (out_dtype == MNNLLM_F32) reinterpret_cast<float*>(out)[idx] = r;
         else reinterpret_cast<__half*>(out)[idx] = __float2half_rn(r);
     }
@@ -246,13 +363,32 @@ __global__ void __launch_bounds__(kThreads) attn_decode_kernel(AttnCache c, cons
 
 }  // namespace
 
-int attn_splits(int Hk, int S) {
-    // enough CTAs for every SM twice over, each with at least one chunk of tokens
+constexpr size_t kDynSmem = 2 * (size_t)kAttnChunk * kD;   // key and value rows of a chunk
+
+template <int REP>
+static cudaError_t ensure_smem() {
+    static PerDevice<bool> configured;   // per instantiation and device
+    return configured.with([&](bool& done) {
+        if (done) return cudaSuccess;
+        cudaError_t e = cudaFuncSetAttribute(attn_decode_kernel<REP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDynSmem);
+        done = e == cudaSuccess;
+        return e;
+    });
+}
+
+// Tokens per CTA: the sequence over about two CTAs per SM, in multiples of 32 and at least 128 (a part
+// costs a merge step: short sequences are not cut finer than that).
+static int tokens_per_split(int Hk, int S) {
     const int n_sm = device_sm_count() > 0 ? device_sm_count() : 148;
     int want = (2 * n_sm + Hk - 1) / Hk;
-    const int chunks = (S + kAttnChunk - 1) / kAttnChunk;
-    if (want > chunks) want = chunks;
-    return want < 1 ? 1 : want;
+    if (want > kAttnChunk) want = kAttnChunk;   // the merge keeps one weight per part in a chunk-sized array
+    int per = ((S + want - 1) / want + 31) / 32 * 32;
+    return per < kAttnMinSplit ? kAttnMinSplit : per;
+}
+
+int attn_splits(int Hk, int S) {
+    const int per = tokens_per_split(Hk, S);
+    return (S + per - 1) / per;
 }
 
 size_t attn_partials_bytes(int H, int Hk, int S) {
@@ -266,13 +402,11 @@ cudaError_t attn_append_launch(const AttnCache& c, const void* k_new, const void
 
 cudaError_t attn_decode_launch(const AttnCache& c, const void* q, void* out, int out_dtype, int H, int S, float* partials,
                                unsigned int* counters, uint32_t* status, cudaStream_t stream) {
-    const int rep = H / c.Hk, splits = attn_splits(c.Hk, S);
-    // whole chunks per split, so that only the last split of the sequence is ragged
-    const int chunks = (S + kAttnChunk - 1) / kAttnChunk;
-    const int per_split = ((chunks + splits - 1) / splits) * kAttnChunk;
+    const int rep = H / c.Hk, splits = attn_splits(c.Hk, S), per_split = tokens_per_split(c.Hk, S);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)splits, (unsigned)c.Hk);
     cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = kDynSmem;
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -280,8 +414,10 @@ cudaError_t attn_decode_launch(const AttnCache& c, const void* q, void* out, int
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     const __half* qh = (const __half*)q;
-#define MNN_CASE(R) \
-    case R: return cudaLaunchKernelEx(&cfg, attn_decode_kernel<R>, c, qh, out, out_dtype, S, per_split, partials, counters, status);
+#define MNN_CASE(R)                                                                                                      \
+    case R:                                                                                                             \
+        if (cudaError_t e = ensure_smem<R>(); e != cudaSuccess) return e;                                               \
+        return cudaLaunchKernelEx(&cfg, attn_decode_kernel<R>, c, qh, out, out_dtype, S, per_split, partials, counters, status);
     switch (rep) {
         MNN_CASE(1) MNN_CASE(2) MNN_CASE(3) MNN_CASE(4) MNN_CASE(5) MNN_CASE(6) MNN_CASE(7) MNN_CASE(8)
     }

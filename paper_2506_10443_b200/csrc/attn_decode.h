@@ -10,6 +10,7 @@ namespace mnnllm {
 constexpr int kAttnHeadDim = 128;      // head_dim the kernels are built for
 constexpr int kAttnMaxRep = 8;         // query heads per kv head at most
 constexpr int kAttnChunk = 256;        // tokens a CTA handles per step
+constexpr int kAttnMinSplit = 128;     // tokens per CTA at least
 
 struct AttnCache {
     uint8_t* k_codes;    // [Hk, S_cap, 128] uint8 codes of the keys
