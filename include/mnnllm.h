@@ -90,7 +90,8 @@ int mnnllm_unpack_w8(const void* packed, uint8_t* q, uint16_t* scale_bits, uint1
 
 /* ------------------------------------------------------------------------------------------------
  * W4A16: y[m, n] = sum_g scale[n, g] * sum_{k in g} (q[n, k] - zero[n, g]) * x[m, k]
- * (Section 4.2, "W4A16 ... on GPUs"; Section 5.1 for the operand shapes).  Accumulation is fp32.
+ * (Section 4.2: the weight-only floating-point pairing that the paper assigns to GPUs; Section 5.1 for
+ * the operand shapes).  Accumulation is fp32.
  *
  *   x       device, fp16 [M, K]
  *   packed  device, a buffer written by mnnllm_pack_w4 for the same N, K, group
