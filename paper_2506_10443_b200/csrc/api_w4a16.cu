@@ -140,23 +140,26 @@ Plan make_plan(int nb_total, int nc_max, int group, int MP, int bits = 4) {
         return bits == 4 ? gemv_w4a16_smem(group, MP, p.WC * p.SR, p.SR, st) : gemv_w8a16_smem(p.WC * p.SR, p.SR, st);
     };
     while (p.stages > 1 && smem(p.stages) > 220 * 1024) --p.stages;
-    const int occ = cached_occupancy(bits, group, MP, p.WC * p.SR, p.SR, p.stages);
-    int clusters = n_sms * occ / p.CS;
-    const int max_useful = (nb_total + p.SR - 1) / p.SR;  // at least SR row blocks per cluster
-    if (clusters > max_useful) clusters = max_useful;
-    if (forced_clusters) clusters = forced_clusters;
-    if (clusters < 1) clusters = 1;
-    p.clusters = clusters;
-    if (p.RBI == 0) {
-        p.RBI = (nb_total + clusters * p.SR - 1) / (clusters * p.SR);
-        p.RBI = p.RBI < 1 ? 1 : (p.RBI > kGemvMaxRBI ? kGemvMaxRBI : p.RBI);
-    }
     // Ring depth: a warp with only a few quanta wants them all in flight before the activations
-    // arrive (three slots); long streams ran 3 % faster with two (measured on the 7B stack and the LM head).
-    if (!stages_forced) {
+    // arrive (three slots); long streams ran 3 % faster with two (measured on the 7B stack and the LM
+    // head).  The shallower ring can also let one more CTA fit an SM, so the grid is sized again
+    // after the depth has been chosen.
+    for (int pass = 0; pass < 2; ++pass) {
+        const int occ = cached_occupancy(bits, group, MP, p.WC * p.SR, p.SR, p.stages);
+        int clusters = n_sms * occ / p.CS;
+        const int max_useful = (nb_total + p.SR - 1) / p.SR;  // at least SR row blocks per cluster
+        if (clusters > max_useful) clusters = max_useful;
+        if (forced_clusters) clusters = forced_clusters;
+        if (clusters < 1) clusters = 1;
+        p.clusters = clusters;
+        if (stages_forced || pass == 1) break;
         const long long warps = (long long)clusters * p.CS * p.WC * p.SR;
         const long long quanta = (long long)nb_total * nc_max;
-        if (quanta > 4 * warps && p.stages > 2) p.stages = 2;
+        if (quanta > 4 * warps && p.stages > 2) p.stages = 2; else break;
+    }
+    if (p.RBI == 0) {
+        p.RBI = (nb_total + p.clusters * p.SR - 1) / (p.clusters * p.SR);
+        p.RBI = p.RBI < 1 ? 1 : (p.RBI > kGemvMaxRBI ? kGemvMaxRBI : p.RBI);
     }
     return p;
 }

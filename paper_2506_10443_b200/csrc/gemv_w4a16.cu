@@ -126,7 +126,7 @@ __device__ __forceinline__ float lora_term(const GemvProblem& P, const float* ts
 }
 
 template <int GROUP, int MP, bool XBF, bool LORA>   // XBF: activations are bf16; LORA: outputs take the bypass term (converted to fp16 as the fragments are built)
-__global__ void __launch_bounds__(kGemvMaxWarps * 32, (MP <= 2 ? 2 : 1))
+__global__ void __launch_bounds__(kGemvMaxWarps * 32, (MP <= 4 ? 2 : 1))
 gemv_w4a16_kernel(const __grid_constant__ GemvLaunch L, uint32_t* __restrict__ status) {
     using C = Cfg<GROUP, MP>;
     extern __shared__ __align__(128) uint8_t smem[];
@@ -236,7 +236,9 @@ gemv_w4a16_kernel(const __grid_constant__ GemvLaunch L, uint32_t* __restrict__ s
 
     const int tokB = r % MP, gsB = r / MP;  // B-operand role of this lane: column r of the MMA
     constexpr bool x_bf16 = XBF;
-    uint32_t B[8][4][2];
+    constexpr bool COMPACT = MP == 4;   // B fragments without their zeros: room for two CTAs per SM
+    BFrag<GROUP, MP, COMPACT> B;
+    B.gs = gsB;
     float C1[C::NSETS][2], C2[C::NSETS][2];
     int cur_j = -1, slot = 0;
     uint32_t phase = 0;
@@ -258,7 +260,10 @@ gemv_w4a16_kernel(const __grid_constant__ GemvLaunch L, uint32_t* __restrict__ s
                     // a lane holds the slabs of its groups gsB + GPS * s only (its other B entries are
                     // zero): load those once, take the group sums from the same registers
                     float v1[C::NSETS], v2[C::NSETS];
-                    uint32_t Pm[C::NSETS][C::SPG][4][2];
+                    uint32_t Pl[COMPACT ? 1 : C::NSETS][C::SPG][4][2];
+                    auto Pm = [&](int s, int sp) -> uint32_t (&)[4][2] {
+                        if constexpr (COMPACT) return B.v[s * C::SPG + sp]; else return Pl[s][sp];
+                    };
 #pragma unroll
                     for (int s = 0; s < C::NSETS; ++s) {
                         float lo = 0.f, hi = 0.f;
@@ -273,14 +278,14 @@ gemv_w4a16_kernel(const __grid_constant__ GemvLaunch L, uint32_t* __restrict__ s
                                 u1 = px[1];
                                 if (x_bf16) { u0 = bf16x8_to_f16x8(u0); u1 = bf16x8_to_f16x8(u1); }
                             }
-                            Pm[s][sp][0][0] = __byte_perm(u0.x, u0.y, 0x5410);
-                            Pm[s][sp][0][1] = __byte_perm(u0.z, u0.w, 0x5410);
-                            Pm[s][sp][1][0] = __byte_perm(u0.x, u0.y, 0x7632);
-                            Pm[s][sp][1][1] = __byte_perm(u0.z, u0.w, 0x7632);
-                            Pm[s][sp][2][0] = __byte_perm(u1.x, u1.y, 0x5410);
-                            Pm[s][sp][2][1] = __byte_perm(u1.z, u1.w, 0x5410);
-                            Pm[s][sp][3][0] = __byte_perm(u1.x, u1.y, 0x7632);
-                            Pm[s][sp][3][1] = __byte_perm(u1.z, u1.w, 0x7632);
+                            Pm(s, sp)[0][0] = __byte_perm(u0.x, u0.y, 0x5410);
+                            Pm(s, sp)[0][1] = __byte_perm(u0.z, u0.w, 0x5410);
+                            Pm(s, sp)[1][0] = __byte_perm(u0.x, u0.y, 0x7632);
+                            Pm(s, sp)[1][1] = __byte_perm(u0.z, u0.w, 0x7632);
+                            Pm(s, sp)[2][0] = __byte_perm(u1.x, u1.y, 0x5410);
+                            Pm(s, sp)[2][1] = __byte_perm(u1.z, u1.w, 0x5410);
+                            Pm(s, sp)[3][0] = __byte_perm(u1.x, u1.y, 0x7632);
+                            Pm(s, sp)[3][1] = __byte_perm(u1.z, u1.w, 0x7632);
                             const float2 a0 = h2f2(u0.x), a1 = h2f2(u0.y), a2 = h2f2(u1.x), a3 = h2f2(u1.y);
                             const float2 b0 = h2f2(u0.z), b1 = h2f2(u0.w), b2 = h2f2(u1.z), b3 = h2f2(u1.w);
                             lo += ((a0.x + a0.y) + (a1.x + a1.y)) + ((a2.x + a2.y) + (a3.x + a3.y));
@@ -293,14 +298,16 @@ gemv_w4a16_kernel(const __grid_constant__ GemvLaunch L, uint32_t* __restrict__ s
                         v1[s] = 1024.f * lo + 64.f * hi;
                         v2[s] = lo + hi;
                     }
+                    if constexpr (!COMPACT) {
 #pragma unroll
-                    for (int sl = 0; sl < 8; ++sl) {
-                        const int gi = sl / C::SPG;
-                        const bool mine = gsB == gi % C::GPS;
+                        for (int sl = 0; sl < 8; ++sl) {
+                            const int gi = sl / C::SPG;
+                            const bool mine = gsB == gi % C::GPS;
 #pragma unroll
-                        for (int a = 0; a < 4; ++a)
+                            for (int a = 0; a < 4; ++a)
 #pragma unroll
-                            for (int b = 0; b < 2; ++b) B[sl][a][b] = mine ? Pm[gi / C::GPS][sl % C::SPG][a][b] : 0u;
+                                for (int b = 0; b < 2; ++b) B.v[sl][a][b] = mine ? Pl[gi / C::GPS][sl % C::SPG][a][b] : 0u;
+                        }
                     }
                     // the correction terms of accumulator column 2c + e = (token, group slot) sit in
                     // the quad whose row index r equals that column
@@ -324,8 +331,8 @@ gemv_w4a16_kernel(const __grid_constant__ GemvLaunch L, uint32_t* __restrict__ s
                     const uint4* slabs = reinterpret_cast<const uint4*>(qp);
 
                     float D[C::NSETS][4];
-                    if (ns == 8) quantum_mma<GROUP, MP, true>(slabs, lane, 8, B, D);
-                    else quantum_mma<GROUP, MP, false>(slabs, lane, ns, B, D);
+                    if (ns == 8) quantum_mma<GROUP, MP, true, COMPACT>(slabs, lane, 8, B, D);
+                    else quantum_mma<GROUP, MP, false, COMPACT>(slabs, lane, ns, B, D);
 
                     // ---- rescale: column (2c + e) of tile s is (token, group) = (col % MP, s*GPS + col / MP) ----
                     float out[2][2] = {{0.f, 0.f}, {0.f, 0.f}};  // [row half h][column e]

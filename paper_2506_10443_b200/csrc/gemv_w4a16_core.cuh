@@ -47,9 +47,24 @@ __device__ __forceinline__ void store_out(void* y, int dtype, size_t idx, float 
 // and logic ops of different slabs can be interleaved.  Accumulator tile `set` collects GPS groups;
 // with few tiles the four MMAs of a slab go to separate banks (summed afterwards) to keep the
 // dependent-MMA chains short.
-template <int GROUP, int MP, bool FULL>
+// B operand of slab sl, MMA a: either the full array (zeros stored for the groups that are not this
+// lane's), or, in the compact form, only the lane's own slabs Pm[set][slab of the group], with the
+// zeros made by a select where they are needed (half the registers at MP = 4, two selects per MMA).
+template <int GROUP, int MP, bool COMPACT>
+struct BFrag {
+    using C = Cfg<GROUP, MP>;
+    uint32_t v[COMPACT ? C::NSETS * C::SPG : 8][4][2];
+    int gs;   // this lane's group slot (compact form)
+    __device__ __forceinline__ uint32_t get(int sl, int a, int b) const {
+        if (!COMPACT) return v[sl][a][b];
+        const int gi = sl / C::SPG;
+        return gs == gi % C::GPS ? v[(gi / C::GPS) * C::SPG + sl % C::SPG][a][b] : 0u;
+    }
+};
+
+template <int GROUP, int MP, bool FULL, bool COMPACT>
 __device__ __forceinline__ void quantum_mma(const uint4* __restrict__ slabs, int lane, int ns,
-                                            const uint32_t (&B)[8][4][2], float (&D)[Cfg<GROUP, MP>::NSETS][4]) {
+                                            const BFrag<GROUP, MP, COMPACT>& B, float (&D)[Cfg<GROUP, MP>::NSETS][4]) {
     using C = Cfg<GROUP, MP>;
     constexpr int NBANK = C::NSETS == 1 ? 2 : 1;  // four banks spill at the 128-register cap and run slower
     constexpr uint32_t LO = 0x000F000Fu, HI = 0x00F000F0u, M1024 = 0x64006400u, M64 = 0x54005400u;
@@ -65,13 +80,13 @@ __device__ __forceinline__ void quantum_mma(const uint4* __restrict__ slabs, int
             const int set = (sl / C::SPG) / C::GPS;
             const uint32_t x8 = w.x >> 8, z8 = w.z >> 8, y8 = w.y >> 8, w8 = w.w >> 8;
             mma_m16n8k16_f16(acc[set][0 % NBANK], lop3_and_or(w.x, LO, M1024), lop3_and_or(w.z, LO, M1024),
-                             lop3_and_or(w.x, HI, M64), lop3_and_or(w.z, HI, M64), B[sl][0][0], B[sl][0][1]);
+                             lop3_and_or(w.x, HI, M64), lop3_and_or(w.z, HI, M64), B.get(sl, 0, 0), B.get(sl, 0, 1));
             mma_m16n8k16_f16(acc[set][1 % NBANK], lop3_and_or(x8, LO, M1024), lop3_and_or(z8, LO, M1024),
-                             lop3_and_or(x8, HI, M64), lop3_and_or(z8, HI, M64), B[sl][1][0], B[sl][1][1]);
+                             lop3_and_or(x8, HI, M64), lop3_and_or(z8, HI, M64), B.get(sl, 1, 0), B.get(sl, 1, 1));
             mma_m16n8k16_f16(acc[set][2 % NBANK], lop3_and_or(w.y, LO, M1024), lop3_and_or(w.w, LO, M1024),
-                             lop3_and_or(w.y, HI, M64), lop3_and_or(w.w, HI, M64), B[sl][2][0], B[sl][2][1]);
+                             lop3_and_or(w.y, HI, M64), lop3_and_or(w.w, HI, M64), B.get(sl, 2, 0), B.get(sl, 2, 1));
             mma_m16n8k16_f16(acc[set][3 % NBANK], lop3_and_or(y8, LO, M1024), lop3_and_or(w8, LO, M1024),
-                             lop3_and_or(y8, HI, M64), lop3_and_or(w8, HI, M64), B[sl][3][0], B[sl][3][1]);
+                             lop3_and_or(y8, HI, M64), lop3_and_or(w8, HI, M64), B.get(sl, 3, 0), B.get(sl, 3, 1));
         }
     }
 #pragma unroll

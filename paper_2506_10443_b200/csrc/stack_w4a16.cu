@@ -212,7 +212,7 @@ stack_w4a16_kernel(const __grid_constant__ StackHeader H, const StackProblem* __
         // =================== consumers ===================
         const int r = lane >> 2, c = lane & 3;
         const int tokB = r % MP, gsB = r / MP;   // B-operand role of this lane: column r of the MMA
-        uint32_t B[8][4][2];
+        BFrag<GROUP, MP, false> B;
         float C1[C::NSETS][2], C2[C::NSETS][2];
         uint32_t n_finished = 0;                  // problems this CTA has stored outputs of
         // this warp's slots of the ring, used in order across problems
@@ -354,7 +354,7 @@ stack_w4a16_kernel(const __grid_constant__ StackHeader H, const StackProblem* __
                             for (int a = 0; a < 4; ++a)
 #pragma unroll
                                 for (int b = 0; b < 2; ++b)
-                                    B[sl][a][b] = mine ? Pm[gi / C::GPS][sl % C::SPG][a][b] : 0u;
+                                    B.v[sl][a][b] = mine ? Pm[gi / C::GPS][sl % C::SPG][a][b] : 0u;
                         }
                         if (staged) {
                             // correction terms of accumulator column 2c + e = (token, group slot) of tile s
@@ -395,8 +395,8 @@ stack_w4a16_kernel(const __grid_constant__ StackHeader H, const StackProblem* __
                     const uint8_t* qp = my_ring + (size_t)slot * C::QB;
                     const uint4* slabs = reinterpret_cast<const uint4*>(qp);
                     float Dm[C::NSETS][4];
-                    if (ns == 8) quantum_mma<GROUP, MP, true>(slabs, lane, 8, B, Dm);
-                    else quantum_mma<GROUP, MP, false>(slabs, lane, ns, B, Dm);
+                    if (ns == 8) quantum_mma<GROUP, MP, true, false>(slabs, lane, 8, B, Dm);
+                    else quantum_mma<GROUP, MP, false, false>(slabs, lane, ns, B, Dm);
 
                     float out[2][2] = {{0.f, 0.f}, {0.f, 0.f}};   // [row half h][column e]
                     auto rescale = [&](const int ngc) {
