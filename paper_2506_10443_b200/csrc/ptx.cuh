@@ -125,6 +125,22 @@ __device__ __forceinline__ uint32_t cluster_nctarank() {
 __device__ __forceinline__ void cluster_sync() {
     asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
+// 8- and 16-byte loads from the shared memory of another CTA of the cluster (the address aligned likewise);
+// not volatile: independent loads may be in flight together, the cluster barrier's "memory" clobber orders them
+__device__ __forceinline__ float2 ld_dsmem_f32x2(const float* local_smem_ptr, uint32_t cta_rank) {
+    uint32_t remote;
+    float2 v;
+    asm("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(smem_u32(local_smem_ptr)), "r"(cta_rank));
+    asm volatile("ld.shared::cluster.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(remote));
+    return v;
+}
+__device__ __forceinline__ float4 ld_dsmem_f32x4(const float* local_smem_ptr, uint32_t cta_rank) {
+    uint32_t remote;
+    float4 v;
+    asm("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(smem_u32(local_smem_ptr)), "r"(cta_rank));
+    asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(remote));
+    return v;
+}
 __device__ __forceinline__ float ld_dsmem_f32(const float* local_smem_ptr, uint32_t cta_rank) {
     uint32_t remote;
     float v;
