@@ -119,8 +119,9 @@ __global__ void __launch_bounds__(kThreads) attn_decode_kernel(AttnCache c, cons
                                                                int out_dtype, int S, int per_split, float* partials,
                                                                unsigned int* counters, uint32_t* status) {
     __shared__ float sc[REP][kAttnChunk];   // scores, then weights
-    __shared__ float qsum[REP];             // sum_d q[h, d]
-    __shared__ float m_run[REP], l_run[REP], rescale[REP];
+    __shared__ float m_run[REP], l_run[REP];
+    __shared__ __align__(16) float ps[kThreads / 32][REP * 16 + 8];   // per warp: weights of its 16 tokens, rescale factors
+    __shared__ float wm[kThreads / 32][REP], wl[kThreads / 32][REP];  // the warps' maxima and sums, merged at the end
     __shared__ __align__(16) float red[4][REP][kD];   // cross-warp sum of the accumulators
     __shared__ unsigned int last_flag;
     __shared__ uint32_t meta_s[2][kTile];    // a tile's (scale, zero) pairs
@@ -160,6 +161,7 @@ __global__ void __launch_bounds__(kThreads) attn_decode_kernel(AttnCache c, cons
 
     // query fragments: k-step s covers head_dim entries 16 (cq + 4 (s >> 2)) + 4 (s & 3) + {0, 1 | 2, 3}
     uint32_t qa0[8], qa2[8];
+    float qs;   // sum_d q[g, d] of this lane's head
     {
         const __half* qr = q + (size_t)(hk * REP + (g < REP ? g : 0)) * kD;
         float sum = 0.f;
@@ -174,27 +176,31 @@ __global__ void __launch_bounds__(kThreads) attn_decode_kernel(AttnCache c, cons
         }
         sum += __shfl_xor_sync(0xffffffffu, sum, 1);
         sum += __shfl_xor_sync(0xffffffffu, sum, 2);
-        if (warp == 0 && cq == 0 && g < REP) qsum[g] = sum;
+        qs = sum;
     }
-    if (tid < REP) { m_run[tid] = -INFINITY; l_run[tid] = 0.f; }
     __syncthreads();
     bool dead = false;   // a bounded wait gave up
 
-    float acc[REP][4];
+    // Every warp keeps its own online softmax over the tokens it is dealt (16 of each tile): its
+    // scores, weights and weighted values need no barrier of the CTA; the warps' states are merged
+    // once, after the last tile.
+    uint64_t acc2[REP][2];   // packed pairs of fp32: this lane's four value entries per head
 #pragma unroll
-    for (int h = 0; h < REP; ++h)
-#pragma unroll
-        for (int i = 0; i < 4; ++i) acc[h][i] = 0.f;
+    for (int h = 0; h < REP; ++h) acc2[h][0] = acc2[h][1] = 0ull;
+    float m_w = -INFINITY, l_w = 0.f;   // head g of this lane's quad: running maximum, this lane's share of the sum
+    float* pw = &ps[warp][0];           // [REP][16] weights of the warp's tokens, then [8] rescale factors
 
     for (int c0 = t0, it = 0; c0 < t1; c0 += kTile, ++it) {
         const int n = min(kTile, t1 - c0), st = it & 1;
         const uint8_t* kbuf = dyn + (size_t)st * 2 * kTile * kD;
         const uint8_t* vbuf = kbuf + kTile * kD;
         const uint32_t* meta_t = meta_s[st];
-        // the next tile into the other stage (its last readers passed the barrier that ended the
-        // previous round), so that its rows arrive while this tile is worked on
+        // one barrier per tile: every warp is through with the previous tile (so the other stage may be
+        // refilled and its scale/zero pairs rewritten), and a wait that gave up is known to all
+        dead = __syncthreads_or(dead);
+        if (dead) break;
         const int c1 = c0 + kTile;
-        if (c1 < t1 && !dead) {
+        if (c1 < t1) {
             const int n1 = min(kTile, t1 - c1);
             if (tid == 0) {
                 ptx::mbar_arrive_expect_tx(&bar[st ^ 1], 2u * (uint32_t)n1 * kD);
@@ -202,15 +208,17 @@ __global__ void __launch_bounds__(kThreads) attn_decode_kernel(AttnCache c, cons
             }
             if (tid < n1) meta_s[st ^ 1][tid] = __ldg(c.k_meta + (size_t)hk * c.S_cap + c1 + tid);
         }
-        if (!dead && !ptx::mbar_wait_bounded(&bar[st], (uint32_t)(it >> 1) & 1u, 1u << 22)) {
+        if (!ptx::mbar_wait_bounded(&bar[st], (uint32_t)(it >> 1) & 1u, 1u << 22)) {
             dead = true;
             if (lane == 0) atomicOr(status, 0x800u);
         }
-        dead = __syncthreads_or(dead);
-        if (dead) break;
-        // ---- 1. scores: token groups of eight, one group per warp and round
-        for (int g0 = warp * 8; g0 < n; g0 += 64) {
-            const int tok = g0 + g;   // this lane's B-operand column
+        const int w0 = warp * 16;         // this warp's tokens of the tile: w0 .. w0 + 15
+        if (w0 >= n) continue;            // (uniform per warp)
+        // ---- 1. scores of two groups of eight tokens; lane (g, cq) gets head g, tokens 2 cq, 2 cq + 1
+        float sv[4];
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            const int tok = w0 + j * 8 + g;   // this lane's B-operand column
             uint4 u0 = make_uint4(0, 0, 0, 0), u1 = u0;
             if (tok < n) {
                 const uint4* kr = reinterpret_cast<const uint4*>(kbuf + tok * kD);
@@ -223,66 +231,110 @@ __global__ void __launch_bounds__(kThreads) attn_decode_kernel(AttnCache c, cons
             for (int s = 0; s < 8; ++s)
                 ptx::mma_m16n8k16_f16(d, qa0[s], 0u, qa2[s], 0u, __byte_perm(w[s], 0x64646464u, 0x4140),
                                       __byte_perm(w[s], 0x64646464u, 0x4342));
-            // d[0], d[1]: query head g, tokens g0 + 2 cq and + 1
-            if (g < REP) {
 #pragma unroll
-                for (int e = 0; e < 2; ++e) {
-                    const int t = g0 + 2 * cq + e;
-                    if (t < n) {
-                        const uint32_t meta = meta_t[t];
-                        const __half2 sz = *reinterpret_cast<const __half2*>(&meta);
-                        sc[g][t] = (__low2float(sz) * 0.08838834764831845f) * (d[e] - (1024.f + __high2float(sz)) * qsum[g]);
+            for (int e = 0; e < 2; ++e) {
+                const int t = w0 + j * 8 + 2 * cq + e;
+                float v = -INFINITY;
+                if (t < n) {
+                    const uint32_t meta = meta_t[t];
+                    const __half2 sz = *reinterpret_cast<const __half2*>(&meta);
+                    v = (__low2float(sz) * 0.08838834764831845f) * (d[e] - (1024.f + __high2float(sz)) * qs);
+                }
+                sv[2 * j + e] = v;
+            }
+        }
+        // ---- 2. the quad's new maximum for head g, the factor for what is accumulated, the weights
+        float mx = fmaxf(fmaxf(sv[0], sv[1]), fmaxf(sv[2], sv[3]));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+        const float m_new = fmaxf(m_w, mx);             // finite: token w0 is below n
+        const float r = expf(m_w - m_new);              // 0 on the warp's first tile (m_w = -inf)
+        float psum = 0.f;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            sv[i] = expf(sv[i] - m_new);                // 0 for a token past the end (-inf)
+            psum += sv[i];
+        }
+        l_w = l_w * r + psum;
+        m_w = m_new;
+        if (g < REP) {
+            *reinterpret_cast<float2*>(pw + g * 16 + 2 * cq) = make_float2(sv[0], sv[1]);
+            *reinterpret_cast<float2*>(pw + g * 16 + 8 + 2 * cq) = make_float2(sv[2], sv[3]);
+            if (cq == 0) pw[REP * 16 + g] = r;
+        }
+        __syncwarp();
+        // ---- 3. weighted values: a lane holds four entries of a value row, for every head
+        {
+            const float4 r0 = *reinterpret_cast<const float4*>(pw + REP * 16);
+            const float4 r1 = *reinterpret_cast<const float4*>(pw + REP * 16 + 4);
+            const float rr[8] = {r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w};
+#pragma unroll
+            for (int h = 0; h < REP; ++h) {
+                const uint64_t r2 = ptx::f32x2_pack(__float_as_uint(rr[h]), __float_as_uint(rr[h]));
+                acc2[h][0] = ptx::f32x2_fma(acc2[h][0], r2, 0ull);   // + (+0, +0)
+                acc2[h][1] = ptx::f32x2_fma(acc2[h][1], r2, 0ull);
+            }
+        }
+        const uint32_t* vr = reinterpret_cast<const uint32_t*>(vbuf) + (size_t)w0 * (kD / 4) + lane;
+#pragma unroll
+        for (int t4 = 0; t4 < 4; ++t4) {
+            if (w0 + 4 * t4 >= n) break;
+            float4 p4[REP];
+#pragma unroll
+            for (int h = 0; h < REP; ++h) p4[h] = *reinterpret_cast<const float4*>(pw + h * 16 + 4 * t4);
+#pragma unroll
+            for (int tt = 0; tt < 4; ++tt) {
+                if (w0 + 4 * t4 + tt < n) {   // rows past the end hold whatever the buffer held before
+                    float val[4];
+                    e4m3x4_to_f32_scaled(vr[(4 * t4 + tt) * (kD / 4)], val);
+                    const uint64_t v01 = ptx::f32x2_pack(__float_as_uint(val[0]), __float_as_uint(val[1]));
+                    const uint64_t v23 = ptx::f32x2_pack(__float_as_uint(val[2]), __float_as_uint(val[3]));
+#pragma unroll
+                    for (int h = 0; h < REP; ++h) {
+                        const float pv = tt == 0 ? p4[h].x : (tt == 1 ? p4[h].y : (tt == 2 ? p4[h].z : p4[h].w));
+                        const uint64_t pp = ptx::f32x2_pack(__float_as_uint(pv), __float_as_uint(pv));
+                        acc2[h][0] = ptx::f32x2_fma(pp, v01, acc2[h][0]);
+                        acc2[h][1] = ptx::f32x2_fma(pp, v23, acc2[h][1]);
                     }
                 }
             }
         }
-        __syncthreads();
-        // ---- 2. running maximum and weights
-        if (warp < REP) {
-            float mx = -INFINITY;
-            for (int t = lane; t < n; t += 32) mx = fmaxf(mx, sc[warp][t]);
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-            const float m_new = fmaxf(m_run[warp], mx);
-            float sum = 0.f;
-            for (int t = lane; t < n; t += 32) {
-                const float p = expf(sc[warp][t] - m_new);
-                sc[warp][t] = p;
-                sum += p;
-            }
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-            if (lane == 0) {
-                const float r = expf(m_run[warp] - m_new);   // 0 on the first chunk (m_run = -inf)
-                rescale[warp] = r;
-                l_run[warp] = l_run[warp] * r + sum;
-                m_run[warp] = m_new;
-            }
-        }
-        __syncthreads();
-        // ---- 3. weighted values
-#pragma unroll
-        for (int h = 0; h < REP; ++h)
-#pragma unroll
-            for (int i = 0; i < 4; ++i) acc[h][i] *= rescale[h];
-        const uint32_t* vr = reinterpret_cast<const uint32_t*>(vbuf) + lane;
-#pragma unroll 4
-        for (int t = warp; t < n; t += 8) {
-            float val[4];
-            e4m3x4_to_f32_scaled(vr[t * (kD / 4)], val);
-#pragma unroll
-            for (int h = 0; h < REP; ++h) {
-                const float p = sc[h][t];
-#pragma unroll
-                for (int i = 0; i < 4; ++i) acc[h][i] = fmaf(p, val[i], acc[h][i]);
-            }
-        }
-        __syncthreads();   // sc, rescale and the row buffers are rewritten by the next chunk
+        __syncwarp();   // pw is rewritten for the next tile
     }
+    dead = __syncthreads_or(dead);
     if (dead)   // give copies in flight time to land; this CTA's part is not counted (the status word says why)
         for (int i = 0; i < 50; ++i) __nanosleep(1000);
 
     ptx::pdl_launch_dependents();   // the next kernel's CTAs come in (and request their rows) while the parts are merged
+    // ---- the warps' states brought to the CTA's maximum per head
+    l_w += __shfl_xor_sync(0xffffffffu, l_w, 1);
+    l_w += __shfl_xor_sync(0xffffffffu, l_w, 2);
+    if (cq == 0 && g < REP) {
+        wm[warp][g] = m_w;
+        wl[warp][g] = l_w;
+    }
+    __syncthreads();
+    float acc[REP][4];
+#pragma unroll
+    for (int h = 0; h < REP; ++h) {
+        float M = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < kThreads / 32; ++w) M = fmaxf(M, wm[w][h]);
+        const float mine_m = wm[warp][h];
+        const float f = mine_m == -INFINITY ? 0.f : expf(mine_m - M);   // a warp without tokens carries nothing
+        ptx::f32x2_unpack(acc2[h][0], acc[h][0], acc[h][1]);
+        ptx::f32x2_unpack(acc2[h][1], acc[h][2], acc[h][3]);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) acc[h][i] *= f;
+    }
+    if (tid < REP) {
+        float M = -INFINITY, l = 0.f;
+        for (int w = 0; w < kThreads / 32; ++w) M = fmaxf(M, wm[w][tid]);
+        for (int w = 0; w < kThreads / 32; ++w)   // warp order: the same sum whatever the timing
+            l += wm[w][tid] == -INFINITY ? 0.f : wl[w][tid] * expf(wm[w][tid] - M);
+        m_run[tid] = M;
+        l_run[tid] = l;
+    }
     // ---- the eight warps' accumulators summed in a fixed tree (4 + 4, 2 + 2, 1 + 1)
 #pragma unroll
     for (int stride = 4; stride >= 1; stride >>= 1) {
