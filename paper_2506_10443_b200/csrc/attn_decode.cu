@@ -23,7 +23,9 @@ namespace {
 
 constexpr int kD = kAttnHeadDim;
 constexpr int kThreads = 256;
+constexpr int kMaxParts = 32;   // parts per kv head that reach the final merge (256 CTAs in clusters of eight, or fewer than 16 single CTAs)
 constexpr int kTile = 128;   // tokens per stage of the row buffers (two stages)
+constexpr size_t kRowBytes = 2 * 2 * (size_t)kTile * 128;   // two stages of key and value rows
 
 // fp16 bits of v, saturating at +-65504 instead of infinity
 __device__ __forceinline__ uint16_t f16_sat_bits(float v) {
@@ -118,11 +120,10 @@ template <int REP>
 __global__ void __launch_bounds__(kThreads) attn_decode_kernel(AttnCache c, const __half* __restrict__ q, void* out,
                                                                int out_dtype, int S, int per_split, float* partials,
                                                                unsigned int* counters, uint32_t* status) {
-    __shared__ float sc[REP][kAttnChunk];   // scores, then weights
+    __shared__ float sc[REP][kMaxParts];    // final merge: the parts' weights
     __shared__ float m_run[REP], l_run[REP];
     __shared__ __align__(16) float ps[kThreads / 32][REP * 16 + 8];   // per warp: weights of its 16 tokens, rescale factors
     __shared__ float wm[kThreads / 32][REP], wl[kThreads / 32][REP];  // the warps' maxima and sums, merged at the end
-    __shared__ __align__(16) float red[4][REP][kD];   // cross-warp sum of the accumulators
     __shared__ unsigned int last_flag;
     __shared__ uint32_t meta_s[2][kTile];    // a tile's (scale, zero) pairs
     __shared__ __align__(8) uint64_t bar[2];  // a tile's key and value rows have landed
@@ -314,18 +315,21 @@ __global__ void __launch_bounds__(kThreads) attn_decode_kernel(AttnCache c, cons
         wl[warp][g] = l_w;
     }
     __syncthreads();
-    float acc[REP][4];
+    // every warp scales its accumulators to the CTA's maximum and leaves them in the row buffers
+    // (all tiles have been consumed); then each (head, four entries) is summed over the warps in warp
+    // order by one thread: two CTA barriers in all
+    float* wacc = reinterpret_cast<float*>(dyn);   // [warps][REP][128]
 #pragma unroll
     for (int h = 0; h < REP; ++h) {
         float M = -INFINITY;
 #pragma unroll
         for (int w = 0; w < kThreads / 32; ++w) M = fmaxf(M, wm[w][h]);
         const float mine_m = wm[warp][h];
-        const float f = mine_m == -INFINITY ? 0.f : expf(mine_m - M);   // a warp without tokens carries nothing
-        ptx::f32x2_unpack(acc2[h][0], acc[h][0], acc[h][1]);
-        ptx::f32x2_unpack(acc2[h][1], acc[h][2], acc[h][3]);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) acc[h][i] *= f;
+        const float f = mine_m == -INFINITY ? 0.f : expf(mine_m - M) * 256.f;   // a warp without tokens carries nothing; 2^8: the values' scale
+        float a0, a1, a2, a3;
+        ptx::f32x2_unpack(acc2[h][0], a0, a1);
+        ptx::f32x2_unpack(acc2[h][1], a2, a3);
+        *reinterpret_cast<float4*>(wacc + (size_t)(warp * REP + h) * kD + lane * 4) = make_float4(a0 * f, a1 * f, a2 * f, a3 * f);
     }
     if (tid < REP) {
         float M = -INFINITY, l = 0.f;
@@ -335,89 +339,67 @@ __global__ void __launch_bounds__(kThreads) attn_decode_kernel(AttnCache c, cons
         m_run[tid] = M;
         l_run[tid] = l;
     }
-    // ---- the eight warps' accumulators summed in a fixed tree (4 + 4, 2 + 2, 1 + 1)
-#pragma unroll
-    for (int stride = 4; stride >= 1; stride >>= 1) {
-        if (warp >= stride && warp < 2 * stride)
-#pragma unroll
-            for (int h = 0; h < REP; ++h)
-                *reinterpret_cast<float4*>(&red[warp - stride][h][lane * 4]) = make_float4(acc[h][0], acc[h][1], acc[h][2], acc[h][3]);
-        __syncthreads();
-        if (warp < stride)
-#pragma unroll
-            for (int h = 0; h < REP; ++h) {
-                const float4 o = *reinterpret_cast<const float4*>(&red[warp][h][lane * 4]);
-                acc[h][0] += o.x; acc[h][1] += o.y; acc[h][2] += o.z; acc[h][3] += o.w;
-            }
-        __syncthreads();
-    }
-    // ---- this CTA's part: {m, l, acc[128]} per query head.  In a cluster the parts of its CTAs are
-    // first merged through distributed shared memory by the CTA of rank 0 (in rank order: the same sum
-    // whatever the timing), so that the final merge reads an eighth of the parts.
+    __syncthreads();
+    // ---- this CTA's part: {m, l, acc[128]} per query head.  In a cluster every CTA stores its part
+    // into the shared memory of the CTA of rank 0 (distributed shared memory), which merges them in
+    // rank order (the same sum whatever the timing): the final merge reads an eighth of the parts.
     constexpr int kPart = kD + 2;
+    constexpr int kPitch = kD + 4;   // in shared memory {m, l, -, -, acc[128]}: the accumulators on a 16-byte boundary
     const int CS = (int)ptx::cluster_nctarank(), crank = (int)ptx::cluster_ctarank();
     const int n_parts = n_splits / CS;
     float* mine = partials + ((size_t)(hk * n_parts + split / CS) * REP) * kPart;
-    if (CS == 1) {
-        if (warp == 0)
+    float* cbuf = reinterpret_cast<float*>(dyn + kRowBytes);   // [8 ranks][REP][kPitch], written by the peers
+    for (int idx = tid; idx < REP * 32; idx += kThreads) {
+        const int h = idx >> 5;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-            for (int h = 0; h < REP; ++h)
-#pragma unroll
-                for (int i = 0; i < 4; ++i) __stcg(mine + h * kPart + 2 + lane * 4 + i, acc[h][i] * 256.f);
-        if (tid < REP) {
-            __stcg(mine + tid * kPart, m_run[tid]);
-            __stcg(mine + tid * kPart + 1, l_run[tid]);
+        for (int w = 0; w < kThreads / 32; ++w) {
+            const float4 o = *reinterpret_cast<const float4*>(wacc + (size_t)(w * REP + h) * kD + lane * 4);
+            v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w;
         }
-    } else {
-        constexpr int kPitch = kD + 4;   // {m, l, -, -, acc[128]}: the accumulators on a 16-byte boundary
-        float* part_s = &red[0][0][0];   // [REP][kPitch]; the tree above is done with it
-        if (warp == 0)
-#pragma unroll
-            for (int h = 0; h < REP; ++h)
-                *reinterpret_cast<float4*>(part_s + h * kPitch + 4 + lane * 4) =
-                    make_float4(acc[h][0] * 256.f, acc[h][1] * 256.f, acc[h][2] * 256.f, acc[h][3] * 256.f);
-        if (tid < REP) {
-            part_s[tid * kPitch] = m_run[tid];
-            part_s[tid * kPitch + 1] = l_run[tid];
+        if (CS == 1) {
+            __stcg(reinterpret_cast<float2*>(mine + h * kPart + 2 + lane * 4), make_float2(v.x, v.y));
+            __stcg(reinterpret_cast<float2*>(mine + h * kPart + 4 + lane * 4), make_float2(v.z, v.w));
+            if (lane == 0) __stcg(reinterpret_cast<float2*>(mine + h * kPart), make_float2(m_run[h], l_run[h]));
+        } else {
+            float* slot = cbuf + (size_t)(crank * REP + h) * kPitch;
+            ptx::st_dsmem_f32x4(slot + 4 + lane * 4, 0u, v);
+            if (lane == 0) ptx::st_dsmem_f32x2(slot, 0u, make_float2(m_run[h], l_run[h]));
         }
-        ptx::cluster_sync();
-        if (crank == 0) {
-            for (int idx = tid; idx < REP * 32; idx += kThreads) {
-                const int h = idx >> 5;
-                const float* ph = part_s + h * kPitch;
-                // every remote load first (they are independent), then the arithmetic
-                float2 ml[8];
-                float4 av[8];
+    }
+    if (CS > 1) {
+        ptx::cluster_arrive_release();   // this CTA's stores into rank 0 are ordered before the arrival
+        if (crank != 0) return;          // nothing reads a peer's shared memory: it may go
+        ptx::cluster_wait_acquire();
+        for (int idx = tid; idx < REP * 32; idx += kThreads) {
+            const int h = idx >> 5;
+            float2 ml[8];
+            float4 av[8];
 #pragma unroll
-                for (int r = 0; r < 8; ++r) {
-                    ml[r] = make_float2(-INFINITY, 0.f);
-                    av[r] = make_float4(0.f, 0.f, 0.f, 0.f);
-                    if (r < CS) {
-                        ml[r] = ptx::ld_dsmem_f32x2(ph, (uint32_t)r);
-                        av[r] = ptx::ld_dsmem_f32x4(ph + 4 + lane * 4, (uint32_t)r);
-                    }
-                }
-                float m = -INFINITY;
-#pragma unroll
-                for (int r = 0; r < 8; ++r) m = fmaxf(m, ml[r].x);
-                float l = 0.f, a4[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-                for (int r = 0; r < 8; ++r) {   // rank order: the same sum whatever the timing
-                    const float w = ml[r].x == -INFINITY ? 0.f : expf(ml[r].x - m);   // a CTA without tokens carries nothing
-                    l = fmaf(ml[r].y, w, l);
-                    a4[0] = fmaf(av[r].x, w, a4[0]); a4[1] = fmaf(av[r].y, w, a4[1]);
-                    a4[2] = fmaf(av[r].z, w, a4[2]); a4[3] = fmaf(av[r].w, w, a4[3]);
-                }
-#pragma unroll
-                for (int i = 0; i < 4; ++i) __stcg(mine + h * kPart + 2 + lane * 4 + i, a4[i]);
-                if (lane == 0) {
-                    __stcg(mine + h * kPart, m);
-                    __stcg(mine + h * kPart + 1, l);
+            for (int r = 0; r < 8; ++r) {
+                ml[r] = make_float2(-INFINITY, 0.f);
+                av[r] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (r < CS) {
+                    const float* slot = cbuf + (size_t)(r * REP + h) * kPitch;
+                    ml[r] = *reinterpret_cast<const float2*>(slot);
+                    av[r] = *reinterpret_cast<const float4*>(slot + 4 + lane * 4);
                 }
             }
+            float m = -INFINITY;
+#pragma unroll
+            for (int r = 0; r < 8; ++r) m = fmaxf(m, ml[r].x);
+            float l = 0.f, a4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int r = 0; r < 8; ++r) {   // rank order
+                const float w = ml[r].x == -INFINITY ? 0.f : expf(ml[r].x - m);   // a CTA without tokens carries nothing
+                l = fmaf(ml[r].y, w, l);
+                a4[0] = fmaf(av[r].x, w, a4[0]); a4[1] = fmaf(av[r].y, w, a4[1]);
+                a4[2] = fmaf(av[r].z, w, a4[2]); a4[3] = fmaf(av[r].w, w, a4[3]);
+            }
+            __stcg(reinterpret_cast<float2*>(mine + h * kPart + 2 + lane * 4), make_float2(a4[0], a4[1]));
+            __stcg(reinterpret_cast<float2*>(mine + h * kPart + 4 + lane * 4), make_float2(a4[2], a4[3]));
+            if (lane == 0) __stcg(reinterpret_cast<float2*>(mine + h * kPart), make_float2(m, l));
         }
-        ptx::cluster_sync();   // rank 0 has read its peers' shared memory
-        if (crank != 0) return;
     }
     __threadfence();
     __syncthreads();
@@ -432,21 +414,21 @@ __global__ void __launch_bounds__(kThreads) attn_decode_kernel(AttnCache c, cons
     // warp h: head h's {m, l} of every part in one pass of loads (n_parts <= 256: eight per lane), the
     // overall maximum, every part's weight exp(m_s - m) (into sc) and the sum of the weighted l_s
     if (warp < REP) {
-        float2 ml[kAttnChunk / 32];
+        float2 ml[kMaxParts / 32];
 #pragma unroll
-        for (int i = 0; i < kAttnChunk / 32; ++i) {
+        for (int i = 0; i < kMaxParts / 32; ++i) {
             const int s = lane + 32 * i;
             ml[i] = s < n_parts ? __ldcg(reinterpret_cast<const float2*>(parts + ((size_t)s * REP + warp) * kPart))
                                  : make_float2(-INFINITY, 0.f);
         }
         float m = -INFINITY;
 #pragma unroll
-        for (int i = 0; i < kAttnChunk / 32; ++i) m = fmaxf(m, ml[i].x);
+        for (int i = 0; i < kMaxParts / 32; ++i) m = fmaxf(m, ml[i].x);
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
         float l = 0.f;
 #pragma unroll
-        for (int i = 0; i < kAttnChunk / 32; ++i) {
+        for (int i = 0; i < kMaxParts / 32; ++i) {
             const int s = lane + 32 * i;
             const float w = ml[i].x == -INFINITY ? 0.f : expf(ml[i].x - m);   // a part without tokens carries nothing
             if (s < n_parts) sc[warp][s] = w;
@@ -493,7 +475,7 @@ __global__ void __launch_bounds__(kThreads) attn_decode_kernel(AttnCache c, cons
 
 }  // namespace
 
-constexpr size_t kDynSmem = 2 * 2 * (size_t)kTile * kD;   // two stages of key and value rows
+constexpr size_t kDynSmem = kRowBytes + (size_t)8 * kAttnMaxRep * (kD + 4) * sizeof(float);   // row stages, then the parts of a cluster's CTAs
 
 template <int REP>
 static cudaError_t ensure_smem() {
