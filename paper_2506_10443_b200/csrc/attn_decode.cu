@@ -23,7 +23,6 @@ namespace {
 
 constexpr int kD = kAttnHeadDim;
 constexpr int kThreads = 256;
-constexpr int kMaxParts = 32;   // parts per kv head that reach the final merge (256 CTAs in clusters of eight, or fewer than 16 single CTAs)
 constexpr int kTile = 128;   // tokens per stage of the row buffers (two stages)
 constexpr size_t kRowBytes = 2 * 2 * (size_t)kTile * 128;   // two stages of key and value rows
 
@@ -120,7 +119,6 @@ template <int REP>
 __global__ void __launch_bounds__(kThreads) attn_decode_kernel(AttnCache c, const __half* __restrict__ q, void* out,
                                                                int out_dtype, int S, int per_split, float* partials,
                                                                unsigned int* counters, uint32_t* status) {
-    __shared__ float sc[REP][kMaxParts];    // final merge: the parts' weights
     __shared__ float m_run[REP], l_run[REP];
     __shared__ __align__(16) float ps[kThreads / 32][REP * 16 + 8];   // per warp: weights of its 16 tokens, rescale factors
     __shared__ float wm[kThreads / 32][REP], wl[kThreads / 32][REP];  // the warps' maxima and sums, merged at the end
@@ -406,69 +404,52 @@ __global__ void __launch_bounds__(kThreads) attn_decode_kernel(AttnCache c, cons
     if (tid == 0) last_flag = !dead && atomicAdd(counters + hk, 1u) == (unsigned int)n_parts - 1u;
     __syncthreads();
     if (!last_flag) return;
-    // ---- the last CTA of the kv head merges the parts, in the order of the splits (the same sum
-    // whoever comes last), and clears the counter for the next call
+    // ---- the last CTA of the kv head merges the parts, in the order of the parts (the same sum
+    // whoever comes last), and clears the counter for the next call.  One thread per (head, four
+    // entries): all of its loads are issued before any is used, 16 parts at a time, so the merge is
+    // one round trip to L2; no shared memory, no barrier.
     __threadfence();
     if (tid == 0) counters[hk] = 0u;
     const float* parts = partials + ((size_t)hk * n_parts * REP) * kPart;
-    // warp h: head h's {m, l} of every part in one pass of loads (n_parts <= 256: eight per lane), the
-    // overall maximum, every part's weight exp(m_s - m) (into sc) and the sum of the weighted l_s
-    if (warp < REP) {
-        float2 ml[kMaxParts / 32];
+    for (int idx = tid; idx < REP * 32; idx += kThreads) {
+        const int h = idx >> 5;
+        float m = -INFINITY, l = 0.f, a4[4] = {0.f, 0.f, 0.f, 0.f};
+        for (int s0 = 0; s0 < n_parts; s0 += 16) {
+            float2 ml[16], lo[16], hi[16];
 #pragma unroll
-        for (int i = 0; i < kMaxParts / 32; ++i) {
-            const int s = lane + 32 * i;
-            ml[i] = s < n_parts ? __ldcg(reinterpret_cast<const float2*>(parts + ((size_t)s * REP + warp) * kPart))
-                                 : make_float2(-INFINITY, 0.f);
+            for (int i = 0; i < 16; ++i) {
+                ml[i] = make_float2(-INFINITY, 0.f);
+                lo[i] = hi[i] = make_float2(0.f, 0.f);
+                if (s0 + i < n_parts) {
+                    const float* ps_ = parts + ((size_t)(s0 + i) * REP + h) * kPart;
+                    ml[i] = __ldcg(reinterpret_cast<const float2*>(ps_));
+                    lo[i] = __ldcg(reinterpret_cast<const float2*>(ps_ + 2 + lane * 4));
+                    hi[i] = __ldcg(reinterpret_cast<const float2*>(ps_ + 4 + lane * 4));
+                }
+            }
+            float m_new = m;
+#pragma unroll
+            for (int i = 0; i < 16; ++i) m_new = fmaxf(m_new, ml[i].x);
+            const float r = m == -INFINITY ? 0.f : expf(m - m_new);   // what has been summed so far
+            l *= r;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) a4[i] *= r;
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const float w = ml[i].x == -INFINITY ? 0.f : expf(ml[i].x - m_new);   // a part without tokens carries nothing
+                l = fmaf(ml[i].y, w, l);
+                a4[0] = fmaf(lo[i].x, w, a4[0]); a4[1] = fmaf(lo[i].y, w, a4[1]);
+                a4[2] = fmaf(hi[i].x, w, a4[2]); a4[3] = fmaf(hi[i].y, w, a4[3]);
+            }
+            m = m_new;
         }
-        float m = -INFINITY;
+        const size_t o = (size_t)(hk * REP + h) * kD + lane * 4;
 #pragma unroll
-        for (int i = 0; i < kMaxParts / 32; ++i) m = fmaxf(m, ml[i].x);
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-        float l = 0.f;
-#pragma unroll
-        for (int i = 0; i < kMaxParts / 32; ++i) {
-            const int s = lane + 32 * i;
-            const float w = ml[i].x == -INFINITY ? 0.f : expf(ml[i].x - m);   // a part without tokens carries nothing
-            if (s < n_parts) sc[warp][s] = w;
-            l = fmaf(ml[i].y, w, l);
+        for (int i = 0; i < 4; ++i) {
+            const float r = a4[i] / l;
+            if (out_dtype == MNNLLM_F32) reinterpret_cast<float*>(out)[o + i] = r;
+            else reinterpret_cast<__half*>(out)[o + i] = __float2half_rn(r);
         }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
-        if (lane == 0) l_run[warp] = l;
-    }
-    __syncthreads();
-    // the weighted sum of the parts' accumulators: warp w takes parts w, w + 8, ... for all heads (a lane
-    // four entries: one 512-byte row of a part per pair of loads, REP rows per part in flight together);
-    // then the eight warps' sums are added in a fixed order through the row buffers, which are free now
-    float4 a[REP];
-#pragma unroll
-    for (int h = 0; h < REP; ++h) a[h] = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll 2
-    for (int s = warp; s < n_parts; s += 8) {
-#pragma unroll
-        for (int h = 0; h < REP; ++h) {
-            const float* ps = parts + ((size_t)s * REP + h) * kPart + 2 + lane * 4;   // 8 bytes into a part
-            const float w = sc[h][s];
-            const float2 lo = __ldcg(reinterpret_cast<const float2*>(ps)), hi = __ldcg(reinterpret_cast<const float2*>(ps + 2));
-            a[h].x = fmaf(lo.x, w, a[h].x); a[h].y = fmaf(lo.y, w, a[h].y);
-            a[h].z = fmaf(hi.x, w, a[h].z); a[h].w = fmaf(hi.y, w, a[h].w);
-        }
-    }
-    float* mrg = reinterpret_cast<float*>(dyn);   // [8 warps][REP][128]
-#pragma unroll
-    for (int h = 0; h < REP; ++h) *reinterpret_cast<float4*>(mrg + ((warp * REP + h) * kD) + lane * 4) = a[h];
-    __syncthreads();
-    for (int o = tid; o < REP * kD; o += kThreads) {
-        const int h = o / kD;
-        float sum = 0.f;
-#pragma unroll
-        for (int w = 0; w < 8; ++w) sum += mrg[w * REP * kD + o];
-        const float r = sum / l_run[h];
-        const size_t idx = (size_t)(hk * REP) * kD + o;
-        if (out_dtype == MNNLLM_F32) reinterpret_cast<float*>(out)[idx] = r;
-        else reinterpret_cast<__half*>(out)[idx] = __float2half_rn(r);
     }
     (void)status;
 }
